@@ -1,0 +1,209 @@
+/*
+ * amk.h -- C ABI of the B200 single-kernel Llama decode library.
+ *
+ * What the library does (the paper's statement of the problem, Sections 1, 3 and 4): the weights of a
+ * bias-free, full-rotary, SiLU-SwiGLU, RMSNorm, grouped-query-attention Llama-family decoder are laid
+ * out once; afterwards ONE launch of one persistent cooperative kernel is one forward pass is one
+ * decoded token (batch 1), with the KV cache persisting in device memory between launches.  Weight-only
+ * int8 and int4 variants fold the dequantisation into the matrix-vector products while embeddings,
+ * scales and every non-GEMV buffer keep their 16-bit types (Section 5, "Quantized generation").
+ *
+ * Conventions for every entry point
+ *   - Plain C, no exceptions, no aborts: every call returns an amk_status.
+ *   - Pointers are tagged HOST or DEVICE in the comments.  The library never allocates or frees device
+ *     memory: the caller owns the canonical weights, the packed buffer, the workspace, the KV cache and
+ *     the outputs.  (The handle and a few small host tables are the only allocations.)
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - One handle is used from one stream at a time; several handles may coexist.
+ *   - Same inputs give bit-identical outputs (no floating-point atomics, fixed reduction orders).
+ */
+#ifndef AMK_H
+#define AMK_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define AMK_ABI_VERSION 1u
+
+typedef enum {
+  AMK_OK = 0,
+  AMK_ERR_INVALID_ARG = 1, /* NULL pointer, bad struct_size / abi_version, buffer too small            */
+  AMK_ERR_UNSUPPORTED = 2, /* a shape or option the kernel's plan cannot serve                          */
+  AMK_ERR_CUDA = 3,        /* a CUDA runtime call failed (amk_last_status gives the text)               */
+  AMK_ERR_OOM = 4,         /* host allocation failed                                                    */
+  AMK_ERR_TIMEOUT = 5,     /* a bounded device-side wait expired (read through amk_last_status)         */
+  AMK_ERR_ABORTED = 6,     /* the kernel left early because another block reported an error             */
+  AMK_ERR_BAD_POS = 7,     /* pos < 0 or pos >= max_seq                                                 */
+  AMK_ERR_BAD_TOKEN = 8    /* token < 0 or token >= vocab                                               */
+} amk_status;
+
+typedef enum { AMK_W_BF16 = 0, AMK_W_INT8 = 1, AMK_W_INT4 = 2 } amk_wdtype;
+
+/* amk_config.flags */
+#define AMK_FLAG_DEBUG_HIDDEN 1u /* keep the residual stream after the embedding and after every layer */
+
+/* The seven per-layer linears, in the order used by amk_weights.linear[] and amk_debug_unpack. */
+enum { AMK_LIN_Q = 0, AMK_LIN_K = 1, AMK_LIN_V = 2, AMK_LIN_O = 3, AMK_LIN_GATE = 4, AMK_LIN_UP = 5,
+       AMK_LIN_DOWN = 6, AMK_LIN_COUNT = 7, AMK_LIN_LM_HEAD = 7 };
+
+/* Model and plan description.  POD; the Python mirror is checked against sizeof/offsetof. */
+typedef struct amk_config {
+  uint32_t struct_size;      /* = sizeof(amk_config)                                                   */
+  uint32_t abi_version;      /* = AMK_ABI_VERSION                                                      */
+  uint32_t hidden;           /* H; multiple of 8 (16 for int8, 256 for int4)                           */
+  uint32_t n_layers;         /* L                                                                      */
+  uint32_t n_q_heads;        /* multiple of n_kv_heads; n_q_heads / n_kv_heads <= 16                   */
+  uint32_t n_kv_heads;
+  uint32_t head_dim;         /* 64 or 128                                                              */
+  uint32_t mlp;              /* I; same divisibility rule as hidden                                    */
+  uint32_t vocab;            /* V                                                                      */
+  uint32_t max_seq;          /* S: positions the KV cache holds                                        */
+  uint32_t tied_embeddings;  /* 1: the LM head is the embedding matrix                                 */
+  float rms_eps;             /* RMSNorm epsilon (inside the square root)                               */
+  float rope_theta;          /* rotary base; pairs (i, i + head_dim/2), no scaling                     */
+  uint32_t wdtype;           /* amk_wdtype of the seven per-layer linears                              */
+  uint32_t group_size;       /* int4: 128 (the only supported value); ignored otherwise                */
+  uint32_t quantize_lm_head; /* must be 0: embedding and LM head stay bf16, as in the paper            */
+  uint32_t wait_timeout_us;  /* bound on every device-side wait; 0 = 200000                            */
+  uint32_t flags;            /* AMK_FLAG_*                                                             */
+  /* tuning knobs, 0 = automatic */
+  uint32_t stage_bytes;      /* bytes per shared-memory ring stage (multiple of 1024)                  */
+  uint32_t n_stages;         /* ring depth                                                             */
+  uint32_t max_inflight;     /* bulk copies a block keeps in flight (<= n_stages)                      */
+  uint32_t reserved[3];      /* must be 0                                                              */
+} amk_config;
+
+/*
+ * Canonical (unpacked) weights: every data pointer is a DEVICE pointer to a row-major [out][in] array;
+ * the per-layer arrays are HOST arrays of n_layers device pointers.  They are read only inside
+ * amk_create and may be freed once the stream passed to amk_create has been synchronised.
+ *   bf16 : bf16 [out][in]
+ *   int8 : int8 [out][in]; scale fp16 [out]                       w = scale * q, q in [-127, 127]
+ *   int4 : uint8 [out][in/2], element j in byte j/2 (even j: bits 0-3); scale fp16 [out][in/128];
+ *          zero fp16 [out][in/128] holding an integer 0..15        w = scale * (q - zero)
+ */
+typedef struct amk_weights {
+  const void* embed;                        /* bf16 [V][H]                                            */
+  const void* lm_head;                      /* bf16 [V][H]; NULL when tied_embeddings                 */
+  const void* final_norm;                   /* bf16 [H]                                               */
+  const void* const* attn_norm;             /* [L] -> bf16 [H]                                        */
+  const void* const* mlp_norm;              /* [L] -> bf16 [H]                                        */
+  const void* const* linear[AMK_LIN_COUNT]; /* [L] each: q, k, v, o, gate, up, down                   */
+  const void* const* scale[AMK_LIN_COUNT];  /* [L] each; NULL arrays for bf16                         */
+  const void* const* zero[AMK_LIN_COUNT];   /* [L] each; int4 only                                    */
+} amk_weights;
+
+typedef struct amk_handle amk_handle;
+
+/* What the plan looks like; filled by amk_plan_info. */
+typedef struct amk_plan {
+  uint32_t n_blocks;          /* thread blocks = SMs used (one persistent block per SM)                */
+  uint32_t threads;           /* threads per block (one producer warp + consumer warps)                */
+  uint32_t smem_bytes;        /* dynamic shared memory per block                                       */
+  uint32_t stage_bytes, n_stages, max_inflight;
+  uint32_t n_gemv_ops;        /* 4 per layer + LM head                                                 */
+  uint32_t n_phases;          /* dependency joins per token                                            */
+  uint64_t packed_bytes, workspace_bytes, kv_bytes;
+  uint64_t weight_stream_bytes; /* packed weight + scale bytes each token streams                      */
+} amk_plan;
+
+const char* amk_status_str(amk_status s);
+
+/* Sizes of the three caller-owned device buffers for a configuration.  HOST pointers.
+ * Errors: INVALID_ARG (NULL, bad struct_size/abi_version), UNSUPPORTED (shape). */
+amk_status amk_packed_bytes(const amk_config* cfg, size_t* bytes);
+amk_status amk_workspace_bytes(const amk_config* cfg, size_t* bytes);
+amk_status amk_kv_bytes(const amk_config* cfg, size_t* bytes); /* K and V together */
+
+/*
+ * Build a decoder: validates the configuration, lays the weights out for streaming (the "weight
+ * packer": each block's tiles of each matrix-vector product become one contiguous byte run, column
+ * order permuted for conflict-free shared-memory reads, int4 scales and zero points interleaved with
+ * their codes), builds the per-op tables and the rotary table in the workspace, all on `cuda_stream`.
+ *   cfg, weights            HOST structs (weights' data pointers are DEVICE pointers)
+ *   packed_dev / workspace_dev   DEVICE, caller-owned, at least amk_packed_bytes / amk_workspace_bytes,
+ *                           256-byte aligned; must outlive the handle; the library fills them
+ *   out                     HOST: receives the handle
+ * The device must be a compute-capability-10.0 GPU that supports cooperative launch with one block per
+ * SM at the plan's shared-memory size; otherwise UNSUPPORTED.  Asynchronous on the stream apart from
+ * small synchronous table uploads.
+ */
+amk_status amk_create(const amk_config* cfg, const amk_weights* weights, void* packed_dev, size_t packed_bytes,
+                      void* workspace_dev, size_t workspace_bytes, void* cuda_stream, amk_handle** out);
+
+/*
+ * One decode step (Algorithm 1 of the paper: every block walks its queue -- wait, dispatch, signal --
+ * inside one cooperative launch): embedding of `token`, L decoder layers at position `pos`, final norm,
+ * LM head, greedy token.
+ *   kv_cache_dev   DEVICE, caller-owned, amk_kv_bytes: K then V, each [L][n_kv_heads][max_seq][head_dim]
+ *                  bf16.  Entries [0, pos) must be valid; the step writes slot `pos` of every layer (K after
+ *                  the rotation, round-to-nearest-even) and reads [0, pos].
+ *   logits_dev     DEVICE float[vocab], may be NULL
+ *   next_token_dev DEVICE int32[1], may be NULL; lowest index wins an exact tie
+ * Asynchronous: returns after the launch.  Synchronous errors: INVALID_ARG, BAD_POS, BAD_TOKEN, CUDA.
+ * A device-side failure (expired wait) is reported by amk_last_status after the stream has been
+ * synchronised; outputs of that step are then undefined, and the next step is legal.
+ */
+amk_status amk_decode_step(amk_handle* h, int32_t token, int32_t pos, void* kv_cache_dev, float* logits_dev,
+                           int32_t* next_token_dev, void* cuda_stream);
+
+/*
+ * `n_steps` greedy decode steps with the token fed back on the device (no host round trip between
+ * steps): step i decodes position pos0 + i; its input is `first_token` for i = 0 and the previous
+ * step's greedy token afterwards.  Goes beyond the paper, which stops at one launch per token and
+ * measures the host dispatch between launches separately (Section 5, "Methodology").
+ *   tokens_out_dev DEVICE int32[n_steps]: the greedy token of every step
+ *   logits_dev     DEVICE float[vocab] or NULL: logits of the LAST step
+ * Errors as amk_decode_step; BAD_POS if pos0 + n_steps > max_seq.
+ */
+amk_status amk_decode_greedy(amk_handle* h, int32_t first_token, int32_t pos0, int32_t n_steps, void* kv_cache_dev,
+                             int32_t* tokens_out_dev, float* logits_dev, void* cuda_stream);
+
+/* Synchronises the handle's last stream and reports the device status word of the last step.
+ *   st   HOST out: AMK_OK, AMK_ERR_TIMEOUT, ...      msg  HOST out, n bytes, may be NULL. */
+amk_status amk_last_status(amk_handle* h, amk_status* st, char* msg, size_t n);
+
+amk_status amk_plan_info(const amk_handle* h, amk_plan* out); /* HOST out */
+
+/* With AMK_FLAG_DEBUG_HIDDEN: copies the residual stream of the last step to HOST memory,
+ * float[(L+1)][H]: row 0 after the embedding, row l+1 after layer l.  Synchronises. */
+amk_status amk_debug_hidden(amk_handle* h, float* host_out);
+
+/* Inverse of the packer, for bit-exact layout checks: rebuilds one canonical matrix from the packed
+ * buffer into DEVICE memory of the canonical size.  which = AMK_LIN_* (AMK_LIN_LM_HEAD ignores layer).
+ *   out_dev    codes / bf16 in the canonical layout
+ *   scale_dev  fp16 scales in the canonical layout (int8 / int4), may be NULL
+ *   zero_dev   fp16 zero points (int4), may be NULL */
+amk_status amk_debug_unpack(amk_handle* h, int layer, int which, void* out_dev, void* scale_dev, void* zero_dev,
+                            void* cuda_stream);
+
+/* Test hook for the bounded-wait path: the next step's block `block` skips its signal of dependency
+ * join `phase`, so every waiter runs into the time limit and the step ends with AMK_ERR_TIMEOUT
+ * (nothing traps or hangs).  block < 0 clears the hook. */
+amk_status amk_debug_drop_signal(amk_handle* h, int phase, int block);
+
+/* Frees host state only.  The caller's buffers are untouched. */
+amk_status amk_destroy(amk_handle* h);
+
+/*
+ * Round-to-nearest weight quantisers on the device (the paper's "naive round-to-nearest", Section 5),
+ * bit-identical to their definition in IEEE fp32 arithmetic:
+ *   int8: s = fp16(max|w| / 127) per output row (1 if the row is zero); q = clamp(rint(w / s), -127, 127)
+ *   int4: per row and group of 128 columns, mn = min(w, 0), mx = max(w, 0); s = fp16((mx - mn) / 15)
+ *         (1 if mx == mn); z = clamp(rint(-mn / s), 0, 15); q = clamp(rint(w / s) + z, 0, 15);
+ *         two codes per byte, even column in the low nibble; z stored as an fp16 integer.
+ * All pointers DEVICE; w_bf16 is [rows][cols] bf16.  cols % 128 == 0 for int4.  Asynchronous.
+ */
+amk_status amk_quantize_int8(const void* w_bf16, int64_t rows, int64_t cols, void* q_out, void* scale_out,
+                             void* cuda_stream);
+amk_status amk_quantize_int4(const void* w_bf16, int64_t rows, int64_t cols, void* packed_out, void* scale_out,
+                             void* zero_out, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AMK_H */

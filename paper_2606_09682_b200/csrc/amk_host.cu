@@ -1,0 +1,525 @@
+// Host side of the C ABI (include/amk.h): configuration checks, the plan (tables, buffer layouts), the
+// weight packer's driver, and the launch of the decode kernel.  Nothing here computes any part of the
+// decode step: every step of the path runs in the kernels.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "amk.h"
+#include "amk_internal.h"
+
+using namespace amk;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr int kMaxBlocks = 512;   // upper bound on SMs, for sizing the per-block candidate arrays
+inline size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a; }
+
+struct PackedLayout {
+  std::vector<OpDesc> ops;      // packed_off / scale_off filled
+  size_t embed_off, attn_norm_off, mlp_norm_off, final_norm_off, total;
+  size_t weight_stream_bytes;   // op regions + scale regions (what a token streams)
+};
+
+struct WorkspaceLayout {
+  size_t status, phase_ctr, group_ctr, lm_ctr, next_ws, cand_val, cand_idx, ops, x_a, x_b, qkv, o, m, part, hidden,
+      rope, total;
+};
+
+amk_status check_config(const amk_config* c) {
+  if (!c) return AMK_ERR_INVALID_ARG;
+  if (c->struct_size != sizeof(amk_config) || c->abi_version != AMK_ABI_VERSION) return AMK_ERR_INVALID_ARG;
+  for (uint32_t r : c->reserved) if (r) return AMK_ERR_INVALID_ARG;
+  if (!c->hidden || !c->n_layers || !c->n_q_heads || !c->n_kv_heads || !c->mlp || !c->vocab || !c->max_seq)
+    return AMK_ERR_INVALID_ARG;
+  if (c->wdtype > AMK_W_INT4) return AMK_ERR_INVALID_ARG;
+  if (c->head_dim != 64 && c->head_dim != 128) return AMK_ERR_UNSUPPORTED;
+  if (c->n_q_heads % c->n_kv_heads) return AMK_ERR_UNSUPPORTED;
+  if (c->n_q_heads / c->n_kv_heads > (uint32_t)kMaxRep) return AMK_ERR_UNSUPPORTED;
+  if (c->quantize_lm_head) return AMK_ERR_UNSUPPORTED;
+  const uint32_t kdiv = c->wdtype == AMK_W_BF16 ? 8 : (c->wdtype == AMK_W_INT8 ? 16 : 256);
+  const uint32_t qdim = c->n_q_heads * c->head_dim;
+  if (c->hidden % kdiv || c->mlp % kdiv || qdim % kdiv) return AMK_ERR_UNSUPPORTED;
+  if (c->hidden % 8) return AMK_ERR_UNSUPPORTED;                      // LM head is bf16
+  if (c->hidden > (uint32_t)(4 * kConsumerThreads * 4)) return AMK_ERR_UNSUPPORTED;   // norm prologue register budget
+  if (c->wdtype == AMK_W_INT4 && c->group_size != 128) return AMK_ERR_UNSUPPORTED;
+  if (c->wdtype == AMK_W_INT4 && (c->hidden % 2)) return AMK_ERR_UNSUPPORTED;
+  if (c->n_kv_heads > (uint32_t)kMaxBlocks) return AMK_ERR_UNSUPPORTED;
+  if ((uint64_t)c->vocab * c->hidden > (1ull << 40)) return AMK_ERR_UNSUPPORTED;
+  if (c->stage_bytes && (c->stage_bytes % 1024 || c->stage_bytes < 8192 || c->stage_bytes > 65536))
+    return AMK_ERR_INVALID_ARG;
+  if (c->n_stages > (uint32_t)kMaxStages || c->n_stages == 1) return AMK_ERR_INVALID_ARG;
+  return AMK_OK;
+}
+
+uint32_t stage_bytes_of(const amk_config* c) { return c->stage_bytes ? c->stage_bytes : 32768u; }
+
+// Op table and packed-buffer layout (independent of the number of blocks: rows keep their byte size).
+PackedLayout packed_layout(const amk_config* c) {
+  PackedLayout pl;
+  const int H = c->hidden, L = c->n_layers, I = c->mlp, V = c->vocab;
+  const int qd = c->n_q_heads * c->head_dim, kvd = c->n_kv_heads * c->head_dim;
+  const int wd = (int)c->wdtype;
+  const int ur = (wd == W_INT4) ? 2 : 1;
+  size_t off = 0;
+  auto add = [&](int kind, int layer, int K, int rows, int unit_rows, int wdt) {
+    OpDesc d;
+    memset(&d, 0, sizeof(d));
+    d.kind = kind; d.layer = layer; d.K = K; d.rows = rows; d.unit_rows = unit_rows; d.wdtype = wdt;
+    d.rot = (int)((pl.ops.size() * 37u) % 9973u);      // reduced modulo the block count at create time
+    d.packed_off = off;
+    off = align_up(off + (size_t)rows * (size_t)row_bytes(wdt, K));
+    pl.ops.push_back(d);
+  };
+  for (int l = 0; l < L; l++) {
+    add(OP_QKV, l, H, qd + 2 * kvd, ur, wd);
+    add(OP_O, l, qd, H, ur, wd);
+    add(OP_GATEUP, l, H, 2 * I, 2, wd);
+    add(OP_DOWN, l, I, H, ur, wd);
+  }
+  add(OP_LMHEAD, L, H, V, 1, W_BF16);
+  if (wd == W_INT8) {
+    for (auto& d : pl.ops) {
+      if (d.wdtype != W_INT8) continue;
+      d.scale_off = off;
+      off = align_up(off + (size_t)d.rows * 2);
+    }
+  }
+  pl.weight_stream_bytes = off;
+  pl.embed_off = off;      off = align_up(off + (size_t)V * H * 2);
+  pl.attn_norm_off = off;  off = align_up(off + (size_t)L * H * 2);
+  pl.mlp_norm_off = off;   off = align_up(off + (size_t)L * H * 2);
+  pl.final_norm_off = off; off = align_up(off + (size_t)H * 2);
+  pl.total = off;
+  return pl;
+}
+
+WorkspaceLayout workspace_layout(const amk_config* c) {
+  WorkspaceLayout w;
+  const size_t H = c->hidden, L = c->n_layers, I = c->mlp, S = c->max_seq, hd = c->head_dim;
+  const size_t qd = (size_t)c->n_q_heads * hd, kvd = (size_t)c->n_kv_heads * hd;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  w.status = take(sizeof(DevStatus));
+  w.phase_ctr = take(5 * L * 4);
+  w.group_ctr = take((size_t)c->n_kv_heads * 4);
+  w.lm_ctr = take(4);
+  w.next_ws = take(4);
+  w.cand_val = take(kMaxBlocks * 4);
+  w.cand_idx = take(kMaxBlocks * 4);
+  w.ops = take((4 * L + 1) * sizeof(OpDesc));
+  w.x_a = take(H * 4);
+  w.x_b = take(H * 4);
+  w.qkv = take((qd + 2 * kvd) * 4);
+  w.o = take(qd * 4);
+  w.m = take(I * 4);
+  w.part = take((size_t)c->n_q_heads * kMaxChunks * (hd + 2) * 4);
+  w.hidden = take((L + 1) * H * 4);
+  w.rope = take(S * (hd / 2) * sizeof(float2));
+  w.total = off;
+  return w;
+}
+
+size_t kv_bytes_of(const amk_config* c) {
+  return 2ull * c->n_layers * c->n_kv_heads * c->max_seq * c->head_dim * 2ull;
+}
+
+}  // namespace
+
+struct amk_handle {
+  amk_config cfg;
+  amk_plan plan;
+  PackedLayout pl;
+  WorkspaceLayout wl;
+  unsigned char* packed;
+  unsigned char* ws;
+  KParams base;            // everything but the per-step fields
+  unsigned epoch;
+  cudaStream_t last_stream;
+  int drop_phase, drop_block;
+  char errmsg[256];
+};
+
+extern "C" {
+
+const char* amk_status_str(amk_status s) {
+  switch (s) {
+    case AMK_OK: return "ok";
+    case AMK_ERR_INVALID_ARG: return "invalid argument";
+    case AMK_ERR_UNSUPPORTED: return "unsupported configuration";
+    case AMK_ERR_CUDA: return "CUDA error";
+    case AMK_ERR_OOM: return "out of host memory";
+    case AMK_ERR_TIMEOUT: return "device-side wait timed out";
+    case AMK_ERR_ABORTED: return "aborted";
+    case AMK_ERR_BAD_POS: return "position out of range";
+    case AMK_ERR_BAD_TOKEN: return "token out of range";
+  }
+  return "unknown status";
+}
+
+amk_status amk_packed_bytes(const amk_config* cfg, size_t* bytes) {
+  if (!bytes) return AMK_ERR_INVALID_ARG;
+  amk_status st = check_config(cfg);
+  if (st != AMK_OK) return st;
+  *bytes = packed_layout(cfg).total;
+  return AMK_OK;
+}
+
+amk_status amk_workspace_bytes(const amk_config* cfg, size_t* bytes) {
+  if (!bytes) return AMK_ERR_INVALID_ARG;
+  amk_status st = check_config(cfg);
+  if (st != AMK_OK) return st;
+  *bytes = workspace_layout(cfg).total;
+  return AMK_OK;
+}
+
+amk_status amk_kv_bytes(const amk_config* cfg, size_t* bytes) {
+  if (!bytes) return AMK_ERR_INVALID_ARG;
+  amk_status st = check_config(cfg);
+  if (st != AMK_OK) return st;
+  *bytes = kv_bytes_of(cfg);
+  return AMK_OK;
+}
+
+#define AMK_CUDA(call)                                                                       \
+  do {                                                                                       \
+    cudaError_t e_ = (call);                                                                 \
+    if (e_ != cudaSuccess) {                                                                 \
+      if (h) snprintf(h->errmsg, sizeof(h->errmsg), "%s: %s", #call, cudaGetErrorString(e_)); \
+      status = AMK_ERR_CUDA;                                                                 \
+      goto fail;                                                                             \
+    }                                                                                        \
+  } while (0)
+
+amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packed_dev, size_t packed_bytes,
+                      void* workspace_dev, size_t workspace_bytes, void* cuda_stream, amk_handle** out) {
+  if (!out) return AMK_ERR_INVALID_ARG;
+  *out = nullptr;
+  amk_status status = check_config(cfg);
+  if (status != AMK_OK) return status;
+  if (!wts || !packed_dev || !workspace_dev) return AMK_ERR_INVALID_ARG;
+  if (((uintptr_t)packed_dev | (uintptr_t)workspace_dev) & (kAlign - 1)) return AMK_ERR_INVALID_ARG;
+  if (!wts->embed || !wts->final_norm || !wts->attn_norm || !wts->mlp_norm) return AMK_ERR_INVALID_ARG;
+  if (!cfg->tied_embeddings && !wts->lm_head) return AMK_ERR_INVALID_ARG;
+  for (int k = 0; k < AMK_LIN_COUNT; k++) {
+    if (!wts->linear[k]) return AMK_ERR_INVALID_ARG;
+    if (cfg->wdtype != AMK_W_BF16 && !wts->scale[k]) return AMK_ERR_INVALID_ARG;
+    if (cfg->wdtype == AMK_W_INT4 && !wts->zero[k]) return AMK_ERR_INVALID_ARG;
+  }
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  amk_handle* h = new (std::nothrow) amk_handle();
+  if (!h) return AMK_ERR_OOM;
+  h->cfg = *cfg;
+  h->pl = packed_layout(cfg);
+  h->wl = workspace_layout(cfg);
+  h->packed = (unsigned char*)packed_dev;
+  h->ws = (unsigned char*)workspace_dev;
+  h->drop_phase = -1;
+  h->drop_block = -1;
+  h->last_stream = stream;
+  {
+    if (packed_bytes < h->pl.total || workspace_bytes < h->wl.total) { status = AMK_ERR_INVALID_ARG; goto fail; }
+    int dev = 0, sms = 0, coop = 0, smem_optin = 0, cc_major = 0;
+    AMK_CUDA(cudaGetDevice(&dev));
+    AMK_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    AMK_CUDA(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
+    AMK_CUDA(cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    AMK_CUDA(cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev));
+    if (cc_major != 10 || !coop || sms < 1 || sms > kMaxBlocks || (int)cfg->n_kv_heads > sms) {
+      snprintf(h->errmsg, sizeof(h->errmsg), "needs a compute-capability-10.x GPU with cooperative launch");
+      status = AMK_ERR_UNSUPPORTED;
+      goto fail;
+    }
+    const int n_blocks = sms;
+    const int H = cfg->hidden, L = cfg->n_layers, I = cfg->mlp, hd = cfg->head_dim;
+    const int qd = cfg->n_q_heads * hd, n_rep = cfg->n_q_heads / cfg->n_kv_heads;
+
+    // ---- shared-memory plan -----------------------------------------------------------------------
+    const size_t hdr = (sizeof(SmemHeader) + 127) & ~(size_t)127;
+    size_t kmax = (size_t)(H > I ? H : I);
+    if ((size_t)qd > kmax) kmax = qd;
+    size_t act = kmax * 4;
+    const size_t attn_need = ((size_t)n_rep * hd + (size_t)kConsumerWarps * 4 * (hd + 2)) * 4;
+    if (attn_need > act) act = attn_need;
+    act = (act + 127) & ~(size_t)127;
+    const uint32_t stage_bytes = stage_bytes_of(cfg);
+    uint32_t n_stages = cfg->n_stages;
+    const size_t avail = (size_t)smem_optin > hdr + act ? (size_t)smem_optin - hdr - act : 0;
+    const uint32_t fit = (uint32_t)(avail / stage_bytes);
+    if (n_stages == 0) n_stages = fit < (uint32_t)kMaxStages ? fit : (uint32_t)kMaxStages;
+    if (n_stages < 2 || n_stages > fit) {
+      snprintf(h->errmsg, sizeof(h->errmsg), "shared-memory plan does not fit: need %zu + %u stages of %u, have %d",
+               hdr + act, n_stages, stage_bytes, smem_optin);
+      status = AMK_ERR_UNSUPPORTED;
+      goto fail;
+    }
+    uint32_t max_inflight = cfg->max_inflight ? cfg->max_inflight : n_stages;
+    if (max_inflight > n_stages) max_inflight = n_stages;
+    const size_t smem_bytes = hdr + act + (size_t)n_stages * stage_bytes;
+    int per_sm = 0;
+    AMK_CUDA(decode_kernel_attrs(smem_bytes, &per_sm));
+    if (per_sm < 1) {
+      snprintf(h->errmsg, sizeof(h->errmsg), "decode kernel does not fit one block per SM");
+      status = AMK_ERR_UNSUPPORTED;
+      goto fail;
+    }
+
+    // ---- op table, rotations reduced modulo the block count ------------------------------------------
+    for (auto& d : h->pl.ops) d.rot = d.rot % n_blocks;
+    AMK_CUDA(cudaMemsetAsync(h->ws, 0, h->wl.total, stream));
+    AMK_CUDA(cudaMemcpyAsync(h->ws + h->wl.ops, h->pl.ops.data(), h->pl.ops.size() * sizeof(OpDesc),
+                             cudaMemcpyHostToDevice, stream));
+
+    // ---- rotary table (cos, sin)[pos][i], angles formed in double --------------------------------------
+    {
+      const int half = hd / 2;
+      std::vector<float2> tab((size_t)cfg->max_seq * half);
+      for (int i = 0; i < half; i++) {
+        const double f = std::pow((double)cfg->rope_theta, -2.0 * (double)i / (double)hd);
+        for (uint32_t s = 0; s < cfg->max_seq; s++) {
+          const double phi = (double)s * f;
+          tab[(size_t)s * half + i] = make_float2((float)std::cos(phi), (float)std::sin(phi));
+        }
+      }
+      AMK_CUDA(cudaMemcpyAsync(h->ws + h->wl.rope, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice,
+                               stream));
+      AMK_CUDA(cudaStreamSynchronize(stream));     // `tab` and the op table are pageable host memory
+    }
+
+    // ---- pack the weights ---------------------------------------------------------------------------------
+    for (size_t i = 0; i < h->pl.ops.size(); i++) {
+      const OpDesc& d = h->pl.ops[i];
+      PackSrc s;
+      memset(&s, 0, sizeof(s));
+      const int l = d.layer;
+      auto lin = [&](int slot, int which) {
+        s.w[slot] = wts->linear[which][l];
+        s.scale[slot] = (cfg->wdtype != AMK_W_BF16) ? wts->scale[which][l] : nullptr;
+        s.zero[slot] = (cfg->wdtype == AMK_W_INT4) ? wts->zero[which][l] : nullptr;
+        return s.w[slot] && (cfg->wdtype == AMK_W_BF16 || s.scale[slot]) && (cfg->wdtype != AMK_W_INT4 || s.zero[slot]);
+      };
+      bool okp = true;
+      switch (d.kind) {
+        case OP_QKV:
+          s.mode = 1; s.rows0 = qd; s.rows1 = qd + cfg->n_kv_heads * hd;
+          okp = lin(0, AMK_LIN_Q) & lin(1, AMK_LIN_K) & lin(2, AMK_LIN_V);
+          break;
+        case OP_O: okp = lin(0, AMK_LIN_O); break;
+        case OP_GATEUP: s.mode = 2; okp = lin(0, AMK_LIN_GATE) & lin(1, AMK_LIN_UP); break;
+        case OP_DOWN: okp = lin(0, AMK_LIN_DOWN); break;
+        default: s.w[0] = cfg->tied_embeddings ? wts->embed : wts->lm_head; break;
+      }
+      if (!okp) { status = AMK_ERR_INVALID_ARG; goto fail; }
+      AMK_CUDA(launch_pack(d, s, h->packed, n_blocks, (int)stage_bytes, false, stream));
+    }
+    AMK_CUDA(cudaMemcpyAsync(h->packed + h->pl.embed_off, wts->embed, (size_t)cfg->vocab * H * 2,
+                             cudaMemcpyDeviceToDevice, stream));
+    AMK_CUDA(cudaMemcpyAsync(h->packed + h->pl.final_norm_off, wts->final_norm, (size_t)H * 2,
+                             cudaMemcpyDeviceToDevice, stream));
+    for (int l = 0; l < L; l++) {
+      if (!wts->attn_norm[l] || !wts->mlp_norm[l]) { status = AMK_ERR_INVALID_ARG; goto fail; }
+      AMK_CUDA(cudaMemcpyAsync(h->packed + h->pl.attn_norm_off + (size_t)l * H * 2, wts->attn_norm[l], (size_t)H * 2,
+                               cudaMemcpyDeviceToDevice, stream));
+      AMK_CUDA(cudaMemcpyAsync(h->packed + h->pl.mlp_norm_off + (size_t)l * H * 2, wts->mlp_norm[l], (size_t)H * 2,
+                               cudaMemcpyDeviceToDevice, stream));
+    }
+
+    // ---- kernel parameters that do not change from step to step ---------------------------------------
+    KParams& p = h->base;
+    p.H = H; p.L = L; p.nq = cfg->n_q_heads; p.nkv = cfg->n_kv_heads; p.hd = hd; p.I = I; p.V = cfg->vocab;
+    p.S = cfg->max_seq; p.n_rep = n_rep; p.eps = cfg->rms_eps; p.flags = (int)cfg->flags;
+    p.ops = (const OpDesc*)(h->ws + h->wl.ops);
+    p.n_ops = (int)h->pl.ops.size();
+    p.packed = h->packed;
+    p.embed = (const unsigned short*)(h->packed + h->pl.embed_off);
+    p.attn_norm = (const unsigned short*)(h->packed + h->pl.attn_norm_off);
+    p.mlp_norm = (const unsigned short*)(h->packed + h->pl.mlp_norm_off);
+    p.final_norm = (const unsigned short*)(h->packed + h->pl.final_norm_off);
+    p.rope = (const float2*)(h->ws + h->wl.rope);
+    p.x_a = (float*)(h->ws + h->wl.x_a); p.x_b = (float*)(h->ws + h->wl.x_b);
+    p.qkv = (float*)(h->ws + h->wl.qkv); p.o = (float*)(h->ws + h->wl.o); p.m = (float*)(h->ws + h->wl.m);
+    p.part = (float*)(h->ws + h->wl.part); p.hidden = (float*)(h->ws + h->wl.hidden);
+    p.phase_ctr = (unsigned*)(h->ws + h->wl.phase_ctr); p.group_ctr = (unsigned*)(h->ws + h->wl.group_ctr);
+    p.lm_ctr = (unsigned*)(h->ws + h->wl.lm_ctr); p.cand_val = (float*)(h->ws + h->wl.cand_val);
+    p.cand_idx = (int*)(h->ws + h->wl.cand_idx); p.next_ws = (int*)(h->ws + h->wl.next_ws);
+    p.status = (DevStatus*)(h->ws + h->wl.status);
+    p.stage_bytes = (int)stage_bytes; p.n_stages = (int)n_stages; p.max_inflight = (int)max_inflight;
+    p.act_bytes = (int)act;
+    p.timeout_ns = 1000ull * (cfg->wait_timeout_us ? cfg->wait_timeout_us : 200000u);
+    p.drop_phase = -1; p.drop_block = -1;
+
+    amk_plan& pn = h->plan;
+    pn.n_blocks = n_blocks; pn.threads = kThreads; pn.smem_bytes = (uint32_t)smem_bytes;
+    pn.stage_bytes = stage_bytes; pn.n_stages = n_stages; pn.max_inflight = max_inflight;
+    pn.n_gemv_ops = (uint32_t)h->pl.ops.size(); pn.n_phases = 5 * L;
+    pn.packed_bytes = h->pl.total; pn.workspace_bytes = h->wl.total; pn.kv_bytes = kv_bytes_of(cfg);
+    pn.weight_stream_bytes = h->pl.weight_stream_bytes;
+    h->epoch = 0;
+  }
+  *out = h;
+  return AMK_OK;
+fail:
+  if (getenv("AMK_VERBOSE")) fprintf(stderr, "amk_create: %s: %s\n", amk_status_str(status), h->errmsg);
+  delete h;
+  return status;
+}
+
+static amk_status launch_step(amk_handle* h, int32_t token, const int* token_ptr, int32_t pos, void* kv, float* logits,
+                              int32_t* next_token, cudaStream_t stream) {
+  KParams p = h->base;
+  p.token = token;
+  p.token_ptr = token_ptr;
+  p.pos = pos;
+  p.epoch = ++h->epoch;
+  const size_t half = kv_bytes_of(&h->cfg) / 2;
+  p.kcache = (unsigned short*)kv;
+  p.vcache = (unsigned short*)((unsigned char*)kv + half);
+  p.logits = logits;
+  p.next_token = next_token;
+  p.drop_phase = h->drop_phase;
+  p.drop_block = h->drop_block;
+  h->drop_phase = h->drop_block = -1;
+  h->last_stream = stream;
+  cudaError_t e = launch_decode(p, (int)h->plan.n_blocks, h->plan.smem_bytes, stream);
+  if (e != cudaSuccess) {
+    --h->epoch;
+    snprintf(h->errmsg, sizeof(h->errmsg), "cooperative launch: %s", cudaGetErrorString(e));
+    return AMK_ERR_CUDA;
+  }
+  return AMK_OK;
+}
+
+amk_status amk_decode_step(amk_handle* h, int32_t token, int32_t pos, void* kv_cache_dev, float* logits_dev,
+                           int32_t* next_token_dev, void* cuda_stream) {
+  if (!h || !kv_cache_dev) return AMK_ERR_INVALID_ARG;
+  if (pos < 0 || (uint32_t)pos >= h->cfg.max_seq) return AMK_ERR_BAD_POS;
+  if (token < 0 || (uint32_t)token >= h->cfg.vocab) return AMK_ERR_BAD_TOKEN;
+  return launch_step(h, token, nullptr, pos, kv_cache_dev, logits_dev, next_token_dev, (cudaStream_t)cuda_stream);
+}
+
+amk_status amk_decode_greedy(amk_handle* h, int32_t first_token, int32_t pos0, int32_t n_steps, void* kv_cache_dev,
+                             int32_t* tokens_out_dev, float* logits_dev, void* cuda_stream) {
+  if (!h || !kv_cache_dev || !tokens_out_dev || n_steps < 1) return AMK_ERR_INVALID_ARG;
+  if (pos0 < 0 || (uint64_t)pos0 + (uint64_t)n_steps > h->cfg.max_seq) return AMK_ERR_BAD_POS;
+  if (first_token < 0 || (uint32_t)first_token >= h->cfg.vocab) return AMK_ERR_BAD_TOKEN;
+  for (int i = 0; i < n_steps; i++) {
+    amk_status st = launch_step(h, first_token, i ? tokens_out_dev + (i - 1) : nullptr, pos0 + i, kv_cache_dev,
+                                (i == n_steps - 1) ? logits_dev : nullptr, tokens_out_dev + i, (cudaStream_t)cuda_stream);
+    if (st != AMK_OK) return st;
+  }
+  return AMK_OK;
+}
+
+amk_status amk_last_status(amk_handle* h, amk_status* st, char* msg, size_t n) {
+  if (!h || !st) return AMK_ERR_INVALID_ARG;
+  if (msg && n) msg[0] = 0;
+  cudaError_t e = cudaStreamSynchronize(h->last_stream);
+  DevStatus ds;
+  memset(&ds, 0, sizeof(ds));
+  if (e == cudaSuccess) e = cudaMemcpy(&ds, h->ws + h->wl.status, sizeof(ds), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) {
+    *st = AMK_ERR_CUDA;
+    if (msg && n) snprintf(msg, n, "%s", cudaGetErrorString(e));
+    return AMK_ERR_CUDA;
+  }
+  *st = (amk_status)ds.code;
+  if (ds.code == 0 && ds.abort) *st = AMK_ERR_ABORTED;
+  if (*st != AMK_OK) {
+    if (msg && n)
+      snprintf(msg, n, "%s: block %d, %s %d, counter %u of %u", amk_status_str(*st), ds.block,
+               ds.phase >= 0 ? "join" : "ring wait", ds.phase, ds.seen, ds.want);
+    // the step did not finish: its counters are inconsistent, start over from zero
+    e = cudaMemset(h->ws + h->wl.status, 0, sizeof(DevStatus));
+    if (e == cudaSuccess) e = cudaMemset(h->ws + h->wl.phase_ctr, 0, h->wl.cand_val - h->wl.phase_ctr);
+    if (e != cudaSuccess) return AMK_ERR_CUDA;
+    h->epoch = 0;
+  }
+  return AMK_OK;
+}
+
+amk_status amk_plan_info(const amk_handle* h, amk_plan* out) {
+  if (!h || !out) return AMK_ERR_INVALID_ARG;
+  *out = h->plan;
+  return AMK_OK;
+}
+
+amk_status amk_debug_hidden(amk_handle* h, float* host_out) {
+  if (!h || !host_out) return AMK_ERR_INVALID_ARG;
+  if (!(h->cfg.flags & AMK_FLAG_DEBUG_HIDDEN)) return AMK_ERR_INVALID_ARG;
+  cudaError_t e = cudaStreamSynchronize(h->last_stream);
+  if (e == cudaSuccess)
+    e = cudaMemcpy(host_out, h->ws + h->wl.hidden, (size_t)(h->cfg.n_layers + 1) * h->cfg.hidden * 4,
+                   cudaMemcpyDeviceToHost);
+  return e == cudaSuccess ? AMK_OK : AMK_ERR_CUDA;
+}
+
+amk_status amk_debug_unpack(amk_handle* h, int layer, int which, void* out_dev, void* scale_dev, void* zero_dev,
+                            void* cuda_stream) {
+  if (!h || !out_dev) return AMK_ERR_INVALID_ARG;
+  const int L = h->cfg.n_layers;
+  if (which < 0 || which > AMK_LIN_LM_HEAD) return AMK_ERR_INVALID_ARG;
+  if (which != AMK_LIN_LM_HEAD && (layer < 0 || layer >= L)) return AMK_ERR_INVALID_ARG;
+  int op, slot = 0, mode = 0;
+  switch (which) {
+    case AMK_LIN_Q: op = 4 * layer; mode = 1; slot = 0; break;
+    case AMK_LIN_K: op = 4 * layer; mode = 1; slot = 1; break;
+    case AMK_LIN_V: op = 4 * layer; mode = 1; slot = 2; break;
+    case AMK_LIN_O: op = 4 * layer + 1; break;
+    case AMK_LIN_GATE: op = 4 * layer + 2; mode = 2; slot = 0; break;
+    case AMK_LIN_UP: op = 4 * layer + 2; mode = 2; slot = 1; break;
+    case AMK_LIN_DOWN: op = 4 * layer + 3; break;
+    default: op = 4 * L; break;
+  }
+  PackSrc s;
+  memset(&s, 0, sizeof(s));
+  s.mode = mode;
+  s.rows0 = h->cfg.n_q_heads * h->cfg.head_dim;
+  s.rows1 = s.rows0 + h->cfg.n_kv_heads * h->cfg.head_dim;
+  s.w[slot] = out_dev;
+  s.scale[slot] = scale_dev;
+  s.zero[slot] = zero_dev;
+  cudaError_t e = launch_pack(h->pl.ops[op], s, h->packed, (int)h->plan.n_blocks, (int)h->plan.stage_bytes, true,
+                              (cudaStream_t)cuda_stream);
+  return e == cudaSuccess ? AMK_OK : AMK_ERR_CUDA;
+}
+
+amk_status amk_debug_drop_signal(amk_handle* h, int phase, int block) {
+  if (!h) return AMK_ERR_INVALID_ARG;
+  if (block < 0) { h->drop_phase = h->drop_block = -1; return AMK_OK; }
+  if (phase < 0 || phase >= 5 * (int)h->cfg.n_layers || block >= (int)h->plan.n_blocks) return AMK_ERR_INVALID_ARG;
+  h->drop_phase = phase;
+  h->drop_block = block;
+  return AMK_OK;
+}
+
+amk_status amk_destroy(amk_handle* h) {
+  if (!h) return AMK_ERR_INVALID_ARG;
+  delete h;
+  return AMK_OK;
+}
+
+amk_status amk_quantize_int8(const void* w_bf16, int64_t rows, int64_t cols, void* q_out, void* scale_out,
+                             void* cuda_stream) {
+  if (!w_bf16 || !q_out || !scale_out || rows < 0 || cols <= 0 || rows > 0x7fffffff) return AMK_ERR_INVALID_ARG;
+  return launch_quantize_int8(w_bf16, rows, cols, q_out, scale_out, (cudaStream_t)cuda_stream) == cudaSuccess
+             ? AMK_OK
+             : AMK_ERR_CUDA;
+}
+
+amk_status amk_quantize_int4(const void* w_bf16, int64_t rows, int64_t cols, void* packed_out, void* scale_out,
+                             void* zero_out, void* cuda_stream) {
+  if (!w_bf16 || !packed_out || !scale_out || !zero_out || rows < 0 || cols <= 0 || cols % 128)
+    return AMK_ERR_INVALID_ARG;
+  return launch_quantize_int4(w_bf16, rows, cols, packed_out, scale_out, zero_out, (cudaStream_t)cuda_stream) ==
+                 cudaSuccess
+             ? AMK_OK
+             : AMK_ERR_CUDA;
+}
+
+}  // extern "C"
