@@ -1,0 +1,402 @@
+#!/usr/bin/env python
+"""Benchmark of the batch-1 decode step (one cooperative launch = one token).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+Prints ONE JSON line.  `value` is microseconds per token with everything resident in HBM; `e2e` is the
+same step driven from the host (token read from pinned host memory, greedy token and logits copied back
+and waited for, every step).  `roofline` reports algorithmic bytes / measured launch time against the
+measured HBM copy peak; `cpu_baseline` times the CPU oracle on a bounded sample of the same workload.
+
+`--impl reference` times the CPU oracle (as it stands) on the same workload description.
+With N > 1 (torchrun) every rank runs an independent replica on its own GPU: the path does not shard.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2606_09682_b200 import inputs as inp  # noqa: E402
+
+WORKLOADS = {
+    # name: (shape, weight dtype, position)
+    "llama3_8b_bf16_pos0": ("llama3_8b", "bf16", 0),
+    "llama3_8b_int8_pos0": ("llama3_8b", "int8", 0),
+    "llama3_8b_bf16_pos4096": ("llama3_8b", "bf16", 4096),
+    "tinyllama_1b_bf16_pos0": ("tinyllama_1b", "bf16", 0),
+    "tinyllama_1b_int8_pos0": ("tinyllama_1b", "int8", 0),
+    "tinyllama_1b_int4_pos0": ("tinyllama_1b", "int4", 0),
+    "tinyllama_1b_bf16_pos1024": ("tinyllama_1b", "bf16", 1024),
+    "smollm2_135m_bf16_pos0": ("smollm2_135m", "bf16", 0),
+}
+DEFAULT_WORKLOAD = "llama3_8b_bf16_pos0"      # the largest single-GPU configuration
+OTHER = ["llama3_8b_int8_pos0", "tinyllama_1b_bf16_pos0", "tinyllama_1b_int8_pos0", "tinyllama_1b_int4_pos0",
+         "smollm2_135m_bf16_pos0", "tinyllama_1b_bf16_pos1024"]
+METRIC = "batch-1 decode us/token; achieved HBM GB/s vs B200 measured peak"
+SEED = 0xA3C0
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+def ncu_traffic(workload: str):
+    """DRAM bytes per launch from a committed ncu capture summary, if there is one for this workload."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    try:
+        with open(path) as f:
+            return json.load(f).get(workload)
+    except Exception:
+        return None
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.lines = []
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def build_decoder(workload: str, device, flags: int = 0):
+    from paper_2606_09682_b200 import binding as amk
+    name, wd, pos = WORKLOADS[workload]
+    shape = inp.SHAPES[name]
+    w = inp.make_weights(shape, SEED, device=device)
+    wq = amk.quantize_weights(w, wd)
+    dec = amk.Decoder(shape, wq, wd, flags=flags, device=device)
+    keep = None
+    if flags:      # the parity by-product of the CPU-baseline leg needs layer 0's canonical weights
+        keep = {k: (v[0] if isinstance(v, list) else v) for k, v in wq.items() if k not in ("embed", "lm_head")}
+        keep["embed_row_src"] = w["embed"]
+    del w, wq
+    torch.cuda.empty_cache()
+    kv = inp.make_kv_prefill(shape, SEED, pos, device=device)
+    tok = inp.make_token(shape, SEED)
+    return shape, wd, pos, dec, kv, tok, keep
+
+
+def time_device(dec, tok, pos, kv, steps, warmup):
+    """K launches back to back, CUDA events on the launching stream around each."""
+    for _ in range(warmup):
+        dec.amk_decode_step(tok, pos, kv)
+    st, msg = dec.amk_last_status()
+    if st != 0:
+        raise RuntimeError("decode step failed: " + msg)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    torch.cuda.synchronize()
+    ev[0].record()
+    for i in range(steps):
+        dec.amk_decode_step(tok, pos, kv)
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    per = np.array([ev[i].elapsed_time(ev[i + 1]) * 1e3 for i in range(steps)])     # us
+    total_ms = ev[0].elapsed_time(ev[steps])
+    st, msg = dec.amk_last_status()
+    if st != 0:
+        raise RuntimeError("decode step failed: " + msg)
+    return per, total_ms
+
+
+def time_e2e(dec, shape, tok, pos, kv, steps, warmup):
+    """The call a user makes, driven from host buffers: the token comes from pinned host memory, the
+    greedy token and the logits go back to pinned host memory and are waited for, every step."""
+    tok_host = torch.tensor([tok], dtype=torch.int32).pin_memory()
+    next_host = torch.empty(1, dtype=torch.int32).pin_memory()
+    logits_host = torch.empty(shape.vocab, dtype=torch.float32).pin_memory()
+
+    def step():
+        t = int(tok_host[0])                       # host -> device: the token travels as a kernel argument
+        dec.amk_decode_step(t, pos, kv)
+        next_host.copy_(dec.next_token, non_blocking=True)
+        logits_host.copy_(dec.logits, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        return int(next_host[0])
+
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    return dt / steps * 1e6, 4, 4 + 4 * shape.vocab
+
+
+class OracleSample:
+    """CPU oracle on a bounded sample of the workload: one decoder layer (layer 0) plus the LM head, with
+    weights of the workload's shape; microseconds per token = L * t_layer + t_head.
+    With `gpu_ctx` the layer runs on the GPU run's own layer-0 weights and token, which also gives a parity
+    figure against the CUDA path's hidden state after layer 0."""
+
+    def __init__(self, shape, wd, pos, gpu_ctx=None):
+        from oracle import oracle as orc
+        self.orc, self.shape, self.pos = orc, shape, pos
+        s1 = shape.with_(n_layers=1)
+        wdt = {"bf16": orc.W_BF16, "int8": orc.W_INT8, "int4": orc.W_INT4}[wd]
+        self.hidden_gpu = None
+        if gpu_ctx is None:
+            w = inp.weights_to_numpy(inp.make_weights(s1, SEED, device="cpu"))
+            wq = orc.quantize_weights(w, wdt, 128)
+            tok = inp.make_token(shape, SEED)
+        else:
+            keep, tok, self.hidden_gpu = gpu_ctx
+            wq = {}
+            for k, v in keep.items():
+                if k == "embed_row_src":
+                    continue
+                t = v.detach().cpu()
+                arr = t.view(torch.int16).numpy().view(np.uint16) if t.dtype in (torch.bfloat16, torch.float16) else t.numpy()
+                wq[k] = arr if k == "final_norm" else [arr]
+            wq["embed"] = inp.bits(keep["embed_row_src"])
+            wq["lm_head"] = None if shape.tied else wq["embed"]      # any [V][H] bf16 matrix serves the head timing
+        self.model = orc.Model(s1, wq, wdtype=wdt, group=128)
+        self.kv = np.zeros(orc.kv_elems(s1), dtype=np.uint16)
+        if pos > 0:
+            self.kv[:] = inp.bits(inp.make_kv_prefill(s1, SEED, pos, device="cpu"))
+        self.x0 = (wq["embed"][tok].astype(np.uint32) << 16).view(np.float32)
+        self.cores = orc.num_threads()
+        self.parity = None
+
+    def once(self) -> float:
+        """One sample; returns the microseconds-per-token estimate."""
+        t0 = time.perf_counter()
+        out = self.model.layer_step(0, self.pos, self.x0, self.kv)
+        t1 = time.perf_counter()
+        self.model.head_step(out)
+        t2 = time.perf_counter()
+        if self.hidden_gpu is not None and self.parity is None:
+            self.parity = float(np.linalg.norm(self.hidden_gpu[1].astype(np.float64) - out) / np.linalg.norm(out))
+        return (self.shape.n_layers * (t1 - t0) + (t2 - t1)) * 1e6
+
+
+def run_one(workload, device, steps, warmup, with_cpu):
+    from paper_2606_09682_b200 import binding as amk
+    shape, wd, pos, dec, kv, tok, keep = build_decoder(workload, device, amk.AMK_FLAG_DEBUG_HIDDEN if with_cpu else 0)
+    per, total_ms = time_device(dec, tok, pos, kv, steps, warmup)
+    b = inp.streamed_bytes(shape, wd, pos)
+    res = {"workload": workload, "us_per_token": float(np.mean(per)), "median_us": float(np.median(per)),
+           "p10_us": float(np.percentile(per, 10)), "p90_us": float(np.percentile(per, 90)),
+           "total_ms": total_ms, "bytes": b["total"], "plan": dec.plan()}
+    res["shape"], res["wd"], res["pos"], res["dec"], res["kv"], res["tok"], res["keep"] = shape, wd, pos, dec, kv, tok, keep
+    return res
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=25)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--no-others", action="store_true", help="skip the short runs of the other configurations")
+    a = ap.parse_args()
+    a.warmup = max(a.warmup, 3)
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    name, wd, pos = WORKLOADS[a.workload]
+    shape = inp.SHAPES[name]
+    config = {"workload": f"{name} shape, {wd} weights, batch 1, decode position {pos}, "
+                          f"{'pre-filled N(0,1) bf16 KV cache' if pos else 'empty KV cache'}, random-init N(0,0.02) weights",
+              "l2": "inputs larger than L2: every step streams the whole weight set from HBM",
+              "replicas": world}
+
+    # ---------------------------------------------------------------- reference arm: the CPU oracle
+    if a.impl == "reference":
+        if rank != 0:
+            return
+        smp = OracleSample(shape, wd, pos)
+        t_start = time.perf_counter()
+        n_warm = 0
+        for _ in range(a.warmup):
+            smp.once()
+            n_warm += 1
+            if time.perf_counter() - t_start > 30:
+                break                                      # bounded: the sample is slow by design
+        vals = []
+        t_start = time.perf_counter()
+        for _ in range(a.steps):
+            vals.append(smp.once())
+            if time.perf_counter() - t_start > 120:
+                break
+        cores = smp.cores
+        v = float(np.mean(vals))
+        sample = f"layer 0 + LM head of the {name} shape on host cores, us/token = L * t_layer + t_head"
+        line = {"impl": "reference", "metric": METRIC, "value": v, "unit": "us/token", "n_gpus": a.gpus,
+                "steps": len(vals), "warmup": n_warm, "ms_per_step": v / 1e3, "higher_is_better": False,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32 (fp64 accumulators)", "data": "synthetic",
+                "config": config,
+                "cpu_baseline": {"value": v, "unit": "us/token", "cores": cores, "kind": "oracle", "sample": sample},
+                "e2e": {"value": v, "unit": "us/token", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+        print(json.dumps(line))
+        return
+
+    # ---------------------------------------------------------------- our arm
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (the CUDA path has no fallback)")
+    import torch.distributed as dist
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    from paper_2606_09682_b200 import build as amk_build
+    amk_build.build()
+
+    sampler = ClockSampler(local_rank)
+    r = None
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    with_cpu = (rank == 0 and world == 1)
+    shape, wd, pos, dec, kv, tok, keep = build_decoder(a.workload, device, 1 if with_cpu else 0)
+    for _ in range(a.warmup):
+        dec.amk_decode_step(tok, pos, kv)
+    st, msg = dec.amk_last_status()
+    if st != 0:
+        raise SystemExit("decode step failed: " + msg)
+    hidden_gpu = dec.amk_debug_hidden().numpy() if with_cpu else None
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(a.steps + 1)]
+    barrier()
+    sampler.start()
+    ev[0].record()
+    for i in range(a.steps):
+        dec.amk_decode_step(tok, pos, kv)
+        ev[i + 1].record()
+    barrier()
+    clocks = sampler.stop()
+    st, msg = dec.amk_last_status()
+    if st != 0:
+        raise SystemExit("decode step failed: " + msg)
+    per = np.array([ev[i].elapsed_time(ev[i + 1]) * 1e3 for i in range(a.steps)])
+    total_ms = ev[0].elapsed_time(ev[a.steps])
+    t = torch.tensor([total_ms], device=device, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms = float(t.item())
+    e2e_us, h2d, d2h = time_e2e(dec, shape, tok, pos, kv, max(5, a.steps // 4), 3)
+    te = torch.tensor([e2e_us], device=device, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        e2e_us = float(te.item())
+
+    if rank == 0:
+        peak, peak_src = measured_peak()
+        b = inp.streamed_bytes(shape, wd, pos)
+        us = total_ms * 1e3 / a.steps
+        achieved = b["total"] / (us * 1e-6) / 1e9
+        plan = dec.plan()
+        line = {"metric": METRIC, "value": us / world, "unit": "us/token", "n_gpus": world, "steps": a.steps,
+                "warmup": a.warmup, "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak",
+                "vs_baseline": None, "dtype": wd if wd != "bf16" else "bf16 (fp32 accumulate)", "data": "synthetic",
+                "config": config, "clocks": clocks, "gpu_launches": a.steps,
+                "e2e": {"value": e2e_us / world, "unit": "us/token", "h2d_bytes_per_step": h2d,
+                        "d2h_bytes_per_step": d2h},
+                "latency_us": {"median": float(np.median(per)), "p10": float(np.percentile(per, 10)),
+                               "p90": float(np.percentile(per, 90))},
+                "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                             "frac": achieved / peak, "traffic": ncu_traffic(a.workload), "peak_source": peak_src,
+                             "algorithmic_bytes": b["total"],
+                             "bytes_breakdown": {k: b[k] for k in ("weights", "scales", "kv", "act")}},
+                "plan": {"blocks": plan.n_blocks, "threads": plan.threads, "smem_bytes": plan.smem_bytes,
+                         "stages": plan.n_stages, "stage_bytes": plan.stage_bytes, "joins_per_token": plan.n_phases}}
+        if achieved > 1.15 * peak:
+            line["roofline"]["note"] = "above the physical floor: treated as a measurement artefact"
+        if world > 1:
+            line["config"]["note"] = ("replicas only: the path does not shard; value = max-over-ranks step time / "
+                                      "replicas, i.e. job-level microseconds per decoded token")
+        if with_cpu:
+            smp = OracleSample(shape, wd, pos, (keep, tok, hidden_gpu))
+            cpu_us = float(np.median([smp.once() for _ in range(3)]))
+            parity = smp.parity if pos == 0 else None
+            line["cpu_baseline"] = {"value": cpu_us, "unit": "us/token", "cores": smp.cores, "kind": "oracle",
+                                    "sample": "decoder layer 0 (the GPU run's own weights and token, 3 repeats) + LM head, "
+                                              "us/token = L * t_layer + t_head"}
+            if parity is not None:
+                line["parity"] = {"layer0_hidden_rel_l2_vs_oracle": parity, "pass": bool(parity <= 5e-3)}
+                if parity > 5e-3:
+                    line["value"] = None        # correctness-gated: no latency without a parity pass
+        dec.close()
+        del dec, kv, keep
+        torch.cuda.empty_cache()
+        if world == 1 and not a.no_others:
+            others = []
+            for wl in OTHER:
+                try:
+                    r = run_one(wl, device, min(a.steps, 50), max(3, min(a.warmup, 10)), False)
+                    ach = r["bytes"] / (r["us_per_token"] * 1e-6) / 1e9
+                    others.append({"workload": wl, "us_per_token": r["us_per_token"], "median_us": r["median_us"],
+                                   "achieved_gbs": ach, "frac": ach / peak, "bytes": r["bytes"]})
+                    r["dec"].close()
+                    del r
+                    torch.cuda.empty_cache()
+                except Exception as e:      # a side run must never take the headline line down
+                    others.append({"workload": wl, "error": str(e)})
+            line["other_configs"] = others
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

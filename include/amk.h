@@ -45,6 +45,19 @@ typedef enum { AMK_W_BF16 = 0, AMK_W_INT8 = 1, AMK_W_INT4 = 2 } amk_wdtype;
 
 /* amk_config.flags */
 #define AMK_FLAG_DEBUG_HIDDEN 1u /* keep the residual stream after the embedding and after every layer */
+#define AMK_FLAG_TRACE 2u        /* every block stamps the global timer at the stages of every task          */
+
+/* Trace layout (amk_debug_trace): uint64 nanosecond stamps [n_blocks][n_tasks][AMK_TRACE_EVENTS], where
+ * task 5*l+{0,1,2,3,4} = QKV, attention, O, gate/up, down of layer l and task 5*L = LM head. */
+#define AMK_TRACE_EVENTS 8
+enum { AMK_TR_ENTER = 0,      /* consumer warps reach the task                                          */
+       AMK_TR_JOINED = 1,     /* the dependency wait is over                                            */
+       AMK_TR_LOADED = 2,     /* input vector in shared memory (GEMV tasks)                             */
+       AMK_TR_COMPUTED = 3,   /* last output stored                                                     */
+       AMK_TR_SIGNALLED = 4,  /* counter incremented                                                    */
+       AMK_TR_PROD_FIRST = 5, /* producer issued the task's first ring tile (GEMV tasks)                */
+       AMK_TR_PROD_LAST = 6   /* producer issued the task's last ring tile                              */
+};
 
 /* The seven per-layer linears, in the order used by amk_weights.linear[] and amk_debug_unpack. */
 enum { AMK_LIN_Q = 0, AMK_LIN_K = 1, AMK_LIN_V = 2, AMK_LIN_O = 3, AMK_LIN_GATE = 4, AMK_LIN_UP = 5,
@@ -172,6 +185,10 @@ amk_status amk_plan_info(const amk_handle* h, amk_plan* out); /* HOST out */
 /* With AMK_FLAG_DEBUG_HIDDEN: copies the residual stream of the last step to HOST memory,
  * float[(L+1)][H]: row 0 after the embedding, row l+1 after layer l.  Synchronises. */
 amk_status amk_debug_hidden(amk_handle* h, float* host_out);
+
+/* With AMK_FLAG_TRACE: copies the last step's stamps to HOST memory, n_u64 >= n_blocks * (5 L + 1) *
+ * AMK_TRACE_EVENTS.  Synchronises.  This is how the time spent in cross-SM synchronisation is measured. */
+amk_status amk_debug_trace(amk_handle* h, uint64_t* host_out, size_t n_u64);
 
 /* Inverse of the packer, for bit-exact layout checks: rebuilds one canonical matrix from the packed
  * buffer into DEVICE memory of the canonical size.  which = AMK_LIN_* (AMK_LIN_LM_HEAD ignores layer).

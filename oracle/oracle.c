@@ -218,7 +218,7 @@ void orc_quantize_int4(const uint16_t* W_bf16, int rows, int cols, int group, ui
             float s = orc_f16_to_f32(sh);
             if (s == 0.0f) { sh = orc_f32_to_f16(1.0f); s = 1.0f; }
             float z = rintf(-mn / s);
-            if (z < 0.0f) z = 0.0f;
+            if (!(z > 0.0f)) z = 0.0f;             /* also turns -0 (an all-positive group) into +0 */
             if (z > 15.0f) z = 15.0f;
             scale[(size_t)o * ng + g] = sh;
             zero[(size_t)o * ng + g] = orc_f32_to_f16(z);

@@ -20,6 +20,8 @@ AMK_OK, AMK_ERR_INVALID_ARG, AMK_ERR_UNSUPPORTED, AMK_ERR_CUDA, AMK_ERR_OOM = 0,
 AMK_ERR_TIMEOUT, AMK_ERR_ABORTED, AMK_ERR_BAD_POS, AMK_ERR_BAD_TOKEN = 5, 6, 7, 8
 AMK_W_BF16, AMK_W_INT8, AMK_W_INT4 = 0, 1, 2
 AMK_FLAG_DEBUG_HIDDEN = 1
+AMK_FLAG_TRACE = 2
+AMK_TRACE_EVENTS = 8
 AMK_LIN_Q, AMK_LIN_K, AMK_LIN_V, AMK_LIN_O, AMK_LIN_GATE, AMK_LIN_UP, AMK_LIN_DOWN, AMK_LIN_LM_HEAD = range(8)
 KINDS = ("wq", "wk", "wv", "wo", "wgate", "wup", "wdown")
 WDTYPES = {"bf16": AMK_W_BF16, "int8": AMK_W_INT8, "int4": AMK_W_INT4}
@@ -67,6 +69,7 @@ def _load() -> C.CDLL:
         "amk_last_status": (C.c_int, [vp, C.POINTER(C.c_int), C.c_char_p, sz]),
         "amk_plan_info": (C.c_int, [vp, C.POINTER(amk_plan)]),
         "amk_debug_hidden": (C.c_int, [vp, vp]),
+        "amk_debug_trace": (C.c_int, [vp, vp, sz]),
         "amk_debug_unpack": (C.c_int, [vp, C.c_int, C.c_int, vp, vp, vp, vp]),
         "amk_debug_drop_signal": (C.c_int, [vp, C.c_int, C.c_int]),
         "amk_destroy": (C.c_int, [vp]),
@@ -82,7 +85,7 @@ def _load() -> C.CDLL:
 lib = _load()
 EXPORTS = ("amk_status_str", "amk_packed_bytes", "amk_workspace_bytes", "amk_kv_bytes", "amk_create",
            "amk_decode_step", "amk_decode_greedy", "amk_last_status", "amk_plan_info", "amk_debug_hidden",
-           "amk_debug_unpack", "amk_debug_drop_signal", "amk_destroy", "amk_quantize_int8", "amk_quantize_int4")
+           "amk_debug_trace", "amk_debug_unpack", "amk_debug_drop_signal", "amk_destroy", "amk_quantize_int8", "amk_quantize_int4")
 
 
 class AmkError(RuntimeError):
@@ -245,6 +248,13 @@ class Decoder:
     def amk_debug_hidden(self) -> torch.Tensor:
         out = torch.empty((self.shape.n_layers + 1, self.shape.hidden), dtype=torch.float32)
         _check(lib.amk_debug_hidden(self.h, out.data_ptr()), "amk_debug_hidden")
+        return out
+
+    def amk_debug_trace(self) -> torch.Tensor:
+        """int64 nanosecond stamps [n_blocks][5 L + 1][AMK_TRACE_EVENTS] of the last step."""
+        nb, nt = self.plan().n_blocks, 5 * self.shape.n_layers + 1
+        out = torch.zeros((nb, nt, AMK_TRACE_EVENTS), dtype=torch.int64)
+        _check(lib.amk_debug_trace(self.h, out.data_ptr(), out.numel()), "amk_debug_trace")
         return out
 
     def amk_debug_unpack(self, layer: int, which: int):

@@ -29,7 +29,7 @@ struct PackedLayout {
 
 struct WorkspaceLayout {
   size_t status, phase_ctr, group_ctr, lm_ctr, next_ws, cand_val, cand_idx, ops, x_a, x_b, qkv, o, m, part, hidden,
-      rope, total;
+      rope, trace, total;
 };
 
 amk_status check_config(const amk_config* c) {
@@ -122,6 +122,7 @@ WorkspaceLayout workspace_layout(const amk_config* c) {
   w.part = take((size_t)c->n_q_heads * kMaxChunks * (hd + 2) * 4);
   w.hidden = take((L + 1) * H * 4);
   w.rope = take(S * (hd / 2) * sizeof(float2));
+  w.trace = take((size_t)kMaxBlocks * (5 * L + 1) * AMK_TRACE_EVENTS * 8);
   w.total = off;
   return w;
 }
@@ -349,6 +350,7 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     p.lm_ctr = (unsigned*)(h->ws + h->wl.lm_ctr); p.cand_val = (float*)(h->ws + h->wl.cand_val);
     p.cand_idx = (int*)(h->ws + h->wl.cand_idx); p.next_ws = (int*)(h->ws + h->wl.next_ws);
     p.status = (DevStatus*)(h->ws + h->wl.status);
+    p.trace = (cfg->flags & AMK_FLAG_TRACE) ? (unsigned long long*)(h->ws + h->wl.trace) : nullptr;
     p.stage_bytes = (int)stage_bytes; p.n_stages = (int)n_stages; p.max_inflight = (int)max_inflight;
     p.act_bytes = (int)act;
     p.timeout_ns = 1000ull * (cfg->wait_timeout_us ? cfg->wait_timeout_us : 200000u);
@@ -456,6 +458,16 @@ amk_status amk_debug_hidden(amk_handle* h, float* host_out) {
   if (e == cudaSuccess)
     e = cudaMemcpy(host_out, h->ws + h->wl.hidden, (size_t)(h->cfg.n_layers + 1) * h->cfg.hidden * 4,
                    cudaMemcpyDeviceToHost);
+  return e == cudaSuccess ? AMK_OK : AMK_ERR_CUDA;
+}
+
+amk_status amk_debug_trace(amk_handle* h, uint64_t* host_out, size_t n_u64) {
+  if (!h || !host_out) return AMK_ERR_INVALID_ARG;
+  if (!(h->cfg.flags & AMK_FLAG_TRACE)) return AMK_ERR_INVALID_ARG;
+  const size_t need = (size_t)h->plan.n_blocks * (5 * h->cfg.n_layers + 1) * AMK_TRACE_EVENTS;
+  if (n_u64 < need) return AMK_ERR_INVALID_ARG;
+  cudaError_t e = cudaStreamSynchronize(h->last_stream);
+  if (e == cudaSuccess) e = cudaMemcpy(host_out, h->ws + h->wl.trace, need * 8, cudaMemcpyDeviceToHost);
   return e == cudaSuccess ? AMK_OK : AMK_ERR_CUDA;
 }
 

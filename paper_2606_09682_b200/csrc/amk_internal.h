@@ -71,6 +71,7 @@ struct KParams {
   int* cand_idx;
   int* next_ws;
   DevStatus* status;
+  unsigned long long* trace;              // [n_blocks][5 L + 1][8] or null
   // plan
   int stage_bytes, n_stages, max_inflight;
   int act_bytes;                          // activation / attention scratch area in shared memory

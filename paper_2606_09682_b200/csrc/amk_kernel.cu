@@ -116,6 +116,11 @@ __device__ __forceinline__ void signal_phase(Ctx& c, int phase) {
     red_release_gpu_add(c.p.phase_ctr + phase, 1u);
 }
 
+// One thread stamps the global timer for (task, event) of this block when tracing is on.
+__device__ __forceinline__ void stamp(const KParams& p, int cta, int task, int ev) {
+  if (p.trace) p.trace[((size_t)cta * (5 * p.L + 1) + task) * AMK_TRACE_EVENTS + ev] = globaltimer_ns();
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -278,6 +283,8 @@ __device__ __noinline__ bool gemv_op(Ctx& c, int op_idx, int wait_ph, int sig_ph
     default: src = p.x_a; normw = p.final_norm; break;
   }
 
+  const int task = (d.kind == OP_LMHEAD) ? 5 * p.L : 5 * l + (d.kind == OP_QKV ? 0 : d.kind + 1);
+  if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_ENTER);
   // ---- prologue, part 1: what does not depend on the join (norm weights) -----------------------------
   uint2 gw[kNormVec];
   if (normw) {
@@ -289,6 +296,7 @@ __device__ __noinline__ bool gemv_op(Ctx& c, int op_idx, int wait_ph, int sig_ph
   }
   // ---- the join ---------------------------------------------------------------------------------------
   if (wait_ph >= 0 && !wait_phase(c, wait_ph)) return false;
+  if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_JOINED);
 
   // ---- prologue, part 2: bring the input vector into shared memory ------------------------------------
   float4* xs4 = reinterpret_cast<float4*>(c.xs);
@@ -331,6 +339,7 @@ __device__ __noinline__ bool gemv_op(Ctx& c, int op_idx, int wait_ph, int sig_ph
   }
   c.bad = cons_sync_or(c.bad);
   if (c.bad) return false;
+  if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_LOADED);
 
   // ---- passes -------------------------------------------------------------------------------------------
   float best_val = -CUDART_INF_F;
@@ -402,6 +411,7 @@ __device__ __noinline__ bool gemv_op(Ctx& c, int op_idx, int wait_ph, int sig_ph
     }
   }
 
+  if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_COMPUTED);
   if (d.kind == OP_LMHEAD) {
     // block argmax, then the block that arrives last reduces all blocks' candidates
     if (c.warp < kOutWarps) {
@@ -460,6 +470,7 @@ __device__ __noinline__ bool gemv_op(Ctx& c, int op_idx, int wait_ph, int sig_ph
   c.bad = cons_sync_or(c.bad);
   if (c.bad) return false;
   if (sig_ph >= 0) signal_phase(c, sig_ph);
+  if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_SIGNALLED);
   return true;
 }
 
@@ -659,7 +670,9 @@ __device__ __noinline__ bool attention_phase(Ctx& c, int l) {
   const int n_tasks = p.nkv * C;
   const int rot = (l * 29) % c.nblk;
   const int t = (c.cta + c.nblk - rot) % c.nblk;
+  if (c.tid == 0) stamp(p, c.cta, 5 * l + 1, AMK_TR_ENTER);
   if (!wait_phase(c, 5 * l + 0)) return false;
+  if (c.tid == 0) stamp(p, c.cta, 5 * l + 1, AMK_TR_JOINED);
   if (t < n_tasks) {
     const int g = t / C, ch = t - g * C;
     if (p.hd == 64) attn_task<64>(c, l, g, ch, Lc, C);
@@ -667,7 +680,9 @@ __device__ __noinline__ bool attention_phase(Ctx& c, int l) {
   }
   c.bad = cons_sync_or(c.bad);
   if (c.bad) return false;
+  if (c.tid == 0) stamp(p, c.cta, 5 * l + 1, AMK_TR_COMPUTED);
   signal_phase(c, 5 * l + 1);
+  if (c.tid == 0) stamp(p, c.cta, 5 * l + 1, AMK_TR_SIGNALLED);
   return true;
 }
 
@@ -687,6 +702,8 @@ __device__ __noinline__ void producer(const KParams& p, SmemHeader* sh, unsigned
     const int64_t rb = row_bytes(d.wdtype, d.K);
     const unsigned char* base = p.packed + d.packed_off + (int64_t)sl.row0 * rb;
     const int np = n_passes(sl.rows);
+    const int task = (d.kind == OP_LMHEAD) ? 5 * p.L : 5 * d.layer + (d.kind == OP_QKV ? 0 : d.kind + 1);
+    bool first = true;
     for (int ps = 0; ps < np && ok; ps++) {
       const PassGeom g = pass_geom(pass_rows(sl.rows, ps), d.K, d.wdtype, p.stage_bytes);
       const unsigned char* pbase = base + (int64_t)ps * kPassRows * rb;
@@ -704,8 +721,10 @@ __device__ __noinline__ void producer(const KParams& p, SmemHeader* sh, unsigned
         const unsigned bytes = (unsigned)(o1 - o0);
         mbar_expect_tx(&sh->full[stage], bytes);
         bulk_g2s(ring + (size_t)stage * p.stage_bytes, pbase + o0, bytes, &sh->full[stage], pol);
+        if (first) { stamp(p, cta, task, AMK_TR_PROD_FIRST); first = false; }
       }
     }
+    if (ok) stamp(p, cta, task, AMK_TR_PROD_LAST);
   }
   if (!ok) {
     // leaving early: every copy already issued must land before the block's shared memory is released

@@ -165,7 +165,8 @@ __global__ void quantize_int4_kernel(const unsigned short* __restrict__ w, int64
   float s = __half2float(h);
   if (s == 0.f) { h = __float2half_rn(1.0f); s = 1.0f; }
   float z = rintf(__fdiv_rn(-mn, s));
-  z = fminf(fmaxf(z, 0.f), 15.f);
+  if (!(z > 0.f)) z = 0.f;                 // also turns -0 (an all-positive group) into +0
+  z = fminf(z, 15.f);
   unsigned code[4];
 #pragma unroll
   for (int e = 0; e < 4; e++) {

@@ -1,0 +1,116 @@
+"""CPU-only checks of the boundary: the shared library loads, exports every symbol the header declares,
+the Python mirror of the POD structs matches the C layout, the size queries and argument checks work
+without a GPU, and the packed-weight geometry covers every matrix element exactly once."""
+import ctypes as C
+import os
+import re
+import subprocess
+
+import pytest
+
+from paper_2606_09682_b200 import build as amk_build
+from paper_2606_09682_b200 import inputs as inp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "amk.h")
+
+
+@pytest.fixture(scope="module")
+def amk():
+    amk_build.build()
+    from paper_2606_09682_b200 import binding
+    return binding
+
+
+def header_functions():
+    src = open(HEADER).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"\b(amk_[a-z0-9_]+)\s*\(", src)))
+
+
+def test_library_exports_every_declared_symbol(amk):
+    names = header_functions()
+    assert len(names) >= 15
+    for n in names:
+        assert hasattr(amk.lib, n), n
+    assert sorted(amk.EXPORTS) == names
+
+
+def test_struct_mirror_matches_header(amk, tmp_path):
+    """Compile a tiny C program against the header and compare sizeof/offsetof with the ctypes mirror."""
+    fields = [f for f, _ in amk.amk_config._fields_]
+    plan_fields = [f for f, _ in amk.amk_plan._fields_]
+    prog = ['#include <stdio.h>', '#include <stddef.h>', '#include "amk.h"', 'int main(void){',
+            'printf("%zu %zu %zu\\n", sizeof(amk_config), sizeof(amk_weights), sizeof(amk_plan));']
+    for f in fields:
+        prog.append(f'printf("%zu\\n", offsetof(amk_config, {f}));')
+    for f in plan_fields:
+        prog.append(f'printf("%zu\\n", offsetof(amk_plan, {f}));')
+    prog.append("return 0;}")
+    src = tmp_path / "t.c"
+    src.write_text("\n".join(prog))
+    exe = tmp_path / "t"
+    subprocess.run(["gcc", "-I", os.path.join(ROOT, "include"), "-o", str(exe), str(src)], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()
+    assert [int(x) for x in out[:3]] == [C.sizeof(amk.amk_config), C.sizeof(amk.amk_weights), C.sizeof(amk.amk_plan)]
+    offs = [int(x) for x in out[3:]]
+    assert offs[:len(fields)] == [getattr(amk.amk_config, f).offset for f in fields]
+    assert offs[len(fields):] == [getattr(amk.amk_plan, f).offset for f in plan_fields]
+
+
+def test_size_queries_and_argument_checks(amk):
+    for name in ("smollm2_135m", "tinyllama_1b", "llama3_8b"):
+        s = inp.SHAPES[name]
+        for wd in ("bf16", "int8", "int4"):
+            cfg = amk.make_config(s, wd)
+            if wd == "int4" and name == "smollm2_135m":       # hidden 576 is not a multiple of 256
+                with pytest.raises(amk.AmkError) as e:
+                    amk.amk_packed_bytes(cfg)
+                assert e.value.code == amk.AMK_ERR_UNSUPPORTED
+                continue
+            pb = amk.amk_packed_bytes(cfg)
+            b = inp.streamed_bytes(s, wd, 0)
+            # packed buffer = streamed weights and scales + a canonical embedding copy (+ alignment padding)
+            expect = b["weights"] + b["scales"] - 2.0 * s.hidden + 2.0 * s.vocab * s.hidden
+            assert 0 <= pb - expect < 1e-3 * expect + 1e6, (name, wd, pb, expect)
+            assert amk.amk_kv_bytes(cfg) == 2 * s.n_layers * s.n_kv_heads * s.max_seq * s.head_dim * 2
+            assert amk.amk_workspace_bytes(cfg) > 0
+    cfg = amk.make_config(inp.SHAPES["mini"], "bf16")
+    n = C.c_size_t()
+    assert amk.lib.amk_packed_bytes(None, C.byref(n)) == amk.AMK_ERR_INVALID_ARG
+    assert amk.lib.amk_packed_bytes(C.byref(cfg), None) == amk.AMK_ERR_INVALID_ARG
+    cfg.struct_size = 12
+    assert amk.lib.amk_packed_bytes(C.byref(cfg), C.byref(n)) == amk.AMK_ERR_INVALID_ARG
+    cfg = amk.make_config(inp.SHAPES["mini"], "bf16")
+    cfg.abi_version = 99
+    assert amk.lib.amk_kv_bytes(C.byref(cfg), C.byref(n)) == amk.AMK_ERR_INVALID_ARG
+    for field, val in (("head_dim", 48), ("n_q_heads", 3), ("quantize_lm_head", 1)):
+        cfg = amk.make_config(inp.SHAPES["mini"], "bf16")
+        setattr(cfg, field, val)
+        assert amk.lib.amk_packed_bytes(C.byref(cfg), C.byref(n)) == amk.AMK_ERR_UNSUPPORTED, field
+    # calls on a NULL handle fail cleanly
+    assert amk.lib.amk_decode_step(None, 0, 0, None, None, None, None) == amk.AMK_ERR_INVALID_ARG
+    assert amk.lib.amk_destroy(None) == amk.AMK_ERR_INVALID_ARG
+    assert amk.lib.amk_status_str(amk.AMK_ERR_TIMEOUT) == b"device-side wait timed out"
+
+
+@pytest.fixture(scope="module")
+def layout_check(tmp_path_factory):
+    exe = tmp_path_factory.mktemp("native") / "layout_check"
+    subprocess.run(["g++", "-O2", "-std=c++17", "-I", os.path.join(ROOT, "paper_2606_09682_b200", "csrc"),
+                    "-o", str(exe), os.path.join(ROOT, "tests", "native", "layout_check.cpp")], check=True)
+    return str(exe)
+
+
+@pytest.mark.parametrize("rows,K,wd,unit,nblk", [
+    (2560, 2048, 0, 1, 148), (2048, 2048, 0, 1, 148), (11264, 2048, 0, 2, 148), (2048, 5632, 0, 1, 148),   # TinyLlama bf16
+    (960, 576, 0, 1, 148), (3072, 576, 0, 2, 148), (576, 1536, 0, 1, 148),                                  # SmolLM2 shape
+    (6144, 4096, 1, 1, 148), (28672, 4096, 1, 2, 148), (4096, 14336, 1, 1, 148),                            # Llama-3-8B int8
+    (2560, 2048, 2, 2, 148), (11264, 2048, 2, 2, 148), (2048, 5632, 2, 2, 148),                             # TinyLlama int4
+    (1003, 192, 0, 1, 148), (7, 64, 0, 1, 148), (300, 320, 1, 1, 132), (5000, 1024, 0, 1, 7),               # odd cases
+])
+def test_packed_geometry_covers_every_element_once(layout_check, rows, K, wd, unit, nblk):
+    for stage in (32768, 16384):
+        r = subprocess.run([layout_check, str(rows), str(K), str(wd), str(unit), str(nblk), str(stage)],
+                           capture_output=True, text=True)
+        assert r.stdout.strip() == "ok", (r.stdout, r.stderr)
