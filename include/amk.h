@@ -67,12 +67,12 @@ enum { AMK_LIN_Q = 0, AMK_LIN_K = 1, AMK_LIN_V = 2, AMK_LIN_O = 3, AMK_LIN_GATE 
 typedef struct amk_config {
   uint32_t struct_size;      /* = sizeof(amk_config)                                                   */
   uint32_t abi_version;      /* = AMK_ABI_VERSION                                                      */
-  uint32_t hidden;           /* H; multiple of 8 (16 for int8, 256 for int4)                           */
+  uint32_t hidden;           /* H; multiple of 64 (128 for int4), at most 7680                         */
   uint32_t n_layers;         /* L                                                                      */
   uint32_t n_q_heads;        /* multiple of n_kv_heads; n_q_heads / n_kv_heads <= 16                   */
   uint32_t n_kv_heads;
   uint32_t head_dim;         /* 64 or 128                                                              */
-  uint32_t mlp;              /* I; same divisibility rule as hidden                                    */
+  uint32_t mlp;              /* I; multiple of 64 (128 for int4), at most 15360                        */
   uint32_t vocab;            /* V                                                                      */
   uint32_t max_seq;          /* S: positions the KV cache holds                                        */
   uint32_t tied_embeddings;  /* 1: the LM head is the embedding matrix                                 */
@@ -87,7 +87,12 @@ typedef struct amk_config {
   uint32_t stage_bytes;      /* bytes per shared-memory ring stage (multiple of 1024)                  */
   uint32_t n_stages;         /* ring depth                                                             */
   uint32_t max_inflight;     /* bulk copies a block keeps in flight (<= n_stages)                      */
-  uint32_t reserved[3];      /* must be 0                                                              */
+  uint32_t sync_mode;        /* 0: activations carry sequence numbers AND every task ends with a release-
+                                increment that the next task's readers acquire-spin on (the paper's counter
+                                model); 1: sequence numbers only (no counters, no fences).  Same results.  */
+  uint32_t n_blocks;         /* persistent blocks; 0 = one per SM of the current device (148 if there is
+                                no device).  The packed layout depends on it.                          */
+  uint32_t reserved[1];      /* must be 0                                                              */
 } amk_config;
 
 /*

@@ -18,19 +18,44 @@ using namespace amk;
 namespace {
 
 constexpr size_t kAlign = 256;
-constexpr int kMaxBlocks = 512;   // upper bound on SMs, for sizing the per-block candidate arrays
+constexpr int kMaxBlocks = 512;   // upper bound on persistent blocks
 inline size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a; }
 
-struct PackedLayout {
-  std::vector<OpDesc> ops;      // packed_off / scale_off filled
-  size_t embed_off, attn_norm_off, mlp_norm_off, final_norm_off, total;
-  size_t weight_stream_bytes;   // op regions + scale regions (what a token streams)
+// One matrix-vector product of the step, as the host plans it.
+struct PlanOp {
+  int kind, layer, rot;
+  OpShape s;
+  size_t region_off;                 // byte offset of the op's region in the packed buffer
+  size_t scale_off;                  // int8: fp16 row scales (virtual row order)
+  std::vector<unsigned long long> slice_off;   // [n_blocks] byte offset of each slot's slice inside the region
+};
+
+// Everything that follows from (config, block count): op table, packed-buffer layout, per-block tile lists.
+struct Plan {
+  int n_blocks = 0;
+  uint32_t stage_bytes = 0;
+  OpShape shape[5];
+  std::vector<PlanOp> ops;
+  size_t scale_base = 0, scale_layer_stride = 0, scale_kind_off[4] = {0, 0, 0, 0};
+  size_t embed_off = 0, attn_norm_off = 0, mlp_norm_off = 0, final_norm_off = 0, packed_total = 0;
+  size_t weight_stream_bytes = 0;    // op regions + scale regions (what a token streams)
+  size_t n_tiles = 0;                // total ring tiles over all blocks
 };
 
 struct WorkspaceLayout {
-  size_t status, phase_ctr, group_ctr, lm_ctr, next_ws, cand_val, cand_idx, ops, x_a, x_b, qkv, o, m, part, hidden,
-      rope, trace, total;
+  size_t status, phase_ctr, group_ctr, lm_ctr, next_ws, cand_val, cand_idx, x_a, x_b, qkv, o, m, part, hidden, rope,
+      trace, slice_tab, tile_begin, tiles, total;
 };
+
+int resolve_blocks(const amk_config* c) {
+  if (c->n_blocks) return (int)c->n_blocks;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess &&
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+    return sms;
+  (void)cudaGetLastError();
+  return 148;
+}
 
 amk_status check_config(const amk_config* c) {
   if (!c) return AMK_ERR_INVALID_ARG;
@@ -38,19 +63,17 @@ amk_status check_config(const amk_config* c) {
   for (uint32_t r : c->reserved) if (r) return AMK_ERR_INVALID_ARG;
   if (!c->hidden || !c->n_layers || !c->n_q_heads || !c->n_kv_heads || !c->mlp || !c->vocab || !c->max_seq)
     return AMK_ERR_INVALID_ARG;
-  if (c->wdtype > AMK_W_INT4) return AMK_ERR_INVALID_ARG;
+  if (c->wdtype > AMK_W_INT4 || c->sync_mode > 1) return AMK_ERR_INVALID_ARG;
+  if (c->n_blocks > (uint32_t)kMaxBlocks) return AMK_ERR_INVALID_ARG;
   if (c->head_dim != 64 && c->head_dim != 128) return AMK_ERR_UNSUPPORTED;
   if (c->n_q_heads % c->n_kv_heads) return AMK_ERR_UNSUPPORTED;
   if (c->n_q_heads / c->n_kv_heads > (uint32_t)kMaxRep) return AMK_ERR_UNSUPPORTED;
   if (c->quantize_lm_head) return AMK_ERR_UNSUPPORTED;
-  const uint32_t kdiv = c->wdtype == AMK_W_BF16 ? 8 : (c->wdtype == AMK_W_INT8 ? 16 : 256);
+  const uint32_t kdiv = (c->wdtype == AMK_W_INT4) ? 128 : 64;
   const uint32_t qdim = c->n_q_heads * c->head_dim;
   if (c->hidden % kdiv || c->mlp % kdiv || qdim % kdiv) return AMK_ERR_UNSUPPORTED;
-  if (c->hidden % 8) return AMK_ERR_UNSUPPORTED;                      // LM head is bf16
-  if (c->hidden > (uint32_t)(4 * kConsumerThreads * 4)) return AMK_ERR_UNSUPPORTED;   // norm prologue register budget
+  if (c->hidden > 7680u || c->mlp > 15360u || qdim > 15360u) return AMK_ERR_UNSUPPORTED;   // prologue register budget
   if (c->wdtype == AMK_W_INT4 && c->group_size != 128) return AMK_ERR_UNSUPPORTED;
-  if (c->wdtype == AMK_W_INT4 && (c->hidden % 2)) return AMK_ERR_UNSUPPORTED;
-  if (c->n_kv_heads > (uint32_t)kMaxBlocks) return AMK_ERR_UNSUPPORTED;
   if ((uint64_t)c->vocab * c->hidden > (1ull << 40)) return AMK_ERR_UNSUPPORTED;
   if (c->stage_bytes && (c->stage_bytes % 1024 || c->stage_bytes < 8192 || c->stage_bytes > 65536))
     return AMK_ERR_INVALID_ARG;
@@ -60,47 +83,92 @@ amk_status check_config(const amk_config* c) {
 
 uint32_t stage_bytes_of(const amk_config* c) { return c->stage_bytes ? c->stage_bytes : 32768u; }
 
-// Op table and packed-buffer layout (independent of the number of blocks: rows keep their byte size).
-PackedLayout packed_layout(const amk_config* c) {
-  PackedLayout pl;
+Plan make_plan(const amk_config* c, int n_blocks, bool with_tiles, std::vector<unsigned long long>* tiles,
+               std::vector<unsigned>* tile_begin) {
+  Plan pl;
+  pl.n_blocks = n_blocks;
+  pl.stage_bytes = stage_bytes_of(c);
   const int H = c->hidden, L = c->n_layers, I = c->mlp, V = c->vocab;
   const int qd = c->n_q_heads * c->head_dim, kvd = c->n_kv_heads * c->head_dim;
   const int wd = (int)c->wdtype;
-  const int ur = (wd == W_INT4) ? 2 : 1;
+  pl.shape[OP_QKV] = OpShape{H, qd + 2 * kvd, 1, wd};
+  pl.shape[OP_O] = OpShape{qd, H, 1, wd};
+  pl.shape[OP_GATEUP] = OpShape{H, 2 * I, 2, wd};
+  pl.shape[OP_DOWN] = OpShape{I, H, 1, wd};
+  pl.shape[OP_LMHEAD] = OpShape{H, V, 1, W_BF16};
   size_t off = 0;
-  auto add = [&](int kind, int layer, int K, int rows, int unit_rows, int wdt) {
-    OpDesc d;
-    memset(&d, 0, sizeof(d));
-    d.kind = kind; d.layer = layer; d.K = K; d.rows = rows; d.unit_rows = unit_rows; d.wdtype = wdt;
-    d.rot = (int)((pl.ops.size() * 37u) % 9973u);      // reduced modulo the block count at create time
-    d.packed_off = off;
-    off = align_up(off + (size_t)rows * (size_t)row_bytes(wdt, K));
-    pl.ops.push_back(d);
+  auto add = [&](int kind, int layer) {
+    PlanOp op;
+    op.kind = kind; op.layer = layer; op.s = pl.shape[kind];
+    op.rot = (int)((pl.ops.size() * 37u) % (unsigned)n_blocks);
+    op.region_off = off;
+    op.scale_off = 0;
+    op.slice_off.resize(n_blocks);
+    size_t o = 0;
+    for (int s = 0; s < n_blocks; s++) {
+      op.slice_off[s] = o;
+      o += (size_t)slice_bytes(slot_slice(op.s.rows, op.s.unit_rows, n_blocks, s).rows, op.s.K, op.s.wdtype,
+                               (int)pl.stage_bytes);
+    }
+    off = align_up(off + o);
+    pl.ops.push_back(std::move(op));
   };
   for (int l = 0; l < L; l++) {
-    add(OP_QKV, l, H, qd + 2 * kvd, ur, wd);
-    add(OP_O, l, qd, H, ur, wd);
-    add(OP_GATEUP, l, H, 2 * I, 2, wd);
-    add(OP_DOWN, l, I, H, ur, wd);
+    add(OP_QKV, l);
+    add(OP_O, l);
+    add(OP_GATEUP, l);
+    add(OP_DOWN, l);
   }
-  add(OP_LMHEAD, L, H, V, 1, W_BF16);
+  add(OP_LMHEAD, L);
   if (wd == W_INT8) {
-    for (auto& d : pl.ops) {
-      if (d.wdtype != W_INT8) continue;
-      d.scale_off = off;
-      off = align_up(off + (size_t)d.rows * 2);
-    }
+    pl.scale_base = off;
+    size_t k = 0;
+    for (int kind = 0; kind < 4; kind++) { pl.scale_kind_off[kind] = k; k = align_up(k + (size_t)pl.shape[kind].rows * 2, 16); }
+    pl.scale_layer_stride = k;
+    for (auto& op : pl.ops)
+      if (op.kind != OP_LMHEAD) op.scale_off = pl.scale_base + (size_t)op.layer * k + pl.scale_kind_off[op.kind];
+    off = align_up(off + (size_t)L * k);
   }
   pl.weight_stream_bytes = off;
   pl.embed_off = off;      off = align_up(off + (size_t)V * H * 2);
   pl.attn_norm_off = off;  off = align_up(off + (size_t)L * H * 2);
   pl.mlp_norm_off = off;   off = align_up(off + (size_t)L * H * 2);
   pl.final_norm_off = off; off = align_up(off + (size_t)H * 2);
-  pl.total = off;
+  pl.packed_total = off;
+
+  // per-block tile lists, in the order the block consumes them
+  size_t count = 0;
+  if (with_tiles) { tiles->clear(); tile_begin->assign(n_blocks + 1, 0); }
+  for (int cta = 0; cta < n_blocks; cta++) {
+    if (with_tiles) (*tile_begin)[cta] = (unsigned)count;
+    for (size_t i = 0; i < pl.ops.size(); i++) {
+      const PlanOp& op = pl.ops[i];
+      const int slot = (cta + op.rot) % n_blocks;
+      const Slice sl = slot_slice(op.s.rows, op.s.unit_rows, n_blocks, slot);
+      const int task = (op.kind == OP_LMHEAD) ? 5 * L : 5 * op.layer + (op.kind == OP_QKV ? 0 : op.kind + 1);
+      size_t base = op.region_off + op.slice_off[slot];
+      for (int ps = 0; ps < n_passes(sl.rows); ps++) {
+        const PassGeom g = pass_geom(pass_rows(sl.rows, ps), op.s.K, op.s.wdtype, (int)pl.stage_bytes);
+        for (int t = 0; t < g.n_tiles; t++) {
+          const int64_t o0 = unit_off(g, t * g.upt), o1 = unit_off(g, (t + 1) * g.upt);
+          if (with_tiles) {
+            const unsigned long long e = (unsigned long long)((base + (size_t)o0) >> 4) |
+                                         ((unsigned long long)((o1 - o0) >> 4) << 40) |
+                                         ((unsigned long long)task << 53);
+            tiles->push_back(e);
+          }
+          count++;
+        }
+        base += (size_t)pass_bytes(g);
+      }
+    }
+  }
+  if (with_tiles) (*tile_begin)[n_blocks] = (unsigned)count;
+  pl.n_tiles = count;
   return pl;
 }
 
-WorkspaceLayout workspace_layout(const amk_config* c) {
+WorkspaceLayout workspace_layout(const amk_config* c, const Plan& pl) {
   WorkspaceLayout w;
   const size_t H = c->hidden, L = c->n_layers, I = c->mlp, S = c->max_seq, hd = c->head_dim;
   const size_t qd = (size_t)c->n_q_heads * hd, kvd = (size_t)c->n_kv_heads * hd;
@@ -108,21 +176,23 @@ WorkspaceLayout workspace_layout(const amk_config* c) {
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
   w.status = take(sizeof(DevStatus));
   w.phase_ctr = take(5 * L * 4);
-  w.group_ctr = take((size_t)c->n_kv_heads * 4);
+  w.group_ctr = take(L * (size_t)c->n_kv_heads * 4);
   w.lm_ctr = take(4);
   w.next_ws = take(4);
   w.cand_val = take(kMaxBlocks * 4);
   w.cand_idx = take(kMaxBlocks * 4);
-  w.ops = take((4 * L + 1) * sizeof(OpDesc));
-  w.x_a = take(H * 4);
-  w.x_b = take(H * 4);
-  w.qkv = take((qd + 2 * kvd) * 4);
-  w.o = take(qd * 4);
-  w.m = take(I * 4);
+  w.x_a = take(H * sizeof(ActPair));
+  w.x_b = take(H * sizeof(ActPair));
+  w.qkv = take((qd + 2 * kvd) * sizeof(ActPair));
+  w.o = take(qd * sizeof(ActPair));
+  w.m = take(I * sizeof(ActPair));
   w.part = take((size_t)c->n_q_heads * kMaxChunks * (hd + 2) * 4);
   w.hidden = take((L + 1) * H * 4);
   w.rope = take(S * (hd / 2) * sizeof(float2));
-  w.trace = take((size_t)kMaxBlocks * (5 * L + 1) * AMK_TRACE_EVENTS * 8);
+  w.trace = take((size_t)pl.n_blocks * (5 * L + 1) * AMK_TRACE_EVENTS * 8);
+  w.slice_tab = take(pl.ops.size() * (size_t)pl.n_blocks * 8);
+  w.tile_begin = take(((size_t)pl.n_blocks + 1) * 4);
+  w.tiles = take(pl.n_tiles * 8);
   w.total = off;
   return w;
 }
@@ -136,12 +206,13 @@ size_t kv_bytes_of(const amk_config* c) {
 struct amk_handle {
   amk_config cfg;
   amk_plan plan;
-  PackedLayout pl;
+  Plan pl;
   WorkspaceLayout wl;
   unsigned char* packed;
   unsigned char* ws;
   KParams base;            // everything but the per-step fields
-  unsigned epoch;
+  unsigned epoch;          // steps launched: sequence numbers never repeat
+  unsigned ctr_epoch;      // steps since the counters were last zeroed
   cudaStream_t last_stream;
   int drop_phase, drop_block;
   char errmsg[256];
@@ -168,7 +239,7 @@ amk_status amk_packed_bytes(const amk_config* cfg, size_t* bytes) {
   if (!bytes) return AMK_ERR_INVALID_ARG;
   amk_status st = check_config(cfg);
   if (st != AMK_OK) return st;
-  *bytes = packed_layout(cfg).total;
+  *bytes = make_plan(cfg, resolve_blocks(cfg), false, nullptr, nullptr).packed_total;
   return AMK_OK;
 }
 
@@ -176,7 +247,8 @@ amk_status amk_workspace_bytes(const amk_config* cfg, size_t* bytes) {
   if (!bytes) return AMK_ERR_INVALID_ARG;
   amk_status st = check_config(cfg);
   if (st != AMK_OK) return st;
-  *bytes = workspace_layout(cfg).total;
+  const Plan pl = make_plan(cfg, resolve_blocks(cfg), false, nullptr, nullptr);
+  *bytes = workspace_layout(cfg, pl).total;
   return AMK_OK;
 }
 
@@ -217,27 +289,36 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
   amk_handle* h = new (std::nothrow) amk_handle();
   if (!h) return AMK_ERR_OOM;
   h->cfg = *cfg;
-  h->pl = packed_layout(cfg);
-  h->wl = workspace_layout(cfg);
   h->packed = (unsigned char*)packed_dev;
   h->ws = (unsigned char*)workspace_dev;
   h->drop_phase = -1;
   h->drop_block = -1;
   h->last_stream = stream;
   {
-    if (packed_bytes < h->pl.total || workspace_bytes < h->wl.total) { status = AMK_ERR_INVALID_ARG; goto fail; }
     int dev = 0, sms = 0, coop = 0, smem_optin = 0, cc_major = 0;
     AMK_CUDA(cudaGetDevice(&dev));
     AMK_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     AMK_CUDA(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
     AMK_CUDA(cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
     AMK_CUDA(cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev));
-    if (cc_major != 10 || !coop || sms < 1 || sms > kMaxBlocks || (int)cfg->n_kv_heads > sms) {
-      snprintf(h->errmsg, sizeof(h->errmsg), "needs a compute-capability-10.x GPU with cooperative launch");
+    const int n_blocks = cfg->n_blocks ? (int)cfg->n_blocks : sms;
+    if (cc_major != 10 || !coop || sms < 1 || n_blocks > sms || n_blocks > kMaxBlocks ||
+        (int)cfg->n_kv_heads > n_blocks) {
+      snprintf(h->errmsg, sizeof(h->errmsg),
+               "needs a compute-capability-10.x GPU with cooperative launch and at least n_blocks SMs");
       status = AMK_ERR_UNSUPPORTED;
       goto fail;
     }
-    const int n_blocks = sms;
+    std::vector<unsigned long long> tiles;
+    std::vector<unsigned> tile_begin;
+    h->pl = make_plan(cfg, n_blocks, true, &tiles, &tile_begin);
+    h->wl = workspace_layout(cfg, h->pl);
+    if (packed_bytes < h->pl.packed_total || workspace_bytes < h->wl.total) {
+      snprintf(h->errmsg, sizeof(h->errmsg), "buffers too small: packed %zu < %zu or workspace %zu < %zu", packed_bytes,
+               h->pl.packed_total, workspace_bytes, h->wl.total);
+      status = AMK_ERR_INVALID_ARG;
+      goto fail;
+    }
     const int H = cfg->hidden, L = cfg->n_layers, I = cfg->mlp, hd = cfg->head_dim;
     const int qd = cfg->n_q_heads * hd, n_rep = cfg->n_q_heads / cfg->n_kv_heads;
 
@@ -245,11 +326,12 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     const size_t hdr = (sizeof(SmemHeader) + 127) & ~(size_t)127;
     size_t kmax = (size_t)(H > I ? H : I);
     if ((size_t)qd > kmax) kmax = qd;
-    size_t act = kmax * 4;
+    size_t act = kmax * (cfg->wdtype == AMK_W_BF16 ? 4 : 3);   // bf16 high + low halves, or three int8 digits
+    if ((size_t)H * 4 > act) act = (size_t)H * 4;               // the LM head is always bf16
     const size_t attn_need = ((size_t)n_rep * hd + (size_t)kConsumerWarps * 4 * (hd + 2)) * 4;
     if (attn_need > act) act = attn_need;
     act = (act + 127) & ~(size_t)127;
-    const uint32_t stage_bytes = stage_bytes_of(cfg);
+    const uint32_t stage_bytes = h->pl.stage_bytes;
     uint32_t n_stages = cfg->n_stages;
     const size_t avail = (size_t)smem_optin > hdr + act ? (size_t)smem_optin - hdr - act : 0;
     const uint32_t fit = (uint32_t)(avail / stage_bytes);
@@ -271,34 +353,40 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
       goto fail;
     }
 
-    // ---- op table, rotations reduced modulo the block count ------------------------------------------
-    for (auto& d : h->pl.ops) d.rot = d.rot % n_blocks;
+    // ---- workspace: zero it, upload the slice and tile tables and the rotary table ---------------------
     AMK_CUDA(cudaMemsetAsync(h->ws, 0, h->wl.total, stream));
-    AMK_CUDA(cudaMemcpyAsync(h->ws + h->wl.ops, h->pl.ops.data(), h->pl.ops.size() * sizeof(OpDesc),
-                             cudaMemcpyHostToDevice, stream));
-
-    // ---- rotary table (cos, sin)[pos][i], angles formed in double --------------------------------------
     {
+      std::vector<unsigned long long> slices(h->pl.ops.size() * (size_t)n_blocks);
+      for (size_t i = 0; i < h->pl.ops.size(); i++)
+        memcpy(&slices[i * n_blocks], h->pl.ops[i].slice_off.data(), (size_t)n_blocks * 8);
+      AMK_CUDA(cudaMemcpyAsync(h->ws + h->wl.slice_tab, slices.data(), slices.size() * 8, cudaMemcpyHostToDevice, stream));
+      AMK_CUDA(cudaMemcpyAsync(h->ws + h->wl.tile_begin, tile_begin.data(), tile_begin.size() * 4,
+                               cudaMemcpyHostToDevice, stream));
+      AMK_CUDA(cudaMemcpyAsync(h->ws + h->wl.tiles, tiles.data(), tiles.size() * 8, cudaMemcpyHostToDevice, stream));
+      // rotary table (cos, sin)[pos][i], angles formed in double
       const int half = hd / 2;
       std::vector<float2> tab((size_t)cfg->max_seq * half);
       for (int i = 0; i < half; i++) {
         const double f = std::pow((double)cfg->rope_theta, -2.0 * (double)i / (double)hd);
-        for (uint32_t s = 0; s < cfg->max_seq; s++) {
-          const double phi = (double)s * f;
-          tab[(size_t)s * half + i] = make_float2((float)std::cos(phi), (float)std::sin(phi));
+        for (uint32_t sp = 0; sp < cfg->max_seq; sp++) {
+          const double phi = (double)sp * f;
+          tab[(size_t)sp * half + i] = make_float2((float)std::cos(phi), (float)std::sin(phi));
         }
       }
       AMK_CUDA(cudaMemcpyAsync(h->ws + h->wl.rope, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice,
                                stream));
-      AMK_CUDA(cudaStreamSynchronize(stream));     // `tab` and the op table are pageable host memory
+      AMK_CUDA(cudaStreamSynchronize(stream));     // the host vectors above are pageable memory
     }
 
     // ---- pack the weights ---------------------------------------------------------------------------------
     for (size_t i = 0; i < h->pl.ops.size(); i++) {
-      const OpDesc& d = h->pl.ops[i];
+      const PlanOp& op = h->pl.ops[i];
+      PackOp d;
+      d.s = op.s; d.rot = op.rot; d.region_off = op.region_off; d.scale_off = op.scale_off;
+      d.slice_off = (const unsigned long long*)(h->ws + h->wl.slice_tab) + i * (size_t)n_blocks;
       PackSrc s;
       memset(&s, 0, sizeof(s));
-      const int l = d.layer;
+      const int l = op.layer;
       auto lin = [&](int slot, int which) {
         s.w[slot] = wts->linear[which][l];
         s.scale[slot] = (cfg->wdtype != AMK_W_BF16) ? wts->scale[which][l] : nullptr;
@@ -306,7 +394,7 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
         return s.w[slot] && (cfg->wdtype == AMK_W_BF16 || s.scale[slot]) && (cfg->wdtype != AMK_W_INT4 || s.zero[slot]);
       };
       bool okp = true;
-      switch (d.kind) {
+      switch (op.kind) {
         case OP_QKV:
           s.mode = 1; s.rows0 = qd; s.rows1 = qd + cfg->n_kv_heads * hd;
           okp = lin(0, AMK_LIN_Q) & lin(1, AMK_LIN_K) & lin(2, AMK_LIN_V);
@@ -335,16 +423,21 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     KParams& p = h->base;
     p.H = H; p.L = L; p.nq = cfg->n_q_heads; p.nkv = cfg->n_kv_heads; p.hd = hd; p.I = I; p.V = cfg->vocab;
     p.S = cfg->max_seq; p.n_rep = n_rep; p.eps = cfg->rms_eps; p.flags = (int)cfg->flags;
-    p.ops = (const OpDesc*)(h->ws + h->wl.ops);
-    p.n_ops = (int)h->pl.ops.size();
+    p.sync_mode = (int)cfg->sync_mode;
+    for (int k = 0; k < 5; k++) p.shape[k] = h->pl.shape[k];
     p.packed = h->packed;
+    p.tiles = (const unsigned long long*)(h->ws + h->wl.tiles);
+    p.tile_begin = (const unsigned*)(h->ws + h->wl.tile_begin);
+    p.scale_base = h->pl.scale_base;
+    p.scale_layer_stride = (unsigned)h->pl.scale_layer_stride;
+    for (int k = 0; k < 4; k++) p.scale_kind_off[k] = (unsigned)h->pl.scale_kind_off[k];
     p.embed = (const unsigned short*)(h->packed + h->pl.embed_off);
     p.attn_norm = (const unsigned short*)(h->packed + h->pl.attn_norm_off);
     p.mlp_norm = (const unsigned short*)(h->packed + h->pl.mlp_norm_off);
     p.final_norm = (const unsigned short*)(h->packed + h->pl.final_norm_off);
     p.rope = (const float2*)(h->ws + h->wl.rope);
-    p.x_a = (float*)(h->ws + h->wl.x_a); p.x_b = (float*)(h->ws + h->wl.x_b);
-    p.qkv = (float*)(h->ws + h->wl.qkv); p.o = (float*)(h->ws + h->wl.o); p.m = (float*)(h->ws + h->wl.m);
+    p.x_a = (ActPair*)(h->ws + h->wl.x_a); p.x_b = (ActPair*)(h->ws + h->wl.x_b);
+    p.qkv = (ActPair*)(h->ws + h->wl.qkv); p.o = (ActPair*)(h->ws + h->wl.o); p.m = (ActPair*)(h->ws + h->wl.m);
     p.part = (float*)(h->ws + h->wl.part); p.hidden = (float*)(h->ws + h->wl.hidden);
     p.phase_ctr = (unsigned*)(h->ws + h->wl.phase_ctr); p.group_ctr = (unsigned*)(h->ws + h->wl.group_ctr);
     p.lm_ctr = (unsigned*)(h->ws + h->wl.lm_ctr); p.cand_val = (float*)(h->ws + h->wl.cand_val);
@@ -360,9 +453,10 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     pn.n_blocks = n_blocks; pn.threads = kThreads; pn.smem_bytes = (uint32_t)smem_bytes;
     pn.stage_bytes = stage_bytes; pn.n_stages = n_stages; pn.max_inflight = max_inflight;
     pn.n_gemv_ops = (uint32_t)h->pl.ops.size(); pn.n_phases = 5 * L;
-    pn.packed_bytes = h->pl.total; pn.workspace_bytes = h->wl.total; pn.kv_bytes = kv_bytes_of(cfg);
+    pn.packed_bytes = h->pl.packed_total; pn.workspace_bytes = h->wl.total; pn.kv_bytes = kv_bytes_of(cfg);
     pn.weight_stream_bytes = h->pl.weight_stream_bytes;
     h->epoch = 0;
+    h->ctr_epoch = 0;
   }
   *out = h;
   return AMK_OK;
@@ -379,6 +473,7 @@ static amk_status launch_step(amk_handle* h, int32_t token, const int* token_ptr
   p.token_ptr = token_ptr;
   p.pos = pos;
   p.epoch = ++h->epoch;
+  p.ctr_epoch = ++h->ctr_epoch;
   const size_t half = kv_bytes_of(&h->cfg) / 2;
   p.kcache = (unsigned short*)kv;
   p.vcache = (unsigned short*)((unsigned char*)kv + half);
@@ -391,6 +486,7 @@ static amk_status launch_step(amk_handle* h, int32_t token, const int* token_ptr
   cudaError_t e = launch_decode(p, (int)h->plan.n_blocks, h->plan.smem_bytes, stream);
   if (e != cudaSuccess) {
     --h->epoch;
+    --h->ctr_epoch;
     snprintf(h->errmsg, sizeof(h->errmsg), "cooperative launch: %s", cudaGetErrorString(e));
     return AMK_ERR_CUDA;
   }
@@ -439,8 +535,10 @@ amk_status amk_last_status(amk_handle* h, amk_status* st, char* msg, size_t n) {
     // the step did not finish: its counters are inconsistent, start over from zero
     e = cudaMemset(h->ws + h->wl.status, 0, sizeof(DevStatus));
     if (e == cudaSuccess) e = cudaMemset(h->ws + h->wl.phase_ctr, 0, h->wl.cand_val - h->wl.phase_ctr);
+    // (the activation buffers need no reset: the next step's sequence numbers differ from anything in them)
     if (e != cudaSuccess) return AMK_ERR_CUDA;
-    h->epoch = 0;
+    // the counters restart from zero; the sequence numbers keep growing
+    h->ctr_epoch = 0;
   }
   return AMK_OK;
 }
@@ -496,7 +594,11 @@ amk_status amk_debug_unpack(amk_handle* h, int layer, int which, void* out_dev, 
   s.w[slot] = out_dev;
   s.scale[slot] = scale_dev;
   s.zero[slot] = zero_dev;
-  cudaError_t e = launch_pack(h->pl.ops[op], s, h->packed, (int)h->plan.n_blocks, (int)h->plan.stage_bytes, true,
+  const PlanOp& po = h->pl.ops[op];
+  PackOp d;
+  d.s = po.s; d.rot = po.rot; d.region_off = po.region_off; d.scale_off = po.scale_off;
+  d.slice_off = (const unsigned long long*)(h->ws + h->wl.slice_tab) + (size_t)op * h->plan.n_blocks;
+  cudaError_t e = launch_pack(d, s, h->packed, (int)h->plan.n_blocks, (int)h->plan.stage_bytes, true,
                               (cudaStream_t)cuda_stream);
   return e == cudaSuccess ? AMK_OK : AMK_ERR_CUDA;
 }

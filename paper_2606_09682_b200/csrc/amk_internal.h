@@ -11,10 +11,10 @@ namespace amk {
 struct DevStatus {
   unsigned abort;     // nonzero: leave as soon as possible
   unsigned code;      // amk_status of the first failure
-  int phase;          // dependency join that timed out (-1: ring wait)
+  int phase;          // task whose input never arrived / join that timed out (-1, -2: ring waits)
   int block;          // block that reported
-  unsigned seen;      // counter value seen
-  unsigned want;      // counter value waited for
+  unsigned seen;      // value seen
+  unsigned want;      // value waited for
   unsigned pad[2];
 };
 
@@ -22,13 +22,20 @@ struct DevStatus {
 struct SmemHeader {
   uint64_t full[kMaxStages];
   uint64_t empty[kMaxStages];
-  float red[2][kPassRows];           // cross-k-warp partial sums of a pass (double-buffered)
-  float warp_part[kConsumerWarps];   // block reductions (sum of squares)
+  float red[2][kPassRows];           // cross-k-warp partial sums of a pass: [Wk][R], Wk * R <= warps * kGMax
+  float warp_part[2][kConsumerWarps];  // block reductions (sum of squares, max)
   float cand_val[kConsumerWarps];
   int cand_idx[kConsumerWarps];
-  volatile int abort;                // block-local copy of the abort decision
   int flag;                          // "this block arrived last" broadcast
-  int pad[2];
+  int pad[3];
+};
+
+// An activation element in global memory: the value and the sequence number of the task that wrote it.
+// One aligned 8-byte store publishes both, so a reader that sees the expected sequence number has the
+// value: no fence and no separate flag are needed.
+struct __align__(8) ActPair {
+  float v;
+  unsigned seq;
 };
 
 // Kernel argument, passed by value.
@@ -37,10 +44,15 @@ struct KParams {
   int H, L, nq, nkv, hd, I, V, S, n_rep;
   float eps;
   int flags;
-  // tables and weights
-  const OpDesc* ops;
-  int n_ops;
+  int sync_mode;                          // 0: counter joins (acquire/release) as well; 1: data-carried sequence numbers only
+  OpShape shape[5];                       // per OpKind
+  // weights
   const unsigned char* packed;            // packed buffer base
+  const unsigned long long* tiles;        // per block: its ring tiles {offset/16 | bytes/16 << 40}, in stream order
+  const unsigned* tile_begin;             // [n_blocks + 1] index of each block's first tile
+  unsigned long long scale_base;          // int8: fp16 row scales, op-major in virtual row order
+  unsigned scale_layer_stride;            // bytes per layer
+  unsigned scale_kind_off[4];             // byte offset of each op kind inside a layer's scales
   const unsigned short* embed;            // bf16 [V][H], canonical copy
   const unsigned short* attn_norm;        // bf16 [L][H]
   const unsigned short* mlp_norm;         // bf16 [L][H]
@@ -50,22 +62,23 @@ struct KParams {
   int token;
   const int* token_ptr;                   // if non-null the token is read from device memory
   int pos;
-  unsigned epoch;                         // counters of this step count up to epoch * n_blocks
+  unsigned epoch;                         // step number: sequence numbers never repeat
+  unsigned ctr_epoch;                     // steps since the counters were last zeroed
   // caller buffers
   unsigned short* kcache;
   unsigned short* vcache;
   float* logits;
   int* next_token;
   // workspace
-  float* x_a;
-  float* x_b;
-  float* qkv;
-  float* o;
-  float* m;
+  ActPair* x_a;                           // residual stream entering a layer
+  ActPair* x_b;                           // residual stream after attention
+  ActPair* qkv;
+  ActPair* o;
+  ActPair* m;
   float* part;                            // [nq][kMaxChunks][hd + 2]
   float* hidden;                          // [(L+1)][H]
   unsigned* phase_ctr;                    // [5 L]
-  unsigned* group_ctr;                    // [nkv]
+  unsigned* group_ctr;                    // [L][nkv]
   unsigned* lm_ctr;
   float* cand_val;                        // [n_blocks]
   int* cand_idx;
@@ -76,13 +89,21 @@ struct KParams {
   int stage_bytes, n_stages, max_inflight;
   int act_bytes;                          // activation / attention scratch area in shared memory
   unsigned long long timeout_ns;
-  int drop_phase, drop_block;             // test hook: this block skips this signal
+  int drop_phase, drop_block;             // test hook: this block does not publish this task's output
 };
 
 // Launchers implemented in the .cu files.
 cudaError_t launch_decode(const KParams& p, int n_blocks, size_t smem_bytes, cudaStream_t stream);
 cudaError_t decode_kernel_attrs(size_t smem_bytes, int* max_blocks_per_sm);
 
+// One op to pack: its shape, rotation and region, plus where the canonical rows come from.
+struct PackOp {
+  OpShape s;
+  int rot;
+  unsigned long long region_off;          // byte offset of the op's region in the packed buffer
+  const unsigned long long* slice_off;    // DEVICE [n_blocks]: byte offset of each slot's slice inside the region
+  unsigned long long scale_off;           // int8: byte offset of the fp16 row scales (virtual row order)
+};
 struct PackSrc {
   const void* w[3];
   const void* scale[3];
@@ -90,7 +111,7 @@ struct PackSrc {
   int mode;        // 0 single matrix, 1 three matrices stacked (rows0, rows1 boundaries), 2 two matrices interleaved
   int rows0, rows1;
 };
-cudaError_t launch_pack(const OpDesc& d, const PackSrc& src, unsigned char* packed, int n_blocks, int stage_bytes,
+cudaError_t launch_pack(const PackOp& d, const PackSrc& src, unsigned char* packed, int n_blocks, int stage_bytes,
                         bool inverse, cudaStream_t stream);
 cudaError_t launch_quantize_int8(const void* w, int64_t rows, int64_t cols, void* q, void* scale, cudaStream_t s);
 cudaError_t launch_quantize_int4(const void* w, int64_t rows, int64_t cols, void* packed, void* scale, void* zero,

@@ -1,21 +1,28 @@
 // The decode step as one persistent cooperative kernel for sm_100a: one block per SM, each block walks
-// its statically known queue of tasks -- wait on a dependency counter, compute, signal -- as in the
-// paper's per-SM scheduler loop (Algorithm 1) and counter model (Section 4, "Synchronization model").
+// its statically known queue of tasks -- wait for the inputs, compute, publish -- as in the paper's
+// per-SM scheduler loop (Algorithm 1) and counter model (Section 4, "Synchronization model").
 //
 // What is different from the paper's kernel (written for sm_75..sm_120, where it found the per-tile
 // cross-SM synchronisation to be the limiter, Section 7):
 //   * Weights do not depend on activations, so a dedicated producer warp streams this block's packed
-//     weight bytes -- one contiguous run per block for the whole token -- through a shared-memory ring
-//     with bulk asynchronous copies (TMA) and mbarriers, running ahead across dependency joins.  The
-//     HBM pipe keeps flowing while the consumer warps wait for an activation.
-//   * One counter per join instead of one per tile: five joins per layer, every block signals each once.
-//     Counters are never reset: step e waits for e * n_blocks.
+//     weight bytes through a shared-memory ring with bulk asynchronous copies (TMA) and mbarriers,
+//     running ahead across dependencies: the HBM pipe keeps flowing while consumers wait for an input.
+//   * Activations travel as {value, sequence number} pairs written with one 8-byte store, so a reader
+//     that sees the task's sequence number has the value: producers need no fence and readers no separate
+//     flag.  The paper's release-increment / acquire-spin counters are kept as an optional second layer
+//     (sync_mode 0: one counter per join, every block signals each once, never reset: step e waits for
+//     e * n_blocks) so the two can be measured against each other.
+//   * The matrix-vector products run on the tensor cores (warp-level mma, fragments loaded with ldmatrix
+//     straight from the ring): the activation vector occupies two (bf16: high and low halves) or three
+//     (int8 / int4: base-128 digits) of the eight B columns, so nothing is converted per weight and the
+//     result keeps fp32 / exact-integer accuracy.  A scalar loop needs ~2 instructions per weight; the
+//     traced consumer was 3x slower than the HBM stream with it.
 //   * RMSNorm is folded into the consuming GEMV's prologue, RoPE and the KV append into the attention
 //     task, SiLU*up and the residual adds into GEMV epilogues, the split-K combine and the global argmax
 //     into "last arriver finishes" steps, so no extra joins are needed.
 //   * Every wait is bounded; on expiry the block records the failure and every block drains and exits.
-#include <cuda_runtime.h>
 #include <cuda_fp16.h>
+#include <cuda_runtime.h>
 #include <math_constants.h>
 
 #include "amk.h"
@@ -26,18 +33,23 @@ namespace amk {
 
 namespace {
 
-constexpr int kBarCons = 1;       // named barrier of the consumer warps
-constexpr int kOutWarps = (kPassRows + 31) / 32;   // warps that hold a pass's output rows
-constexpr int kNormVec = 4;       // float4 slots per thread held in registers by a norm prologue (H <= 8192)
+constexpr int kBarCons = 1;                          // named barrier of the consumer warps
+constexpr int kOutWarps = (kPassRows + 31) / 32;     // warps that hold a pass's output rows
+constexpr int kLines = 16;                           // 16-byte activation lines per thread (K <= 2 * 480 * 16)
+constexpr int kBatch = 8;                            // lines gathered at a time
+constexpr int kNormLines = 8;                        // lines per thread of a normed input (H <= 7680)
+constexpr float kDigitScale = 1048575.0f;            // int8 / int4 activations: 3 signed base-128 digits
 
 struct Ctx {
   const KParams& p;
   SmemHeader* sh;
-  float* xs;             // activation vector of the current op / attention scratch
+  unsigned char* xs;     // activation area (bf16 hi/lo halves or int8 digits) / attention scratch
   unsigned char* ring;
   int tid, warp, lane, cta, nblk;
-  unsigned tile_ctr;     // ring tiles this warp has walked
+  int stage;             // ring stage of the next tile this warp walks
+  unsigned parity;       // its phase parity
   int token;
+  float xscale;          // int8 / int4: scale of the digit representation of the current input vector
   bool bad;              // this thread saw a failure; agreed on at the next consumer barrier
 };
 
@@ -102,16 +114,23 @@ __device__ __forceinline__ bool wait_mbar(const KParams& p, uint64_t* bar, unsig
   return wait_mbar_slow(p, bar, parity, kind);
 }
 
-// All consumer threads: wait until every block has signalled `phase` in this step.
+// Sequence number carried by everything task `task` publishes in this step (never 0).
+__device__ __forceinline__ unsigned seq_of(const KParams& p, int task) {
+  return p.epoch * (unsigned)(5 * p.L + 1) + (unsigned)task + 1u;
+}
+
+// Counter layer (sync_mode 0): all consumer threads wait until every block has signalled `phase`.
 __device__ __forceinline__ bool wait_phase(Ctx& c, int phase) {
+  if (c.p.sync_mode != 0) return true;
   if (c.tid == 0) {
-    if (!poll_counter(c.p, c.p.phase_ctr + phase, c.p.epoch * (unsigned)c.nblk, phase)) c.bad = true;
+    if (!poll_counter(c.p, c.p.phase_ctr + phase, c.p.ctr_epoch * (unsigned)c.nblk, phase)) c.bad = true;
   }
   c.bad = cons_sync_or(c.bad);
   return !c.bad;
 }
 // Called after a consumer barrier that follows the task's last store: release-increment the counter.
 __device__ __forceinline__ void signal_phase(Ctx& c, int phase) {
+  if (c.p.sync_mode != 0) return;
   if (c.tid == 0 && !(phase == c.p.drop_phase && c.cta == c.p.drop_block))
     red_release_gpu_add(c.p.phase_ctr + phase, 1u);
 }
@@ -126,261 +145,388 @@ __device__ __forceinline__ float warp_sum(float v) {
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   return v;
 }
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// Spin until both elements of the line at `addr` carry `seq`; bounded.
+__device__ __noinline__ bool poll_pair2_slow(const KParams& p, const void* addr, unsigned seq, int task, uint4* out) {
+  const unsigned long long t0 = globaltimer_ns();
+  unsigned spins = 0;
+  for (;;) {
+    const uint4 v = ld_pair2(addr);
+    if (v.y == seq && v.w == seq) { *out = v; return true; }
+    if ((++spins & 15u) == 0u) {
+      if (ld_relaxed_gpu(&p.status->abort)) return false;
+      if (globaltimer_ns() - t0 > p.timeout_ns) {
+        report_failure(p, (unsigned)AMK_ERR_TIMEOUT, task, v.y == seq ? v.w : v.y, seq);
+        return false;
+      }
+    }
+  }
+}
+__device__ __noinline__ bool poll_pair_slow(const KParams& p, const void* addr, unsigned seq, int task, float* out) {
+  const unsigned long long t0 = globaltimer_ns();
+  unsigned spins = 0;
+  for (;;) {
+    const uint2 v = ld_pair(addr);
+    if (v.y == seq) { *out = __uint_as_float(v.x); return true; }
+    if ((++spins & 15u) == 0u) {
+      if (ld_relaxed_gpu(&p.status->abort)) return false;
+      if (globaltimer_ns() - t0 > p.timeout_ns) {
+        report_failure(p, (unsigned)AMK_ERR_TIMEOUT, task, v.y, seq);
+        return false;
+      }
+    }
+  }
+}
+// One activation element written by `task` in this step.
+__device__ __forceinline__ float read_act(Ctx& c, const ActPair* a, unsigned seq, int task) {
+  const uint2 v = ld_pair(a);
+  if (v.y == seq) return __uint_as_float(v.x);
+  float r = 0.f;
+  if (!poll_pair_slow(c.p, a, seq, task, &r)) c.bad = true;
+  return r;
+}
+
+__device__ __forceinline__ float silu_f(float z) { return z / (1.0f + expf(-z)); }
 
 // ------------------------------------------------------------------------------------------------
-// dot product of one lane's 8 weights of one row chunk with its 8 activations
+// Prologue of a matrix-vector product: bring the input vector (K elements written by `src_task`, or the
+// embedding row) into shared memory in the form the tensor cores take, with RMSNorm folded in.
+//   bf16 weights: X0[K] = bf16(a), X1[K] = bf16(a - X0): two B columns whose sum is a to ~2^-17.
+//   int8 / int4 : a / scale as three signed base-128 digits D2, D1, D0 (three B columns), exact integers.
 // ------------------------------------------------------------------------------------------------
-template <int WD>
-__device__ __forceinline__ float dot8(const unsigned char* row, int lane, const float4& x0, const float4& x1);
-
-template <>
-__device__ __forceinline__ float dot8<W_BF16>(const unsigned char* row, int lane, const float4& x0, const float4& x1) {
-  const uint4 w = *reinterpret_cast<const uint4*>(row + lane * 16);
-  float s0 = bf16_lo(w.x) * x0.x;
-  float s1 = bf16_lo(w.z) * x1.x;
-  s0 = fmaf(bf16_hi(w.x), x0.y, s0);
-  s1 = fmaf(bf16_hi(w.z), x1.y, s1);
-  s0 = fmaf(bf16_lo(w.y), x0.z, s0);
-  s1 = fmaf(bf16_lo(w.w), x1.z, s1);
-  s0 = fmaf(bf16_hi(w.y), x0.w, s0);
-  s1 = fmaf(bf16_hi(w.w), x1.w, s1);
-  return s0 + s1;
-}
-
-// int8 codes are stored biased (q + 128) so that one byte-permute builds the float 2^23 + (q + 128).
-__device__ __forceinline__ float u8_to_f32_biased(unsigned w, unsigned sel) {
-  return __uint_as_float(__byte_perm(w, 0x4B000000u, sel)) - 8388736.0f;   // 2^23 + 128
-}
-template <>
-__device__ __forceinline__ float dot8<W_INT8>(const unsigned char* row, int lane, const float4& x0, const float4& x1) {
-  const uint2 w = *reinterpret_cast<const uint2*>(row + lane * 8);
-  float s0 = u8_to_f32_biased(w.x, 0x7540u) * x0.x;
-  float s1 = u8_to_f32_biased(w.y, 0x7540u) * x1.x;
-  s0 = fmaf(u8_to_f32_biased(w.x, 0x7541u), x0.y, s0);
-  s1 = fmaf(u8_to_f32_biased(w.y, 0x7541u), x1.y, s1);
-  s0 = fmaf(u8_to_f32_biased(w.x, 0x7542u), x0.z, s0);
-  s1 = fmaf(u8_to_f32_biased(w.y, 0x7542u), x1.z, s1);
-  s0 = fmaf(u8_to_f32_biased(w.x, 0x7543u), x0.w, s0);
-  s1 = fmaf(u8_to_f32_biased(w.y, 0x7543u), x1.w, s1);
-  return s0 + s1;
-}
-
-// int4: 8 codes in one word (element e in nibble e); the row chunk ends with fp16 {s, z} of group 2b and 2b+1.
-__device__ __forceinline__ float u4_to_f32(unsigned w, int e, float zbias) {
-  return __uint_as_float(((w >> (4 * e)) & 0xFu) | 0x4B000000u) - zbias;           // (2^23 + q) - (2^23 + z)
-}
-template <>
-__device__ __forceinline__ float dot8<W_INT4>(const unsigned char* row, int lane, const float4& x0, const float4& x1) {
-  const unsigned w = *reinterpret_cast<const unsigned*>(row + lane * 4);
-  const uint2 sz = *reinterpret_cast<const uint2*>(row + 128);
-  const float sA = __half2float(__ushort_as_half((unsigned short)(sz.x & 0xffffu)));
-  const float zA = __half2float(__ushort_as_half((unsigned short)(sz.x >> 16))) + 8388608.0f;
-  const float sB = __half2float(__ushort_as_half((unsigned short)(sz.y & 0xffffu)));
-  const float zB = __half2float(__ushort_as_half((unsigned short)(sz.y >> 16))) + 8388608.0f;
-  float s0 = u4_to_f32(w, 0, zA) * x0.x;
-  float s1 = u4_to_f32(w, 4, zB) * x1.x;
-  s0 = fmaf(u4_to_f32(w, 1, zA), x0.y, s0);
-  s1 = fmaf(u4_to_f32(w, 5, zB), x1.y, s1);
-  s0 = fmaf(u4_to_f32(w, 2, zA), x0.z, s0);
-  s1 = fmaf(u4_to_f32(w, 6, zB), x1.z, s1);
-  s0 = fmaf(u4_to_f32(w, 3, zA), x0.w, s0);
-  s1 = fmaf(u4_to_f32(w, 7, zB), x1.w, s1);
-  return fmaf(sA, s0, sB * s1);
-}
-
-// ------------------------------------------------------------------------------------------------
-// One pass: this warp walks every ring tile of the pass, accumulates its G rows over its column
-// blocks, then publishes the warp sums for the cross-k-warp reduction.
-// ------------------------------------------------------------------------------------------------
-template <int G, int WD>
-__device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, float* red) {
+__device__ __forceinline__ bool load_input(Ctx& c, int wd, int K, const ActPair* src, unsigned seq, int src_task,
+                                           const unsigned short* embed_row, const unsigned short* normw, int task) {
   const KParams& p = c.p;
-  const int wr = c.warp % g.Wr, wk = c.warp / g.Wr;
-  const bool active = wk < g.Wk;
-  const int my_rows = active ? min(G, g.R - wr * G) : 0;
-  float acc[G];
+  const int n2 = K >> 1;                               // lines of two elements
+  float2 v[kLines];
+  unsigned gw[kNormLines];
+  if (normw) {
 #pragma unroll
-  for (int i = 0; i < G; i++) acc[i] = 0.f;
-  const int S = p.n_stages;
-  for (int t = 0; t < g.n_tiles; ++t) {
-    const int stage = (int)(c.tile_ctr % (unsigned)S);
-    const unsigned parity = (c.tile_ctr / (unsigned)S) & 1u;
-    if (!c.bad && !wait_mbar(p, &c.sh->full[stage], parity, -1)) c.bad = true;
-    if (active && !c.bad) {
-      const int u0 = t * g.upt;
-      const int u1 = min(u0 + g.upt, g.n_units);
-      const unsigned char* sbase = c.ring + (size_t)stage * p.stage_bytes - unit_off(g, u0);
-      int b = (u0 > wr) ? (u0 - wr + g.Wr - 1) / g.Wr : 0;            // first column block of row-warp wr in this tile
-      b += ((wk - b) % g.Wk + g.Wk) % g.Wk;                           // first one owned by k-warp wk
-      for (; b * g.Wr + wr < u1; b += g.Wk) {
-        const bool is_tail = g.tail && (b == g.nblk - 1);
-        const int wd = is_tail ? g.tail : kBlockCols;
-        const int rc = is_tail ? g.rc_tail : g.rc_full;
-        const unsigned char* up = sbase + unit_off_br(g, b, wr);
-        if (c.lane < (wd >> 3)) {
-          const float4 x0 = *reinterpret_cast<const float4*>(c.xs + b * kBlockCols + 4 * c.lane);
-          const float4 x1 = *reinterpret_cast<const float4*>(c.xs + b * kBlockCols + (wd >> 1) + 4 * c.lane);
+    for (int i = 0; i < kNormLines; i++) {
+      const int ln = c.tid + i * kConsumerThreads;
+      gw[i] = (ln < n2) ? __ldg(reinterpret_cast<const unsigned*>(normw) + ln) : 0u;
+    }
+  }
+  float ss = 0.f, amax = 0.f;
 #pragma unroll
-          for (int i = 0; i < G; i++)
-            if (i < my_rows) acc[i] += dot8<WD>(up + i * rc, c.lane, x0, x1);
+  for (int i0 = 0; i0 < kLines; i0 += kBatch) {
+    if (i0 * kConsumerThreads >= n2) break;
+    // issue a batch of loads first, then settle the ones that had not arrived
+    uint4 raw[kBatch];
+#pragma unroll
+    for (int i = 0; i < kBatch; i++) {
+      const int ln = c.tid + (i0 + i) * kConsumerThreads;
+      if (ln < n2) {
+        if (embed_row) {
+          const unsigned w = __ldg(reinterpret_cast<const unsigned*>(embed_row) + ln);
+          raw[i] = make_uint4(w << 16, seq, w & 0xffff0000u, seq);
+        } else {
+          raw[i] = ld_pair2(src + 2 * ln);
         }
       }
     }
-    __syncwarp();
-    if (c.lane == 0 && !c.bad) mbar_arrive(&c.sh->empty[stage]);
-    c.tile_ctr++;
-  }
 #pragma unroll
-  for (int i = 0; i < G; i++) acc[i] = warp_sum(acc[i]);
-  if (active && c.lane == 0) {
-#pragma unroll
-    for (int i = 0; i < G; i++)
-      if (i < my_rows) red[wk * g.R + wr * G + i] = acc[i];     // [Wk][R]: Wk * R <= warps * kGMax
+    for (int i = 0; i < kBatch; i++) {
+      const int ln = c.tid + (i0 + i) * kConsumerThreads;
+      if (ln < n2) {
+        if (raw[i].y != seq || raw[i].w != seq) {
+          if (!poll_pair2_slow(p, src + 2 * ln, seq, src_task, &raw[i])) c.bad = true;
+        }
+        float a = __uint_as_float(raw[i].x), b = __uint_as_float(raw[i].z);
+        if (normw) {
+          ss = fmaf(a, a, ss);
+          ss = fmaf(b, b, ss);
+          if (embed_row && c.cta == 0 && (p.flags & AMK_FLAG_DEBUG_HIDDEN))
+            reinterpret_cast<float2*>(p.hidden)[ln] = make_float2(a, b);
+          if (i0 + i < kNormLines) { a *= bf16_lo(gw[(i0 + i) % kNormLines]); b *= bf16_hi(gw[(i0 + i) % kNormLines]); }
+        }
+        v[i0 + i] = make_float2(a, b);                 // norm weight applied; 1/rms follows the sum
+        amax = fmaxf(amax, fmaxf(fabsf(a), fabsf(b)));
+      }
+    }
   }
+  if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_JOINED);
+  float r = 1.0f;
+  if (normw || wd != W_BF16) {
+    ss = warp_sum(ss);
+    amax = warp_max(amax);
+    if (c.lane == 0) { c.sh->warp_part[0][c.warp] = ss; c.sh->warp_part[1][c.warp] = amax; }
+    c.bad = cons_sync_or(c.bad);
+    if (c.bad) return false;
+    float tot = 0.f, mx = 0.f;
+#pragma unroll
+    for (int w = 0; w < kConsumerWarps; w++) { tot += c.sh->warp_part[0][w]; mx = fmaxf(mx, c.sh->warp_part[1][w]); }
+    if (normw) r = 1.0f / sqrtf(tot / (float)K + p.eps);
+    amax = mx * r;
+  }
+  if (wd == W_BF16) {
+    unsigned* X0 = reinterpret_cast<unsigned*>(c.xs);
+    unsigned* X1 = X0 + n2;
+#pragma unroll
+    for (int i = 0; i < kLines; i++) {
+      const int ln = c.tid + i * kConsumerThreads;
+      if (ln < n2) {
+        const float a = v[i].x * r, b = v[i].y * r;
+        const unsigned ha = f32_to_bf16_rne(a), hb = f32_to_bf16_rne(b);
+        const unsigned la = f32_to_bf16_rne(a - __uint_as_float(ha << 16));
+        const unsigned lb = f32_to_bf16_rne(b - __uint_as_float(hb << 16));
+        X0[ln] = ha | (hb << 16);
+        X1[ln] = la | (lb << 16);
+      }
+    }
+  } else {
+    const float inv = amax > 0.f ? kDigitScale / amax : 0.f;
+    c.xscale = amax / kDigitScale;
+    unsigned short* D2 = reinterpret_cast<unsigned short*>(c.xs);
+    unsigned short* D1 = D2 + n2;
+    unsigned short* D0 = D1 + n2;
+#pragma unroll
+    for (int i = 0; i < kLines; i++) {
+      const int ln = c.tid + i * kConsumerThreads;
+      if (ln < n2) {
+        unsigned d2 = 0, d1 = 0, d0 = 0;
+#pragma unroll
+        for (int e = 0; e < 2; e++) {
+          const int X = __float2int_rn((e ? v[i].y : v[i].x) * r * inv);
+          const int e0 = ((X + 64) & 127) - 64;
+          const int X1 = (X - e0) >> 7;
+          const int e1 = ((X1 + 64) & 127) - 64;
+          const int e2 = (X1 - e1) >> 7;
+          d0 |= (unsigned)(e0 & 0xff) << (8 * e);
+          d1 |= (unsigned)(e1 & 0xff) << (8 * e);
+          d2 |= (unsigned)(e2 & 0xff) << (8 * e);
+        }
+        D2[ln] = (unsigned short)d2;
+        D1[ln] = (unsigned short)d1;
+        D0[ln] = (unsigned short)d0;
+      }
+    }
+  }
+  c.bad = cons_sync_or(c.bad);
+  return !c.bad;
 }
+
+// ------------------------------------------------------------------------------------------------
+// One pass on the tensor cores: this warp walks every ring tile of the pass, multiplies its row group
+// (<= 16 rows, one m16 tile) by the input columns over its column blocks, and publishes per-row sums.
+// ------------------------------------------------------------------------------------------------
+#define AMK_LO(x, z) ((((x) & 0x0F0F0F0Fu) + (z)) ^ 0x80808080u)
+#define AMK_HI(x, z) (((((x) >> 4) & 0x0F0F0F0Fu) + (z)) ^ 0x80808080u)
 
 template <int WD>
-__device__ __forceinline__ void consume_pass_g(Ctx& c, const PassGeom& g, float* red) {
-  switch (g.G) {
-    case 1: consume_pass<1, WD>(c, g, red); break;
-    case 2: consume_pass<2, WD>(c, g, red); break;
-    case 3: consume_pass<3, WD>(c, g, red); break;
-    case 4: consume_pass<4, WD>(c, g, red); break;
-    case 5: consume_pass<5, WD>(c, g, red); break;
-    case 6: consume_pass<6, WD>(c, g, red); break;
-    case 7: consume_pass<7, WD>(c, g, red); break;
-    default: consume_pass<8, WD>(c, g, red); break;
+__device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int K, float* red) {
+  const KParams& p = c.p;
+  const int wr = c.warp % g.Wr, wk = c.warp / g.Wr;
+  const bool active = wk < g.Wk;
+  const int urows = (wr == g.Wr - 1) ? g.g_last : g.G;
+  const int gq = c.lane >> 2, q = c.lane & 3;                                  // fragment row / column-pair index
+  const int mrow = min((c.lane & 7) + ((c.lane >> 3) & 1) * 8, urows - 1);     // ldmatrix: my row of my 8x8 matrix
+  const unsigned lane_off = (unsigned)(((c.lane >> 4) * urows + mrow) * 16);   // chunk half h = lane / 16
+  const unsigned step_stride = (unsigned)(2 * urows * 16);                     // two chunks per k step
+  const int S = p.n_stages;
+  constexpr int BC = (WD == W_INT4) ? 128 : 64;
+  constexpr int NCOL = (WD == W_BF16) ? 2 : 3;                                  // B columns in use
+  const unsigned char* xcol = c.xs + (size_t)min(gq, NCOL - 1) * K * (WD == W_BF16 ? 2 : 1);
+
+  float facc[4] = {0.f, 0.f, 0.f, 0.f};
+  int iacc[4] = {0, 0, 0, 0};
+  int next_b = wk;                                   // my next column block
+  const int my_off = wr * g.ub_full;
+  // first unit of the current tile as (block, row-warp), and the step from one tile to the next
+  int t_b = 0, t_r = 0;
+  const int step_b = g.upt / g.Wr, step_r = g.upt - step_b * g.Wr;
+  for (int t = 0; t < g.n_tiles; ++t) {
+    const int tile_off = t_b * g.bb + t_r * g.ub_full;
+    int n_b = t_b + step_b, n_r = t_r + step_r;      // first unit of the next tile
+    if (n_r >= g.Wr) { n_r -= g.Wr; n_b++; }
+    if (!c.bad && !wait_mbar(p, &c.sh->full[c.stage], c.parity, -1)) c.bad = true;
+    if (active && !c.bad) {
+      const unsigned char* sbase = c.ring + (size_t)c.stage * p.stage_bytes;
+      // my units in this tile: blocks next_b, next_b + Wk, ... while (b, wr) comes before (n_b, n_r)
+      while (next_b < g.nblk && (next_b < n_b || (next_b == n_b && wr < n_r))) {
+        const unsigned char* u = sbase + (next_b * g.bb + my_off - tile_off);
+        if (WD == W_BF16) {
+          uint4 xb0 = make_uint4(0u, 0u, 0u, 0u), xb1 = xb0;
+          if (gq < NCOL) {
+            const uint4* xp = reinterpret_cast<const uint4*>(xcol + ((size_t)next_b * BC + 16 * q) * 2);
+            xb0 = xp[0];
+            xb1 = xp[1];
+          }
+          unsigned a[4];
+          ldmatrix_x4(a, u + lane_off);
+          mma_bf16(facc, a, xb0.x, xb0.y);
+          ldmatrix_x4(a, u + lane_off + step_stride);
+          mma_bf16(facc, a, xb0.z, xb0.w);
+          ldmatrix_x4(a, u + lane_off + 2 * step_stride);
+          mma_bf16(facc, a, xb1.x, xb1.y);
+          ldmatrix_x4(a, u + lane_off + 3 * step_stride);
+          mma_bf16(facc, a, xb1.z, xb1.w);
+        } else if (WD == W_INT8) {
+          uint4 xb = make_uint4(0u, 0u, 0u, 0u);
+          if (gq < NCOL) xb = *reinterpret_cast<const uint4*>(xcol + (size_t)next_b * BC + 16 * q);
+          unsigned a[4];
+          ldmatrix_x4(a, u + lane_off);
+          mma_s8(iacc, a[0], a[1], a[2], a[3], xb.x, xb.y);
+          ldmatrix_x4(a, u + lane_off + step_stride);
+          mma_s8(iacc, a[0], a[1], a[2], a[3], xb.z, xb.w);
+        } else {
+          uint4 xb0 = make_uint4(0u, 0u, 0u, 0u), xb1 = xb0;
+          if (gq < NCOL) {
+            const uint4* xp = reinterpret_cast<const uint4*>(xcol + (size_t)next_b * BC + 32 * q);
+            xb0 = xp[0];
+            xb1 = xp[1];
+          }
+          // {scale, zero} of my two fragment rows for this group (= this column block)
+          const unsigned* szp = reinterpret_cast<const unsigned*>(u + urows * 64);
+          const unsigned sz0 = szp[min(gq, urows - 1)], sz1 = szp[min(gq + 8, urows - 1)];
+          const float s0 = __half2float(__ushort_as_half((unsigned short)(sz0 & 0xffffu)));
+          const float s1 = __half2float(__ushort_as_half((unsigned short)(sz1 & 0xffffu)));
+          // code - zero as a signed byte: (code + 128 - zero) ^ 0x80; no carries between bytes
+          const unsigned z0 = (unsigned)(128 - (int)__half2float(__ushort_as_half((unsigned short)(sz0 >> 16)))) * 0x01010101u;
+          const unsigned z1 = (unsigned)(128 - (int)__half2float(__ushort_as_half((unsigned short)(sz1 >> 16)))) * 0x01010101u;
+          int g4[4] = {0, 0, 0, 0};
+          unsigned a[4];
+          ldmatrix_x4(a, u + lane_off);
+          mma_s8(g4, AMK_LO(a[0], z0), AMK_LO(a[1], z1), AMK_LO(a[2], z0), AMK_LO(a[3], z1), xb0.x, xb0.y);
+          mma_s8(g4, AMK_HI(a[0], z0), AMK_HI(a[1], z1), AMK_HI(a[2], z0), AMK_HI(a[3], z1), xb0.z, xb0.w);
+          ldmatrix_x4(a, u + lane_off + step_stride);
+          mma_s8(g4, AMK_LO(a[0], z0), AMK_LO(a[1], z1), AMK_LO(a[2], z0), AMK_LO(a[3], z1), xb1.x, xb1.y);
+          mma_s8(g4, AMK_HI(a[0], z0), AMK_HI(a[1], z1), AMK_HI(a[2], z0), AMK_HI(a[3], z1), xb1.z, xb1.w);
+          facc[0] = fmaf(s0, (float)g4[0], facc[0]);
+          facc[1] = fmaf(s0, (float)g4[1], facc[1]);
+          facc[2] = fmaf(s1, (float)g4[2], facc[2]);
+          facc[3] = fmaf(s1, (float)g4[3], facc[3]);
+        }
+        next_b += g.Wk;
+      }
+    }
+    __syncwarp();
+    if (c.lane == 0 && !c.bad) mbar_arrive(&c.sh->empty[c.stage]);
+    if (++c.stage == S) { c.stage = 0; c.parity ^= 1u; }
+    t_b = n_b;
+    t_r = n_r;
+  }
+  // per-row result: sum of the B columns in use, with the digit weights for integer inputs
+  float y0, y1;
+  if (WD == W_BF16) {
+    y0 = facc[0] + facc[1];
+    y1 = facc[2] + facc[3];
+  } else {
+    // columns 2q and 2q+1 of this lane: digit weights 16384 (col 0), 128 (col 1), 1 (col 2), 0 otherwise
+    const float w0 = (q == 0) ? 16384.f : (q == 1 ? 1.f : 0.f);
+    const float w1 = (q == 0) ? 128.f : 0.f;
+    if (WD == W_INT8) {
+      y0 = w0 * (float)iacc[0] + w1 * (float)iacc[1];
+      y1 = w0 * (float)iacc[2] + w1 * (float)iacc[3];
+    } else {
+      y0 = w0 * facc[0] + w1 * facc[1];
+      y1 = w0 * facc[2] + w1 * facc[3];
+    }
+  }
+  y0 += __shfl_xor_sync(0xffffffffu, y0, 1);
+  y0 += __shfl_xor_sync(0xffffffffu, y0, 2);
+  y1 += __shfl_xor_sync(0xffffffffu, y1, 1);
+  y1 += __shfl_xor_sync(0xffffffffu, y1, 2);
+  if (active && q == 0) {
+    float* dst = red + wk * g.R + wr * g.G;
+    if (gq < urows) dst[gq] = y0;
+    if (gq + 8 < urows) dst[gq + 8] = y1;
   }
 }
-
-__device__ __forceinline__ float4 ldcg4(const float* p, int i4) { return __ldcg(reinterpret_cast<const float4*>(p) + i4); }
-__device__ __forceinline__ float4 bf16x4_to_f32(uint2 v) {
-  return make_float4(bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y));
-}
-__device__ __forceinline__ float silu_f(float z) { return z / (1.0f + expf(-z)); }
+#undef AMK_LO
+#undef AMK_HI
 
 // ------------------------------------------------------------------------------------------------
 // One matrix-vector product with its fused prologue (gather / RMSNorm) and epilogue.
 // ------------------------------------------------------------------------------------------------
-__device__ __noinline__ bool gemv_op(Ctx& c, int op_idx, int wait_ph, int sig_ph) {
+__device__ __noinline__ bool gemv_op(Ctx& c, int kind, int l) {
   const KParams& p = c.p;
-  const OpDesc d = p.ops[op_idx];
-  const int slot = (c.cta + d.rot) % c.nblk;
+  const OpShape d = p.shape[kind];
+  const int op_idx = (kind == OP_LMHEAD) ? 4 * p.L : 4 * l + kind;
+  const int task = (kind == OP_LMHEAD) ? 5 * p.L : 5 * l + (kind == OP_QKV ? 0 : kind + 1);
+  const int slot = (c.cta + (op_idx * 37) % c.nblk) % c.nblk;
   const Slice sl = slot_slice(d.rows, d.unit_rows, c.nblk, slot);
-  const int l = d.layer, K = d.K, n4 = K >> 2;
+  const int K = d.K;
   const bool first_layer = (l == 0);
   const unsigned short* embed_row = p.embed + (size_t)c.token * p.H;
-
-  // input vector and norm weight of this op
-  const float* src = nullptr;
-  const unsigned short* normw = nullptr;
-  bool from_embed = false;
-  switch (d.kind) {
-    case OP_QKV: src = p.x_a; normw = p.attn_norm + (size_t)l * p.H; from_embed = first_layer; break;
-    case OP_O: src = p.o; break;
-    case OP_GATEUP: src = p.x_b; normw = p.mlp_norm + (size_t)l * p.H; break;
-    case OP_DOWN: src = p.m; break;
-    default: src = p.x_a; normw = p.final_norm; break;
-  }
-
-  const int task = (d.kind == OP_LMHEAD) ? 5 * p.L : 5 * l + (d.kind == OP_QKV ? 0 : d.kind + 1);
+  const unsigned my_seq = seq_of(p, task);
   if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_ENTER);
-  // ---- prologue, part 1: what does not depend on the join (norm weights) -----------------------------
-  uint2 gw[kNormVec];
-  if (normw) {
-#pragma unroll
-    for (int k = 0; k < kNormVec; k++) {
-      const int i = c.tid + k * kConsumerThreads;
-      gw[k] = (i < n4) ? __ldg(reinterpret_cast<const uint2*>(normw) + i) : make_uint2(0u, 0u);
-    }
-  }
-  // ---- the join ---------------------------------------------------------------------------------------
-  if (wait_ph >= 0 && !wait_phase(c, wait_ph)) return false;
-  if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_JOINED);
 
-  // ---- prologue, part 2: bring the input vector into shared memory ------------------------------------
-  float4* xs4 = reinterpret_cast<float4*>(c.xs);
-  if (normw) {
-    float4 v[kNormVec];
-    float ss = 0.f;
-#pragma unroll
-    for (int k = 0; k < kNormVec; k++) {
-      const int i = c.tid + k * kConsumerThreads;
-      if (i < n4) {
-        v[k] = from_embed ? bf16x4_to_f32(__ldg(reinterpret_cast<const uint2*>(embed_row) + i)) : ldcg4(src, i);
-        ss = fmaf(v[k].x, v[k].x, ss);
-        ss = fmaf(v[k].y, v[k].y, ss);
-        ss = fmaf(v[k].z, v[k].z, ss);
-        ss = fmaf(v[k].w, v[k].w, ss);
-      } else {
-        v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-      }
-    }
-    ss = warp_sum(ss);
-    if (c.lane == 0) c.sh->warp_part[c.warp] = ss;
-    c.bad = cons_sync_or(c.bad);
-    if (c.bad) return false;
-    float tot = 0.f;
-#pragma unroll
-    for (int w = 0; w < kConsumerWarps; w++) tot += c.sh->warp_part[w];
-    const float r = 1.0f / sqrtf(tot / (float)K + p.eps);
-#pragma unroll
-    for (int k = 0; k < kNormVec; k++) {
-      const int i = c.tid + k * kConsumerThreads;
-      if (i < n4) {
-        const float4 g = bf16x4_to_f32(gw[k]);
-        xs4[i] = make_float4(v[k].x * r * g.x, v[k].y * r * g.y, v[k].z * r * g.z, v[k].w * r * g.w);
-        if (from_embed && c.cta == 0 && (p.flags & AMK_FLAG_DEBUG_HIDDEN))
-          reinterpret_cast<float4*>(p.hidden)[i] = v[k];
-      }
-    }
-  } else {
-    for (int i = c.tid; i < n4; i += kConsumerThreads) xs4[i] = ldcg4(src, i);
+  // input vector, the task that wrote it, and the norm weight of this op
+  const ActPair* src = nullptr;
+  const unsigned short* normw = nullptr;
+  int src_task = -1;
+  bool from_embed = false;
+  switch (kind) {
+    case OP_QKV:
+      src = p.x_a; src_task = 5 * (l - 1) + 4; normw = p.attn_norm + (size_t)l * p.H; from_embed = first_layer;
+      break;
+    case OP_O: src = p.o; src_task = 5 * l + 1; break;
+    case OP_GATEUP: src = p.x_b; src_task = 5 * l + 2; normw = p.mlp_norm + (size_t)l * p.H; break;
+    case OP_DOWN: src = p.m; src_task = 5 * l + 3; break;
+    default: src = p.x_a; src_task = 5 * (p.L - 1) + 4; normw = p.final_norm; break;
   }
-  c.bad = cons_sync_or(c.bad);
-  if (c.bad) return false;
+  // geometry of the first pass while nothing else can be done
+  const int np = n_passes(sl.rows);
+  PassGeom g = pass_geom(np ? pass_rows(sl.rows, 0) : 1, K, d.wdtype, p.stage_bytes);
+
+  if (!from_embed && !wait_phase(c, src_task)) return false;
+  if (np > 0) {
+    if (!load_input(c, d.wdtype, K, src, from_embed ? 1u : seq_of(p, src_task), src_task,
+                    from_embed ? embed_row : nullptr, normw, task))
+      return false;
+  }
   if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_LOADED);
 
   // ---- passes -------------------------------------------------------------------------------------------
   float best_val = -CUDART_INF_F;
   int best_idx = 0x7fffffff;
-  const int np = n_passes(sl.rows);
+  const bool drop = (task == p.drop_phase && c.cta == p.drop_block);
   for (int ps = 0; ps < np; ps++) {
     const int R = pass_rows(sl.rows, ps);
-    const PassGeom g = pass_geom(R, K, d.wdtype, p.stage_bytes);
+    if (ps > 0) g = pass_geom(R, K, d.wdtype, p.stage_bytes);
     const int vrow0 = sl.row0 + ps * kPassRows;
     float* red = c.sh->red[ps & 1];
 
     // epilogue operands fetched ahead of the pass
-    const int n_out = (d.kind == OP_GATEUP) ? (R >> 1) : R;
+    const int n_out = (kind == OP_GATEUP) ? (R >> 1) : R;
     const bool outp = c.tid < n_out;
     float resid = 0.f, sc0 = 1.f, sc1 = 1.f;
     if (outp) {
       const int vrow = vrow0 + c.tid;
-      if (d.kind == OP_O)
-        resid = first_layer ? bf16_lo((unsigned)__ldg(embed_row + vrow)) : __ldcg(p.x_a + vrow);
-      else if (d.kind == OP_DOWN)
-        resid = __ldcg(p.x_b + vrow);
+      if (kind == OP_O) {
+        resid = first_layer ? bf16_lo((unsigned)__ldg(embed_row + vrow))
+                            : read_act(c, p.x_a + vrow, seq_of(p, 5 * (l - 1) + 4), 5 * (l - 1) + 4);
+      } else if (kind == OP_DOWN) {
+        resid = read_act(c, p.x_b + vrow, seq_of(p, 5 * l + 2), 5 * l + 2);
+      }
       if (d.wdtype == W_INT8) {
-        const __half* scales = reinterpret_cast<const __half*>(p.packed + d.scale_off);
-        if (d.kind == OP_GATEUP) {
+        const __half* scales = reinterpret_cast<const __half*>(
+            p.packed + p.scale_base + (size_t)l * p.scale_layer_stride + p.scale_kind_off[kind]);
+        if (kind == OP_GATEUP) {
           sc0 = __half2float(__ldg(scales + vrow0 + 2 * c.tid));
           sc1 = __half2float(__ldg(scales + vrow0 + 2 * c.tid + 1));
         } else {
           sc0 = __half2float(__ldg(scales + vrow));
         }
       }
+      if (d.wdtype != W_BF16) { sc0 *= c.xscale; sc1 *= c.xscale; }
     }
 
-    if (d.wdtype == W_BF16) consume_pass_g<W_BF16>(c, g, red);
-    else if (d.wdtype == W_INT8) consume_pass_g<W_INT8>(c, g, red);
-    else consume_pass_g<W_INT4>(c, g, red);
+    if (d.wdtype == W_BF16) consume_pass<W_BF16>(c, g, K, red);
+    else if (d.wdtype == W_INT8) consume_pass<W_INT8>(c, g, K, red);
+    else consume_pass<W_INT4>(c, g, K, red);
     c.bad = cons_sync_or(c.bad);
     if (c.bad) return false;
 
-    if (outp) {
+    if (outp && !drop) {
       const int vrow = vrow0 + c.tid;
-      if (d.kind == OP_GATEUP) {
+      if (kind == OP_GATEUP) {
         float gt = 0.f, up = 0.f;
         for (int k = 0; k < g.Wk; k++) {
           gt += red[k * R + 2 * c.tid];
@@ -388,17 +534,17 @@ __device__ __noinline__ bool gemv_op(Ctx& c, int op_idx, int wait_ph, int sig_ph
         }
         gt *= sc0;
         up *= sc1;
-        p.m[(vrow0 >> 1) + c.tid] = silu_f(gt) * up;
+        st_pair(p.m + (vrow0 >> 1) + c.tid, silu_f(gt) * up, my_seq);
       } else {
         float y = 0.f;
         for (int k = 0; k < g.Wk; k++) y += red[k * R + c.tid];
         y *= sc0;
-        switch (d.kind) {
-          case OP_QKV: p.qkv[vrow] = y; break;
-          case OP_O: p.x_b[vrow] = resid + y; break;
+        switch (kind) {
+          case OP_QKV: st_pair(p.qkv + vrow, y, my_seq); break;
+          case OP_O: st_pair(p.x_b + vrow, resid + y, my_seq); break;
           case OP_DOWN: {
             const float xn = resid + y;
-            p.x_a[vrow] = xn;
+            st_pair(p.x_a + vrow, xn, my_seq);
             if (p.flags & AMK_FLAG_DEBUG_HIDDEN) p.hidden[(size_t)(l + 1) * p.H + vrow] = xn;
             break;
           }
@@ -410,9 +556,9 @@ __device__ __noinline__ bool gemv_op(Ctx& c, int op_idx, int wait_ph, int sig_ph
       }
     }
   }
-
   if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_COMPUTED);
-  if (d.kind == OP_LMHEAD) {
+
+  if (kind == OP_LMHEAD) {
     // block argmax, then the block that arrives last reduces all blocks' candidates
     if (c.warp < kOutWarps) {
 #pragma unroll
@@ -460,16 +606,18 @@ __device__ __noinline__ bool gemv_op(Ctx& c, int op_idx, int wait_ph, int sig_ph
         if (c.lane == 0) {
           *p.next_ws = ix;
           if (p.next_token) *p.next_token = ix;
-          *p.lm_ctr = 0u;
+          *p.lm_ctr = 0u;                    // next used by the next launch
         }
       }
     }
     return true;
   }
 
-  c.bad = cons_sync_or(c.bad);
-  if (c.bad) return false;
-  if (sig_ph >= 0) signal_phase(c, sig_ph);
+  if (p.sync_mode == 0) {
+    c.bad = cons_sync_or(c.bad);
+    if (c.bad) return false;
+    signal_phase(c, task);
+  }
   if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_SIGNALLED);
   return true;
 }
@@ -490,35 +638,38 @@ __device__ __forceinline__ void attn_task(Ctx& c, int l, int g, int ch, int Lc, 
   const int n_pos = p.pos + 1;
   const int j0 = ch * Lc, j1 = min(n_pos, j0 + Lc);
   const bool owns_new = (j1 == n_pos);
-  float* qs = c.xs;                                   // [n_rep][HD]
-  float* wp = c.xs + n_rep * HD;                      // [warps][4][HD + 2]
+  float* qs = reinterpret_cast<float*>(c.xs);          // [n_rep][HD]
+  float* wp = qs + n_rep * HD;                         // [warps][4][HD + 2]
   const float2* rope = p.rope + (size_t)p.pos * half;
   const float qscale = 1.4426950408889634f * rsqrtf((float)HD);
   const size_t kvrow = ((size_t)l * p.nkv + g) * p.S;
+  const unsigned in_seq = seq_of(p, 5 * l), out_seq = seq_of(p, 5 * l + 1);
+  const bool drop = (5 * l + 1 == p.drop_phase && c.cta == p.drop_block);
 
   for (int i = c.tid; i < n_rep * half; i += kConsumerThreads) {
     const int h = i / half, e = i - h * half;
-    const float* q = p.qkv + (size_t)(g * n_rep + h) * HD;
-    const float a = __ldcg(q + e), b = __ldcg(q + e + half);
+    const ActPair* q = p.qkv + (size_t)(g * n_rep + h) * HD;
+    const float a = read_act(c, q + e, in_seq, 5 * l), b = read_act(c, q + e + half, in_seq, 5 * l);
     const float2 cs = __ldg(rope + e);
     qs[h * HD + e] = (a * cs.x - b * cs.y) * qscale;
     qs[h * HD + e + half] = (b * cs.x + a * cs.y) * qscale;
   }
   if (owns_new) {
     if (c.tid < half) {
-      const float* k = p.qkv + (size_t)p.nq * HD + (size_t)g * HD;
-      const float a = __ldcg(k + c.tid), b = __ldcg(k + c.tid + half);
+      const ActPair* k = p.qkv + (size_t)p.nq * HD + (size_t)g * HD;
+      const float a = read_act(c, k + c.tid, in_seq, 5 * l), b = read_act(c, k + c.tid + half, in_seq, 5 * l);
       const float2 cs = __ldg(rope + c.tid);
       unsigned short* dst = p.kcache + (kvrow + p.pos) * HD;
       dst[c.tid] = f32_to_bf16_rne(a * cs.x - b * cs.y);
       dst[c.tid + half] = f32_to_bf16_rne(b * cs.x + a * cs.y);
     } else if (c.tid >= 64 && c.tid < 64 + HD) {
       const int e = c.tid - 64;
-      const float* v = p.qkv + (size_t)(p.nq + p.nkv) * HD + (size_t)g * HD;
-      p.vcache[(kvrow + p.pos) * HD + e] = f32_to_bf16_rne(__ldcg(v + e));
+      const ActPair* v = p.qkv + (size_t)(p.nq + p.nkv) * HD + (size_t)g * HD;
+      p.vcache[(kvrow + p.pos) * HD + e] = f32_to_bf16_rne(read_act(c, v + e, in_seq, 5 * l));
     }
   }
   c.bad = cons_sync_or(c.bad);           // q in shared memory; the new cache row is visible to this block
+  if (c.tid == 0) stamp(p, c.cta, 5 * l + 1, AMK_TR_LOADED);
 
   const int n_hb = (n_rep + 3) >> 2;     // blocks of four q heads
   const int wph = kConsumerWarps / n_hb; // warps per head block
@@ -532,7 +683,7 @@ __device__ __forceinline__ void attn_task(Ctx& c, int l, int g, int ch, int Lc, 
 #pragma unroll
     for (int e = 0; e < 8; e++) acc[hh][e] = 0.f;
   }
-  if (hb < n_hb) {
+  if (hb < n_hb && !c.bad) {
     const uint4* Kb = reinterpret_cast<const uint4*>(p.kcache + kvrow * HD);
     const uint4* Vb = reinterpret_cast<const uint4*>(p.vcache + kvrow * HD);
     const int stride = wph * PPW;
@@ -610,6 +761,7 @@ __device__ __forceinline__ void attn_task(Ctx& c, int l, int g, int ch, int Lc, 
     }
   }
   c.bad = cons_sync_or(c.bad);
+  if (c.bad) return;
 
   // merge the warps of each head block, in warp order
   for (int i = c.tid; i < n_rep * HD; i += kConsumerThreads) {
@@ -626,7 +778,7 @@ __device__ __forceinline__ void attn_task(Ctx& c, int l, int g, int ch, int Lc, 
     }
     const int hq = g * n_rep + h;
     if (C == 1) {
-      p.o[(size_t)hq * HD + dd] = A / Z;
+      if (!drop) st_pair(p.o + (size_t)hq * HD + dd, A / Z, out_seq);
     } else {
       float* pt = p.part + ((size_t)hq * kMaxChunks + ch) * (HD + 2);
       pt[2 + dd] = A;
@@ -637,14 +789,15 @@ __device__ __forceinline__ void attn_task(Ctx& c, int l, int g, int ch, int Lc, 
 
   // several chunks: the chunk that arrives last for this kv group combines all of them
   c.bad = cons_sync_or(c.bad);
+  unsigned* gctr = p.group_ctr + (size_t)l * p.nkv + g;
   if (c.tid == 0) {
     __threadfence();
-    const unsigned old = atomicAdd(p.group_ctr + g, 1u);
+    const unsigned old = atomicAdd(gctr, 1u);
     __threadfence();
     c.sh->flag = (old == (unsigned)(C - 1));
   }
   c.bad = cons_sync_or(c.bad);
-  if (c.sh->flag) {
+  if (c.sh->flag && !c.bad) {
     for (int i = c.tid; i < n_rep * HD; i += kConsumerThreads) {
       const int h = i / HD, dd = i - h * HD;
       const int hq = g * n_rep + h;
@@ -657,9 +810,9 @@ __device__ __forceinline__ void attn_task(Ctx& c, int l, int g, int ch, int Lc, 
         Z = fmaf(a, __ldcg(pt + (size_t)k * (HD + 2) + 1), Z);
         A = fmaf(a, __ldcg(pt + (size_t)k * (HD + 2) + 2 + dd), A);
       }
-      p.o[(size_t)hq * HD + dd] = A / Z;
+      if (!drop) st_pair(p.o + (size_t)hq * HD + dd, A / Z, out_seq);
     }
-    if (c.tid == 0) p.group_ctr[g] = 0u;
+    if (c.tid == 0) *gctr = 0u;          // next used by the next launch
   }
 }
 
@@ -670,9 +823,11 @@ __device__ __noinline__ bool attention_phase(Ctx& c, int l) {
   const int n_tasks = p.nkv * C;
   const int rot = (l * 29) % c.nblk;
   const int t = (c.cta + c.nblk - rot) % c.nblk;
-  if (c.tid == 0) stamp(p, c.cta, 5 * l + 1, AMK_TR_ENTER);
+  const int task = 5 * l + 1;
+  if (p.sync_mode != 0 && t >= n_tasks) return true;      // nothing to do here and nobody to tell
+  if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_ENTER);
   if (!wait_phase(c, 5 * l + 0)) return false;
-  if (c.tid == 0) stamp(p, c.cta, 5 * l + 1, AMK_TR_JOINED);
+  if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_JOINED);
   if (t < n_tasks) {
     const int g = t / C, ch = t - g * C;
     if (p.hd == 64) attn_task<64>(c, l, g, ch, Lc, C);
@@ -680,59 +835,63 @@ __device__ __noinline__ bool attention_phase(Ctx& c, int l) {
   }
   c.bad = cons_sync_or(c.bad);
   if (c.bad) return false;
-  if (c.tid == 0) stamp(p, c.cta, 5 * l + 1, AMK_TR_COMPUTED);
-  signal_phase(c, 5 * l + 1);
-  if (c.tid == 0) stamp(p, c.cta, 5 * l + 1, AMK_TR_SIGNALLED);
+  if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_COMPUTED);
+  signal_phase(c, task);
+  if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_SIGNALLED);
   return true;
 }
 
 // ------------------------------------------------------------------------------------------------
-// Producer: one thread streams this block's weight tiles, op after op, into the ring.
+// Producer: streams this block's weight tiles, in order, into the ring.  The tile list {offset, bytes,
+// task} was laid out by the host, so the producer only waits for a free stage and issues the copy.
 // ------------------------------------------------------------------------------------------------
-__device__ __noinline__ void producer(const KParams& p, SmemHeader* sh, unsigned char* ring, int cta, int nblk) {
+__device__ __noinline__ void producer(const KParams& p, SmemHeader* sh, unsigned char* ring, int cta, int lane) {
   const uint64_t pol = policy_evict_first();
-  const int S = p.n_stages;
-  const int inflight = p.max_inflight;
-  unsigned t = 0;
-  bool ok = true;
-  for (int op = 0; op < p.n_ops && ok; op++) {
-    const OpDesc d = p.ops[op];
-    const int slot = (cta + d.rot) % nblk;
-    const Slice sl = slot_slice(d.rows, d.unit_rows, nblk, slot);
-    const int64_t rb = row_bytes(d.wdtype, d.K);
-    const unsigned char* base = p.packed + d.packed_off + (int64_t)sl.row0 * rb;
-    const int np = n_passes(sl.rows);
-    const int task = (d.kind == OP_LMHEAD) ? 5 * p.L : 5 * d.layer + (d.kind == OP_QKV ? 0 : d.kind + 1);
-    bool first = true;
-    for (int ps = 0; ps < np && ok; ps++) {
-      const PassGeom g = pass_geom(pass_rows(sl.rows, ps), d.K, d.wdtype, p.stage_bytes);
-      const unsigned char* pbase = base + (int64_t)ps * kPassRows * rb;
-      for (int tt = 0; tt < g.n_tiles; tt++, t++) {
-        const int u0 = tt * g.upt;
-        const int64_t o0 = unit_off(g, u0), o1 = unit_off(g, u0 + g.upt);
-        const int stage = (int)(t % (unsigned)S);
-        if (t >= (unsigned)S) {
-          if (!wait_mbar(p, &sh->empty[stage], ((t / (unsigned)S) & 1u) ^ 1u, -2)) { ok = false; break; }
+  const unsigned S = (unsigned)p.n_stages;
+  const unsigned inflight = (unsigned)p.max_inflight;
+  const unsigned begin = __ldg(p.tile_begin + cta), end = __ldg(p.tile_begin + cta + 1);
+  unsigned t = 0;                                   // tiles issued so far
+  unsigned stage = 0, lap = 0;
+  int cur_task = -1;
+  int ok = 1;
+  unsigned long long e_next = (begin + lane < end) ? __ldg(p.tiles + begin + lane) : 0ull;
+  for (unsigned base = begin; base < end && ok; base += 32) {
+    const unsigned long long e_cur = e_next;
+    if (base + 32 + lane < end) e_next = __ldg(p.tiles + base + 32 + lane);
+    const int n = (int)min(32u, end - base);
+    for (int j = 0; j < n; j++) {
+      const unsigned long long e = __shfl_sync(0xffffffffu, e_cur, j);
+      if (lane == 0) {
+        const unsigned long long off = (e & ((1ull << 40) - 1)) << 4;
+        const unsigned bytes = (unsigned)((e >> 40) & 0x1fffu) << 4;
+        const int task = (int)(e >> 53);
+        if (lap > 0 && !wait_mbar(p, &sh->empty[stage], (lap - 1) & 1u, -2)) ok = 0;
+        if (ok && inflight < S && t >= inflight) {
+          const unsigned tl = t - inflight;          // this older tile must have landed
+          if (!wait_mbar(p, &sh->full[tl % S], (tl / S) & 1u, -2)) ok = 0;
         }
-        if (inflight < S && t >= (unsigned)inflight) {
-          const unsigned tl = t - (unsigned)inflight;      // this older tile must have landed
-          if (!wait_mbar(p, &sh->full[tl % (unsigned)S], (tl / (unsigned)S) & 1u, -2)) { ok = false; break; }
+        if (ok) {
+          mbar_expect_tx(&sh->full[stage], bytes);
+          bulk_g2s(ring + (size_t)stage * p.stage_bytes, p.packed + off, bytes, &sh->full[stage], pol);
+          if (p.trace) {
+            if (task != cur_task) { stamp(p, cta, task, AMK_TR_PROD_FIRST); cur_task = task; }
+            stamp(p, cta, task, AMK_TR_PROD_LAST);
+          }
+          t++;
+          if (++stage == S) { stage = 0; lap++; }
         }
-        const unsigned bytes = (unsigned)(o1 - o0);
-        mbar_expect_tx(&sh->full[stage], bytes);
-        bulk_g2s(ring + (size_t)stage * p.stage_bytes, pbase + o0, bytes, &sh->full[stage], pol);
-        if (first) { stamp(p, cta, task, AMK_TR_PROD_FIRST); first = false; }
       }
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
     }
-    if (ok) stamp(p, cta, task, AMK_TR_PROD_LAST);
   }
-  if (!ok) {
+  if (!ok && lane == 0) {
     // leaving early: every copy already issued must land before the block's shared memory is released
-    const unsigned first = (t > (unsigned)S) ? t - (unsigned)S : 0u;
+    const unsigned first = (t > S) ? t - S : 0u;
     for (unsigned i = first; i < t; i++) {
-      uint64_t* bar = &sh->full[i % (unsigned)S];
-      const unsigned parity = (i / (unsigned)S) & 1u;
-      for (unsigned spins = 0; spins < (1u << 24) && !mbar_try_wait(bar, parity); spins++) {}
+      uint64_t* bar = &sh->full[i % S];
+      const unsigned par = (i / S) & 1u;
+      for (unsigned spins = 0; spins < (1u << 24) && !mbar_try_wait(bar, par); spins++) {}
     }
   }
 }
@@ -743,7 +902,7 @@ __global__ void __launch_bounds__(kThreads, 1) amk_decode_kernel(const __grid_co
   extern __shared__ __align__(128) unsigned char smem[];
   SmemHeader* sh = reinterpret_cast<SmemHeader*>(smem);
   const size_t hdr = (sizeof(SmemHeader) + 127) & ~(size_t)127;
-  float* xs = reinterpret_cast<float*>(smem + hdr);
+  unsigned char* xs = smem + hdr;
   unsigned char* ring = smem + hdr + p.act_bytes;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int cta = blockIdx.x, nblk = gridDim.x;
@@ -753,29 +912,28 @@ __global__ void __launch_bounds__(kThreads, 1) amk_decode_kernel(const __grid_co
       mbar_init(&sh->full[s], 1);
       mbar_init(&sh->empty[s], kConsumerWarps);
     }
-    sh->abort = 0;
     sh->flag = 0;
     mbar_fence_init();
   }
   __syncthreads();
 
   if (warp == kConsumerWarps) {
-    if (lane == 0) producer(p, sh, ring, cta, nblk);
+    producer(p, sh, ring, cta, lane);
     return;
   }
 
   int token = p.token_ptr ? __ldcg(p.token_ptr) : p.token;
   token = min(max(token, 0), p.V - 1);
-  Ctx c{p, sh, xs, ring, tid, warp, lane, cta, nblk, 0u, token, false};
+  Ctx c{p, sh, xs, ring, tid, warp, lane, cta, nblk, 0, 0u, token, 1.0f, false};
   bool ok = true;
   for (int l = 0; l < p.L && ok; l++) {
-    ok = gemv_op(c, 4 * l + 0, l > 0 ? 5 * (l - 1) + 4 : -1, 5 * l + 0);
+    ok = gemv_op(c, OP_QKV, l);
     ok = ok && attention_phase(c, l);
-    ok = ok && gemv_op(c, 4 * l + 1, 5 * l + 1, 5 * l + 2);
-    ok = ok && gemv_op(c, 4 * l + 2, 5 * l + 2, 5 * l + 3);
-    ok = ok && gemv_op(c, 4 * l + 3, 5 * l + 3, 5 * l + 4);
+    ok = ok && gemv_op(c, OP_O, l);
+    ok = ok && gemv_op(c, OP_GATEUP, l);
+    ok = ok && gemv_op(c, OP_DOWN, l);
   }
-  if (ok) gemv_op(c, 4 * p.L, 5 * (p.L - 1) + 4, -1);
+  if (ok) gemv_op(c, OP_LMHEAD, p.L);
 }
 
 cudaError_t decode_kernel_attrs(size_t smem_bytes, int* max_blocks_per_sm) {

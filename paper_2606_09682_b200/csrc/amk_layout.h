@@ -3,20 +3,19 @@
 // A matrix-vector product y = W x (W: [rows][K]) is split by rows across the persistent blocks; block
 // `slot` owns a contiguous run of "units" (1 row, or 2 rows where rows must stay together).  Inside a
 // block the rows are processed in passes of at most kPassRows rows.  In a pass the consumer warps form
-// a W_r x W_k grid: row-warp wr owns G consecutive rows, k-warp wk owns every W_k-th 256-column block.
-// The bytes of a pass are stored block-major: for column block b, rows 0..R-1, each row's 256 columns
-// (the last block may be narrower).  A "work unit" (b, wr) -- G rows of one column block -- is therefore
-// contiguous, and a ring tile is a run of consecutive work units, so each block's whole weight stream is
-// one contiguous byte range that a single producer thread can fetch with bulk copies, never waiting on
-// a data dependency.
+// a Wr x Wk grid: row-warp wr owns G <= 16 consecutive rows (one m16 tensor-core tile), k-warp wk owns
+// every Wk-th column block (64 columns; 128 for int4 = one quantisation group).  The bytes of a pass are
+// stored block-major: for column block b, the work units (b, wr = 0..Wr-1) one after another.  A work
+// unit -- the rows of one row-warp in one column block -- is contiguous, and a ring tile is a run of
+// `upt` consecutive units, so each block's weight stream is a sequence of contiguous byte runs that one
+// producer thread fetches with bulk copies, never waiting on a data dependency.
 //
-// Column order inside a 256-column block of width Wd: lane l (< Wd/8) holds columns
-// {4l..4l+3} and {Wd/2 + 4l .. Wd/2 + 4l + 3}, so its activation reads are two conflict-free 16-byte
-// shared-memory loads and, for int4 (Wd = 256, groups of 128), its first four codes belong to group 2b
-// and its last four to group 2b+1.
-//
-// Bytes per row per full column block: bf16 512, int8 256, int4 128 + 8 (fp16 scale and zero point of
-// its two groups follow the 128 code bytes of the same row).
+// Inside a unit the bytes are ordered for ldmatrix: 16-byte chunk c (8 bf16 / 16 int8 / 32 int4 codes
+// along K) of row r sits at (c * rows + r) * 16, so the eight rows of an 8x8 matrix are 128 contiguous
+// bytes (no bank conflicts).  The k order inside a block is permuted (col_of_k) so that the activation
+// values one lane feeds to the tensor core -- its B fragments for every k step of the block -- are
+// contiguous in the natural column order.  An int4 unit ends with fp16 {scale, zero} per row (its block
+// is one group).
 #pragma once
 #include <stdint.h>
 
@@ -31,9 +30,8 @@ namespace amk {
 constexpr int kConsumerWarps = 15;            // consumer warps per block (+1 producer warp = 512 threads)
 constexpr int kThreads = 32 * (kConsumerWarps + 1);
 constexpr int kConsumerThreads = 32 * kConsumerWarps;
-constexpr int kGMax = 8;                      // rows per row-warp
+constexpr int kGMax = 16;                     // rows per row-warp: one m16n8 tile
 constexpr int kPassRows = kConsumerWarps * kGMax;
-constexpr int kBlockCols = 256;               // columns per column block
 constexpr int kMaxStages = 16;
 constexpr int kMaxRep = 16;                   // q heads per kv head
 constexpr int kAttnMinChunk = 32;             // fewest cache positions per split-K chunk
@@ -42,29 +40,43 @@ constexpr int kMaxChunks = 64;
 enum OpKind : int { OP_QKV = 0, OP_O = 1, OP_GATEUP = 2, OP_DOWN = 3, OP_LMHEAD = 4 };
 enum WDtype : int { W_BF16 = 0, W_INT8 = 1, W_INT4 = 2 };
 
-// One matrix-vector product of the step.  Lives in device memory (table built by amk_create).
-struct OpDesc {
-  int32_t kind;          // OpKind
-  int32_t layer;
-  int32_t K;             // input length
-  int32_t rows;          // output rows (virtual rows: QKV = q|k|v rows, GATEUP = g0,u0,g1,u1,...)
-  int32_t unit_rows;     // rows per ownership unit (1, or 2)
-  int32_t wdtype;        // WDtype of this op (LM head is always bf16)
-  int32_t rot;           // slot rotation: block c takes slot (c + rot) % n_blocks
-  int32_t pad;
-  uint64_t packed_off;   // byte offset of this op's region in the packed buffer
-  uint64_t scale_off;    // int8: byte offset of the fp16 row scales (virtual row order); else 0
-};
-
 AMK_HD int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
-// bytes of one row inside a column block of width wd
-AMK_HD int rowchunk_bytes(int wdtype, int wd) {
-  return wdtype == W_BF16 ? wd * 2 : (wdtype == W_INT8 ? wd : (wd / 2 + 8 * (wd / kBlockCols)));
+AMK_HD int block_cols(int wdtype) { return wdtype == W_INT4 ? 128 : 64; }        // columns per column block
+AMK_HD int block_chunks(int wdtype) { return wdtype == W_BF16 ? 8 : 4; }          // 16-byte chunks per row per block
+// bytes of a work unit holding `rows` rows (int4: codes, then 4 bytes {scale, zero} per row, padded to 16)
+AMK_HD int unit_bytes(int wdtype, int rows) {
+  if (wdtype == W_BF16) return rows * 128;
+  if (wdtype == W_INT8) return rows * 64;
+  return (rows * 68 + 15) & ~15;
 }
-AMK_HD int64_t row_bytes(int wdtype, int K) {
-  int nbf = K / kBlockCols, tail = K % kBlockCols;
-  return (int64_t)nbf * rowchunk_bytes(wdtype, kBlockCols) + (tail ? rowchunk_bytes(wdtype, tail) : 0);
+
+// Logical k index inside a block (what the tensor-core fragments see) -> natural column inside the block.
+// Lane-quad q of a warp supplies, for k step s (bf16 k16, int8 k32, int4: k32 after nibble expansion) and
+// fragment half h, the values j; its whole supply for a block is the contiguous column run starting at
+// q * (block_cols / 4).
+//   bf16: k = 16 s + 8 h + 2 q + j  (s<4, h<2, q<4, j<2)  ->  col 16 q + 4 s + 2 h + j
+//   int8: k = 32 s + 16 h + 4 q + j (s<2, h<2, q<4, j<4)  ->  col 16 q + 8 s + 4 h + j
+//   int4: k = 32 s + 16 h + 4 q + j (s<4, h<2, q<4, j<4)  ->  col 32 q + 8 s + 4 h + j
+AMK_HD int col_of_k(int wdtype, int k) {
+  if (wdtype == W_BF16) {
+    const int s = k >> 4, h = (k >> 3) & 1, q = (k >> 1) & 3, j = k & 1;
+    return 16 * q + 4 * s + 2 * h + j;
+  }
+  const int s = k >> 5, h = (k >> 4) & 1, q = (k >> 2) & 3, j = k & 3;
+  return (wdtype == W_INT8 ? 16 : 32) * q + 8 * s + 4 * h + j;
+}
+
+// Where logical k of a row is stored inside its unit: the 16-byte chunk, and the element inside the chunk
+// (bf16: 2-byte element; int8: byte; int4: nibble, low nibble of a byte first).
+//   bf16 / int8: k-major.   int4: one ldmatrix word (8 nibbles) of chunk 2 (s >> 1) + h expands into the
+//   fragment registers of k steps s = 2x (even nibbles) and s = 2x + 1 (odd nibbles).
+AMK_HD void place_of_k(int wdtype, int k, int* chunk, int* elem) {
+  if (wdtype == W_BF16) { *chunk = k >> 3; *elem = k & 7; return; }
+  if (wdtype == W_INT8) { *chunk = k >> 4; *elem = k & 15; return; }
+  const int s = k >> 5, h = (k >> 4) & 1, q = (k >> 2) & 3, j = k & 3;
+  *chunk = 2 * (s >> 1) + h;
+  *elem = 8 * q + 2 * j + (s & 1);
 }
 
 // Rows owned by slot s: units are dealt as evenly as possible, the first (units % n) slots get one more.
@@ -90,70 +102,64 @@ AMK_HD int slot_of_row(int total_rows, int unit_rows, int n_slots, int row) {
 // Geometry of one pass of R rows over K columns.
 struct PassGeom {
   int R;        // rows in the pass
-  int G;        // rows per row-warp (the last row-warp may have fewer)
+  int G;        // rows per row-warp (the last row-warp has g_last)
+  int g_last;
   int Wr;       // row-warps
   int Wk;       // k-warps
-  int nblk;     // column blocks (the last may be narrower)
-  int tail;     // width of the last block if narrower than 256, else 0
-  int n_units;  // Wr * nblk work units
+  int nblk;     // column blocks
+  int n_units;  // Wr * nblk work units, ordered (b, wr)
   int upt;      // work units per ring tile
   int n_tiles;
-  int rc_full;  // bytes of one row in a full block
-  int rc_tail;  // bytes of one row in the tail block
+  int ub_full;  // bytes of a unit of G rows
+  int ub_last;  // bytes of the last row-warp's unit
+  int bb;       // bytes of one column block = (Wr - 1) * ub_full + ub_last
 };
 
 AMK_HD PassGeom pass_geom(int R, int K, int wdtype, int stage_bytes) {
   PassGeom g;
   g.R = R;
-  const int galign = (wdtype == W_INT4) ? 2 : 1;     // int4 row chunks are 136 B: keep unit offsets 16-byte aligned
   // fewest row-warps that keep G <= kGMax; if at most half the warps are needed, several k-warps share a
   // row group and the row-warps are spread over what the k split leaves; otherwise every warp is a row-warp.
   const int wr_min = ceil_div(R, kGMax);
   int wr;
   if (2 * wr_min > kConsumerWarps) wr = kConsumerWarps;
   else wr = kConsumerWarps / (kConsumerWarps / wr_min);
-  int G = ceil_div(R, wr);
-  G = ceil_div(G, galign) * galign;
-  if (G > kGMax) G = kGMax;
+  const int G = ceil_div(R, wr);
   g.G = G;
   g.Wr = ceil_div(R, G);
+  g.g_last = R - (g.Wr - 1) * G;
   g.Wk = kConsumerWarps / g.Wr;
-  g.nblk = ceil_div(K, kBlockCols);
-  g.tail = K % kBlockCols;
+  g.nblk = K / block_cols(wdtype);
   if (g.Wk > g.nblk) g.Wk = g.nblk;
   g.n_units = g.Wr * g.nblk;
-  g.rc_full = rowchunk_bytes(wdtype, kBlockCols);
-  g.rc_tail = g.tail ? rowchunk_bytes(wdtype, g.tail) : g.rc_full;
-  int ub = G * g.rc_full;
-  g.upt = stage_bytes / ub;
+  g.ub_full = unit_bytes(wdtype, G);
+  g.ub_last = unit_bytes(wdtype, g.g_last);
+  g.bb = (g.Wr - 1) * g.ub_full + g.ub_last;
+  g.upt = stage_bytes / g.ub_full;
   if (g.upt < 1) g.upt = 1;
   g.n_tiles = ceil_div(g.n_units, g.upt);
   return g;
 }
 
 // Byte offset of work unit (column block b, row-warp r) from the start of the pass.
-AMK_HD int64_t unit_off_br(const PassGeom& g, int b, int r) {
-  int rc = (g.tail && b == g.nblk - 1) ? g.rc_tail : g.rc_full;
-  return (int64_t)b * g.R * g.rc_full + (int64_t)r * g.G * rc;   // every block before b is full
-}
-// Total bytes of the pass.
-AMK_HD int64_t pass_bytes(const PassGeom& g) {
-  int nbf = g.nblk - (g.tail ? 1 : 0);
-  return (int64_t)nbf * g.R * g.rc_full + (g.tail ? (int64_t)g.R * g.rc_tail : 0);
-}
-// Byte offset of work unit u (= b * Wr + r); u == n_units gives the pass size.
+AMK_HD int64_t unit_off_br(const PassGeom& g, int b, int r) { return (int64_t)b * g.bb + (int64_t)r * g.ub_full; }
+AMK_HD int64_t pass_bytes(const PassGeom& g) { return (int64_t)g.nblk * g.bb; }
+// Byte offset of work unit u (= b * Wr + r); u >= n_units gives the pass size.
 AMK_HD int64_t unit_off(const PassGeom& g, int u) {
   if (u >= g.n_units) return pass_bytes(g);
   int b = u / g.Wr;
   return unit_off_br(g, b, u - b * g.Wr);
 }
 
-// Number of passes for a slice of `rows` rows and the rows of pass p.
 AMK_HD int n_passes(int rows) { return ceil_div(rows, kPassRows); }
 AMK_HD int pass_rows(int rows, int p) { int left = rows - p * kPassRows; return left < kPassRows ? left : kPassRows; }
 
-// Column held at element e (0..7) of lane l in a block of width wd.
-AMK_HD int lane_col(int wd, int lane, int e) { return (e < 4) ? 4 * lane + e : wd / 2 + 4 * lane + (e - 4); }
+// Packed bytes of a slice of `rows` rows.
+AMK_HD int64_t slice_bytes(int rows, int K, int wdtype, int stage_bytes) {
+  int64_t t = 0;
+  for (int p = 0; p < n_passes(rows); p++) t += pass_bytes(pass_geom(pass_rows(rows, p), K, wdtype, stage_bytes));
+  return t;
+}
 
 // Split-K plan of the attention over positions [0, n_pos): chunk length and count.
 AMK_HD void attn_chunks(int n_pos, int n_blocks, int n_kv, int* chunk_len, int* n_chunks) {
@@ -165,5 +171,10 @@ AMK_HD void attn_chunks(int n_pos, int n_blocks, int n_kv, int* chunk_len, int* 
   *chunk_len = lc;
   *n_chunks = ceil_div(n_pos, lc);
 }
+
+// One matrix-vector product kind of a model (the same for every layer).
+struct OpShape {
+  int32_t K, rows, unit_rows, wdtype;
+};
 
 }  // namespace amk

@@ -11,13 +11,13 @@ namespace amk {
 namespace {
 
 struct RowSrc {
-  const unsigned char* w;       // row start in the canonical matrix
-  const unsigned short* scale;  // int8: &scale[row]; int4: &scale[row][0]
-  const unsigned short* zero;   // int4: &zero[row][0]
+  unsigned char* w;             // row start in the canonical matrix (nullptr: this row is not wanted)
+  unsigned short* scale;        // int8: &scale[row]; int4: &scale[row][0]
+  unsigned short* zero;         // int4: &zero[row][0]
 };
 
 // Canonical location of virtual row `vrow` of an op.
-__device__ __forceinline__ RowSrc row_source(const OpDesc& d, const PackSrc& s, int vrow) {
+__device__ __forceinline__ RowSrc row_source(const OpShape& d, const PackSrc& s, int vrow) {
   int which = 0, row = vrow;
   if (s.mode == 1) {
     if (vrow >= s.rows1) { which = 2; row = vrow - s.rows1; }
@@ -29,79 +29,104 @@ __device__ __forceinline__ RowSrc row_source(const OpDesc& d, const PackSrc& s, 
   const size_t K = (size_t)d.K;
   const size_t rowb = d.wdtype == W_BF16 ? K * 2 : (d.wdtype == W_INT8 ? K : K / 2);
   RowSrc r;
-  r.w = s.w[which] ? reinterpret_cast<const unsigned char*>(s.w[which]) + (size_t)row * rowb : nullptr;
+  r.w = s.w[which] ? (unsigned char*)s.w[which] + (size_t)row * rowb : nullptr;
   r.scale = nullptr;
   r.zero = nullptr;
-  if (d.wdtype == W_INT8 && s.scale[which]) r.scale = reinterpret_cast<const unsigned short*>(s.scale[which]) + row;
+  if (d.wdtype == W_INT8 && s.scale[which]) r.scale = (unsigned short*)s.scale[which] + row;
   if (d.wdtype == W_INT4) {
-    if (s.scale[which]) r.scale = reinterpret_cast<const unsigned short*>(s.scale[which]) + (size_t)row * (K / 128);
-    if (s.zero[which]) r.zero = reinterpret_cast<const unsigned short*>(s.zero[which]) + (size_t)row * (K / 128);
+    if (s.scale[which]) r.scale = (unsigned short*)s.scale[which] + (size_t)row * (K / 128);
+    if (s.zero[which]) r.zero = (unsigned short*)s.zero[which] + (size_t)row * (K / 128);
   }
   return r;
 }
 
-// grid.x = virtual rows; threads loop over (column block, lane) chunks of 8 elements.
-// inverse = false: canonical -> packed;  true: packed -> canonical (s.* then point at writable outputs).
-__global__ void pack_kernel(const OpDesc d, const PackSrc s, unsigned char* packed, int n_blocks, int stage_bytes,
+// grid.x = virtual rows; threads loop over the 16-byte chunks of the row.
+// inverse = 0: canonical -> packed;  1: packed -> canonical (s.* then point at writable outputs).
+__global__ void pack_kernel(const PackOp d, const PackSrc s, unsigned char* packed, int n_blocks, int stage_bytes,
                             int inverse) {
   const int vrow = blockIdx.x;
-  const int slot = slot_of_row(d.rows, d.unit_rows, n_blocks, vrow);
-  const Slice sl = slot_slice(d.rows, d.unit_rows, n_blocks, slot);
+  const int wd = d.s.wdtype, K = d.s.K;
+  const int slot = slot_of_row(d.s.rows, d.s.unit_rows, n_blocks, vrow);
+  const Slice sl = slot_slice(d.s.rows, d.s.unit_rows, n_blocks, slot);
   const int local = vrow - sl.row0;
   const int ps = local / kPassRows, rp = local - ps * kPassRows;
-  const PassGeom g = pass_geom(pass_rows(sl.rows, ps), d.K, d.wdtype, stage_bytes);
+  int64_t pass_off = 0;
+  for (int p = 0; p < ps; p++) pass_off += pass_bytes(pass_geom(pass_rows(sl.rows, p), K, wd, stage_bytes));
+  const PassGeom g = pass_geom(pass_rows(sl.rows, ps), K, wd, stage_bytes);
   const int wr = rp / g.G, gi = rp - wr * g.G;
-  const int64_t rb = row_bytes(d.wdtype, d.K);
-  unsigned char* pass_base = packed + d.packed_off + (int64_t)sl.row0 * rb + (int64_t)ps * kPassRows * rb;
-  const RowSrc src = row_source(d, s, vrow);
+  const int urows = (wr == g.Wr - 1) ? g.g_last : g.G;
+  unsigned char* pass_base = packed + d.region_off + d.slice_off[slot] + pass_off;
+  const RowSrc src = row_source(d.s, s, vrow);
   if (src.w == nullptr) return;                 // (unpacking one matrix of a stacked op: not this row)
 
-  if (d.wdtype == W_INT8 && threadIdx.x == 0 && src.scale) {
-    // row scales live in a separate region in virtual-row order
+  if (wd == W_INT8 && threadIdx.x == 0 && src.scale) {
     unsigned short* dst = reinterpret_cast<unsigned short*>(packed + d.scale_off) + vrow;
     if (!inverse) *dst = *src.scale;
-    else *const_cast<unsigned short*>(src.scale) = *dst;
+    else *src.scale = *dst;
   }
-
-  for (int ci = threadIdx.x; ci < g.nblk * 32; ci += blockDim.x) {
-    const int b = ci >> 5, lane = ci & 31;
-    const bool is_tail = g.tail && (b == g.nblk - 1);
-    const int wd = is_tail ? g.tail : kBlockCols;
-    const int rc = is_tail ? g.rc_tail : g.rc_full;
-    unsigned char* chunk = pass_base + unit_off_br(g, b, wr) + (int64_t)gi * rc;
-    if (lane >= (wd >> 3)) continue;
-    const int c0 = b * kBlockCols + 4 * lane, c1 = b * kBlockCols + (wd >> 1) + 4 * lane;
-    if (d.wdtype == W_BF16) {
-      uint2* a0 = (uint2*)(src.w + (size_t)c0 * 2);
-      uint2* a1 = (uint2*)(src.w + (size_t)c1 * 2);
-      uint4* dst = (uint4*)(chunk + lane * 16);
-      if (!inverse) { const uint2 v0 = *a0, v1 = *a1; *dst = make_uint4(v0.x, v0.y, v1.x, v1.y); }
-      else { const uint4 v = *dst; *a0 = make_uint2(v.x, v.y); *a1 = make_uint2(v.z, v.w); }
-    } else if (d.wdtype == W_INT8) {
-      unsigned* a0 = (unsigned*)(src.w + c0);
-      unsigned* a1 = (unsigned*)(src.w + c1);
-      uint2* dst = (uint2*)(chunk + lane * 8);
-      if (!inverse) *dst = make_uint2(*a0 ^ 0x80808080u, *a1 ^ 0x80808080u);      // two's complement -> biased
-      else { const uint2 v = *dst; *a0 = v.x ^ 0x80808080u; *a1 = v.y ^ 0x80808080u; }
+  const int cpb = block_chunks(wd), bc = block_cols(wd);
+  for (int ci = threadIdx.x; ci < g.nblk * cpb; ci += blockDim.x) {
+    const int b = ci / cpb, c = ci - b * cpb;
+    unsigned char* unit = pass_base + unit_off_br(g, b, wr);
+    uint4* chunk = reinterpret_cast<uint4*>(unit + ((size_t)c * urows + gi) * 16);
+    const int col0 = b * bc;
+    if (wd == W_BF16) {
+      // chunk c = 2 s + hh holds logical k = 16 s + 8 hh + 2 q + j: for q = 0..3 the pair at column 16 q + 4 s + 2 hh
+      const int sidx = c >> 1, hh = c & 1;
+      unsigned* w32 = reinterpret_cast<unsigned*>(src.w);
+      unsigned v[4];
+      if (inverse) { const uint4 t = *chunk; v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w; }
+      for (int q = 0; q < 4; q++) {
+        const int col = col0 + 16 * q + 4 * sidx + 2 * hh;
+        if (!inverse) v[q] = w32[col >> 1];
+        else w32[col >> 1] = v[q];
+      }
+      if (!inverse) *chunk = make_uint4(v[0], v[1], v[2], v[3]);
+    } else if (wd == W_INT8) {
+      // chunk c = 2 s + hh holds logical k = 32 s + 16 hh + 4 q + j: for q = 0..3 the word at column 16 q + 8 s + 4 hh
+      const int sidx = c >> 1, hh = c & 1;
+      unsigned* w32 = reinterpret_cast<unsigned*>(src.w);
+      unsigned v[4];
+      if (inverse) { const uint4 t = *chunk; v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w; }
+      for (int q = 0; q < 4; q++) {
+        const int col = col0 + 16 * q + 8 * sidx + 4 * hh;
+        if (!inverse) v[q] = w32[col >> 2];
+        else w32[col >> 2] = v[q];
+      }
+      if (!inverse) *chunk = make_uint4(v[0], v[1], v[2], v[3]);
     } else {
-      unsigned short* a0 = (unsigned short*)(src.w + (c0 >> 1));
-      unsigned short* a1 = (unsigned short*)(src.w + (c1 >> 1));
-      unsigned* dst = (unsigned*)(chunk + lane * 4);
-      if (!inverse) *dst = (unsigned)*a0 | ((unsigned)*a1 << 16);
-      else { const unsigned v = *dst; *a0 = (unsigned short)(v & 0xffffu); *a1 = (unsigned short)(v >> 16); }
-      if (lane == 0) {
-        // fp16 {scale, zero} of groups 2b and 2b+1 follow the 128 code bytes of this row chunk
-        uint2* sz = (uint2*)(chunk + 128);
-        unsigned short* sc = const_cast<unsigned short*>(src.scale);
-        unsigned short* zr = const_cast<unsigned short*>(src.zero);
+      // chunk c = 2 x + hh; word q, nibble 2 j + sb holds logical k of step s = 2 x + sb: column 32 q + 8 s + 4 hh + j
+      const int x = c >> 1, hh = c & 1;
+      unsigned v[4];
+      if (inverse) { const uint4 t = *chunk; v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w; }
+      for (int q = 0; q < 4; q++) {
+        unsigned word = inverse ? v[q] : 0u;
+        for (int sb = 0; sb < 2; sb++) {
+          for (int jp = 0; jp < 2; jp++) {               // columns 2 jp and 2 jp + 1 share a canonical byte
+            const int col = col0 + 32 * q + 8 * (2 * x + sb) + 4 * hh + 2 * jp;
+            unsigned char* byte = src.w + (col >> 1);
+            const int n0 = 2 * (2 * jp) + sb, n1 = 2 * (2 * jp + 1) + sb;
+            if (!inverse) {
+              const unsigned bv = *byte;
+              word |= (bv & 0xFu) << (4 * n0);
+              word |= (bv >> 4) << (4 * n1);
+            } else {
+              *byte = (unsigned char)(((word >> (4 * n0)) & 0xFu) | (((word >> (4 * n1)) & 0xFu) << 4));
+            }
+          }
+        }
+        v[q] = word;
+      }
+      if (!inverse) *chunk = make_uint4(v[0], v[1], v[2], v[3]);
+      if (c == 0) {
+        // fp16 {scale, zero} of this row's group (= this block) after the unit's code bytes
+        unsigned* sz = reinterpret_cast<unsigned*>(unit + (size_t)urows * 64 + (size_t)gi * 4);
         if (!inverse) {
-          if (sc && zr)
-            *sz = make_uint2((unsigned)sc[2 * b] | ((unsigned)zr[2 * b] << 16),
-                           (unsigned)sc[2 * b + 1] | ((unsigned)zr[2 * b + 1] << 16));
+          if (src.scale && src.zero) *sz = (unsigned)src.scale[b] | ((unsigned)src.zero[b] << 16);
         } else {
-          const uint2 v = *sz;
-          if (sc) { sc[2 * b] = (unsigned short)(v.x & 0xffffu); sc[2 * b + 1] = (unsigned short)(v.y & 0xffffu); }
-          if (zr) { zr[2 * b] = (unsigned short)(v.x >> 16); zr[2 * b + 1] = (unsigned short)(v.y >> 16); }
+          const unsigned t = *sz;
+          if (src.scale) src.scale[b] = (unsigned short)(t & 0xffffu);
+          if (src.zero) src.zero[b] = (unsigned short)(t >> 16);
         }
       }
     }
@@ -182,10 +207,10 @@ __global__ void quantize_int4_kernel(const unsigned short* __restrict__ w, int64
 
 }  // namespace
 
-cudaError_t launch_pack(const OpDesc& d, const PackSrc& src, unsigned char* packed, int n_blocks, int stage_bytes,
+cudaError_t launch_pack(const PackOp& d, const PackSrc& src, unsigned char* packed, int n_blocks, int stage_bytes,
                         bool inverse, cudaStream_t stream) {
-  if (d.rows <= 0) return cudaSuccess;
-  pack_kernel<<<d.rows, 256, 0, stream>>>(d, src, packed, n_blocks, stage_bytes, inverse ? 1 : 0);
+  if (d.s.rows <= 0) return cudaSuccess;
+  pack_kernel<<<d.s.rows, 128, 0, stream>>>(d, src, packed, n_blocks, stage_bytes, inverse ? 1 : 0);
   return cudaGetLastError();
 }
 

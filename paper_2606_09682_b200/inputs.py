@@ -56,7 +56,7 @@ SHAPES: Dict[str, ModelShape] = {
     "toy_ragged": ModelShape("toy_ragged", 192, 3, 6, 2, 32, 328, 1003, 96, True),
     # small shapes the CUDA kernel accepts (head_dim 64 / 128), spanning several tiles and ragged tails
     "mini": ModelShape("mini", 256, 2, 4, 2, 64, 512, 1000, 128, False),
-    "mini_ragged": ModelShape("mini_ragged", 208, 3, 3, 1, 64, 336, 1003, 96, True),
+    "mini_ragged": ModelShape("mini_ragged", 192, 3, 3, 1, 64, 320, 1003, 96, True),
     "mini_hd128": ModelShape("mini_hd128", 512, 2, 8, 2, 128, 1024, 2048, 256, False, rope_theta=500000.0),
     "mini_wide": ModelShape("mini_wide", 1024, 2, 16, 2, 64, 2816, 5000, 512, False),
     "smollm2_135m": ModelShape("smollm2_135m", 576, 30, 9, 3, 64, 1536, 49152, 2048, True),

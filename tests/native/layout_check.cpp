@@ -1,7 +1,11 @@
-// Host-side exhaustive check of the packed-weight geometry (amk_layout.h): for one op it replays what the
-// packer writes, what the producer copies and what every consumer warp reads, and verifies that
-//   * every (row, column) of the matrix is read exactly once, with the activation index it belongs to,
-//   * every ring tile is 16-byte aligned, fits the stage, and tiles are contiguous and cover the slice,
+// Host-side exhaustive check of the packed-weight geometry (amk_layout.h): for one op it replays where the
+// packer puts every weight, what the producer copies and which work units every consumer warp reads, and
+// verifies that
+//   * every (row, column) of the matrix lands in exactly one place, and every stored element is read by
+//     exactly one warp (its row group, its column blocks),
+//   * inside a block, logical k -> (chunk, element) and logical k -> natural column are bijections, and the
+//     columns one lane quad supplies to the tensor core for a block are one contiguous run,
+//   * every ring tile is 16-byte aligned, fits the stage, and the tiles of a pass are contiguous and cover it,
 //   * every work unit a consumer warp touches lies inside the tile it waits for.
 // Usage: layout_check rows K wdtype unit_rows n_blocks stage_bytes   -> prints "ok" or a diagnostic.
 #include <cstdio>
@@ -16,78 +20,110 @@ int main(int argc, char** argv) {
   if (argc < 7) return 2;
   const int rows = atoi(argv[1]), K = atoi(argv[2]), wd = atoi(argv[3]), unit_rows = atoi(argv[4]);
   const int N = atoi(argv[5]), stage = atoi(argv[6]);
-  const int64_t rb = row_bytes(wd, K);
-  const int64_t total = (int64_t)rows * rb;
-  // packer: for each element, the byte offset (and nibble for int4) where it lands; record owner (row, col)
-  // granularity: one entry per 8-element lane chunk start offset -> (row, c0, c1)
+  const int bc = block_cols(wd), cpb = block_chunks(wd);
+  const int epc = bc / cpb;                     // elements per 16-byte chunk
+  if (K % bc) { printf("K not a multiple of the column block\n"); return 1; }
+  // the in-block permutation
+  {
+    std::vector<int> col_seen(bc, 0), place_seen(bc, 0);
+    for (int k = 0; k < bc; k++) {
+      int ch, el;
+      place_of_k(wd, k, &ch, &el);
+      const int col = col_of_k(wd, k);
+      if (col < 0 || col >= bc || ch < 0 || ch >= cpb || el < 0 || el >= epc) { printf("k map out of range\n"); return 1; }
+      col_seen[col]++;
+      place_seen[ch * epc + el]++;
+    }
+    for (int i = 0; i < bc; i++) if (col_seen[i] != 1 || place_seen[i] != 1) { printf("k map not a bijection\n"); return 1; }
+    // lane quad q supplies, for every step and half, consecutive columns starting at q * bc / 4
+    const int per_q = bc / 4, jn = (wd == W_BF16) ? 2 : 4, kstep = (wd == W_BF16) ? 16 : 32;
+    for (int k = 0; k < bc; k++) {
+      const int q = (wd == W_BF16) ? ((k >> 1) & 3) : ((k >> 2) & 3);
+      const int s = k / kstep, h = (k / (kstep / 2)) & 1, j = k % jn;
+      const int expect = q * per_q + (s * 2 + h) * jn + j;
+      if (col_of_k(wd, k) != expect) { printf("lane supply not contiguous at k=%d\n", k); return 1; }
+    }
+  }
   std::vector<int> seen((size_t)rows * K, 0);
-  std::vector<unsigned char> owner_mark((size_t)total, 0);
-  int64_t covered = 0;
+  long long covered = 0;
   for (int slot = 0; slot < N; slot++) {
     const Slice sl = slot_slice(rows, unit_rows, N, slot);
     for (int r = sl.row0; r < sl.row0 + sl.rows; r++)
       if (slot_of_row(rows, unit_rows, N, r) != slot) { printf("slot_of_row mismatch row %d\n", r); return 1; }
-    const int64_t base = (int64_t)sl.row0 * rb;
     const int np = n_passes(sl.rows);
-    int64_t slice_bytes = 0;
+    long long sbytes = 0;
     for (int ps = 0; ps < np; ps++) {
       const int R = pass_rows(sl.rows, ps);
       const PassGeom g = pass_geom(R, K, wd, stage);
-      if (g.G < 1 || g.G > kGMax || g.Wr * g.Wk > kConsumerWarps || g.Wr < 1 || g.Wk < 1) { printf("bad geom R=%d G=%d Wr=%d Wk=%d\n", R, g.G, g.Wr, g.Wk); return 1; }
-      if ((g.Wr - 1) * g.G >= R || g.Wr * g.G < R) { printf("row split wrong R=%d G=%d Wr=%d\n", R, g.G, g.Wr); return 1; }
-      const int64_t pbase = base + (int64_t)ps * kPassRows * rb;
-      if (pass_bytes(g) != (int64_t)R * rb) { printf("pass bytes %lld != %lld\n", (long long)pass_bytes(g), (long long)R * rb); return 1; }
+      if (g.G < 1 || g.G > kGMax || g.Wr * g.Wk > kConsumerWarps || g.Wr < 1 || g.Wk < 1 || g.g_last < 1 || g.g_last > g.G ||
+          (g.Wr - 1) * g.G + g.g_last != R) {
+        printf("bad geom R=%d G=%d g_last=%d Wr=%d Wk=%d\n", R, g.G, g.g_last, g.Wr, g.Wk);
+        return 1;
+      }
+      std::vector<unsigned char> mark((size_t)pass_bytes(g), 0);
       // producer tiles
-      int64_t prev_end = 0;
+      long long prev_end = 0;
       for (int t = 0; t < g.n_tiles; t++) {
-        const int u0 = t * g.upt;
-        const int64_t o0 = unit_off(g, u0), o1 = unit_off(g, u0 + g.upt);
+        const long long o0 = unit_off(g, t * g.upt), o1 = unit_off(g, (t + 1) * g.upt);
         if (o0 != prev_end) { printf("tile gap\n"); return 1; }
-        if ((o1 - o0) > stage || (o1 - o0) <= 0 || ((pbase + o0) & 15) || ((o1 - o0) & 15)) {
-          printf("tile size/alignment: R=%d K=%d t=%d o0=%lld o1=%lld\n", R, K, t, (long long)o0, (long long)o1); return 1;
+        if ((o1 - o0) > stage || (o1 - o0) <= 0 || ((sbytes + o0) & 15) || ((o1 - o0) & 15)) {
+          printf("tile size/alignment: R=%d K=%d t=%d o0=%lld o1=%lld\n", R, K, t, o0, o1);
+          return 1;
         }
         prev_end = o1;
       }
       if (prev_end != pass_bytes(g)) { printf("tiles do not cover the pass\n"); return 1; }
-      slice_bytes += prev_end;
-      // consumers
+      // consumers: the incremental walk of the kernel
       for (int warp = 0; warp < kConsumerWarps; warp++) {
         const int wr = warp % g.Wr, wk = warp / g.Wr;
         if (wk >= g.Wk) continue;
-        const int my_rows = (g.R - wr * g.G) < g.G ? (g.R - wr * g.G) : g.G;
+        const int urows = (wr == g.Wr - 1) ? g.g_last : g.G;
+        int next_b = wk, t_b = 0, t_r = 0;
+        const int step_b = g.upt / g.Wr, step_r = g.upt - step_b * g.Wr;
         for (int t = 0; t < g.n_tiles; t++) {
-          const int u0 = t * g.upt, u1 = (u0 + g.upt < g.n_units) ? u0 + g.upt : g.n_units;
-          const int64_t t0 = unit_off(g, u0), t1 = unit_off(g, u0 + g.upt);
-          int b = (u0 > wr) ? (u0 - wr + g.Wr - 1) / g.Wr : 0;
-          b += ((wk - b) % g.Wk + g.Wk) % g.Wk;
-          for (; b * g.Wr + wr < u1; b += g.Wk) {
-            const bool is_tail = g.tail && (b == g.nblk - 1);
-            const int wdt = is_tail ? g.tail : kBlockCols;
-            const int rc = is_tail ? g.rc_tail : g.rc_full;
-            const int64_t uo = unit_off_br(g, b, wr);
-            if (uo < t0 || uo + (int64_t)my_rows * rc > t1) { printf("unit outside its tile\n"); return 1; }
-            for (int i = 0; i < my_rows; i++) {
+          const long long tile_off = (long long)t_b * g.bb + (long long)t_r * g.ub_full;
+          if (tile_off != unit_off(g, t * g.upt)) { printf("tile walk drifted\n"); return 1; }
+          const long long tile_end = unit_off(g, (t + 1) * g.upt);
+          int n_b = t_b + step_b, n_r = t_r + step_r;
+          if (n_r >= g.Wr) { n_r -= g.Wr; n_b++; }
+          while (next_b < g.nblk && (next_b < n_b || (next_b == n_b && wr < n_r))) {
+            const long long uo = (long long)next_b * g.bb + (long long)wr * g.ub_full;
+            if (uo < tile_off || uo + unit_bytes(wd, urows) > tile_end) { printf("unit outside its tile\n"); return 1; }
+            // every element of the unit: row i, chunk c, element e  ->  (row, column)
+            for (int i = 0; i < urows; i++) {
               const int row = sl.row0 + ps * kPassRows + wr * g.G + i;
-              for (int lane = 0; lane < wdt / 8; lane++) {
-                const int64_t off = pbase + uo + (int64_t)i * rc + lane * (wd == W_BF16 ? 16 : (wd == W_INT8 ? 8 : 4));
-                if (off < 0 || off >= total) { printf("offset out of range\n"); return 1; }
-                if (owner_mark[off]) { printf("byte read twice: off %lld\n", (long long)off); return 1; }
-                owner_mark[off] = 1;
-                for (int e = 0; e < 8; e++) {
-                  const int col = b * kBlockCols + lane_col(wdt, lane, e);
-                  if (col >= K) { printf("column out of range\n"); return 1; }
-                  seen[(size_t)row * K + col]++;
-                }
+              for (int k = 0; k < bc; k++) {
+                int ch, el;
+                place_of_k(wd, k, &ch, &el);
+                const long long byte = uo + ((long long)ch * urows + i) * 16 + (wd == W_BF16 ? el * 2 : (wd == W_INT8 ? el : el / 2));
+                if (byte >= (long long)mark.size()) { printf("element outside the pass\n"); return 1; }
+                mark[byte] = 1;
+                if (wd == W_BF16) mark[byte + 1] = 1;
+                seen[(size_t)row * K + (size_t)next_b * bc + col_of_k(wd, k)]++;
+              }
+              if (wd == W_INT4) {
+                const long long sz = uo + (long long)urows * 64 + i * 4;
+                for (int e = 0; e < 4; e++) mark[sz + e] = 1;
               }
             }
+            next_b += g.Wk;
           }
+          t_b = n_b;
+          t_r = n_r;
         }
+        if (next_b < g.nblk) { printf("a warp did not reach all its blocks\n"); return 1; }
       }
+      // every byte except unit padding is used
+      long long used = 0;
+      for (unsigned char m : mark) used += m;
+      const long long expect = (long long)R * g.nblk * (wd == W_BF16 ? 128 : (wd == W_INT8 ? 64 : 68));
+      if (used != expect) { printf("bytes used %lld, expected %lld\n", used, expect); return 1; }
+      sbytes += pass_bytes(g);
     }
-    if (slice_bytes != (int64_t)sl.rows * rb) { printf("slice bytes mismatch\n"); return 1; }
+    if (sbytes != slice_bytes(sl.rows, K, wd, stage)) { printf("slice bytes mismatch\n"); return 1; }
     covered += sl.rows;
   }
-  if (covered != rows) { printf("rows covered %lld of %d\n", (long long)covered, rows); return 1; }
+  if (covered != rows) { printf("rows covered %lld of %d\n", covered, rows); return 1; }
   for (size_t i = 0; i < seen.size(); i++)
     if (seen[i] != 1) { printf("element (%zu,%zu) read %d times\n", i / K, i % K, seen[i]); return 1; }
   printf("ok\n");
