@@ -67,12 +67,12 @@ enum { AMK_LIN_Q = 0, AMK_LIN_K = 1, AMK_LIN_V = 2, AMK_LIN_O = 3, AMK_LIN_GATE 
 typedef struct amk_config {
   uint32_t struct_size;      /* = sizeof(amk_config)                                                   */
   uint32_t abi_version;      /* = AMK_ABI_VERSION                                                      */
-  uint32_t hidden;           /* H; multiple of 64 (128 for int4), at most 7680                         */
+  uint32_t hidden;           /* H; multiple of 64 (128 for int4), at most 5632                         */
   uint32_t n_layers;         /* L                                                                      */
   uint32_t n_q_heads;        /* multiple of n_kv_heads; n_q_heads / n_kv_heads <= 16                   */
   uint32_t n_kv_heads;
   uint32_t head_dim;         /* 64 or 128                                                              */
-  uint32_t mlp;              /* I; multiple of 64 (128 for int4), at most 15360                        */
+  uint32_t mlp;              /* I; multiple of 64 (128 for int4)                                       */
   uint32_t vocab;            /* V                                                                      */
   uint32_t max_seq;          /* S: positions the KV cache holds                                        */
   uint32_t tied_embeddings;  /* 1: the LM head is the embedding matrix                                 */
@@ -92,7 +92,8 @@ typedef struct amk_config {
                                 model); 1: sequence numbers only (no counters, no fences).  Same results.  */
   uint32_t n_blocks;         /* persistent blocks; 0 = one per SM of the current device (148 if there is
                                 no device).  The packed layout depends on it.                          */
-  uint32_t reserved[1];      /* must be 0                                                              */
+  uint32_t l2_ahead;         /* ring tiles the producer requests into L2 beyond the ring (weight prefetch
+                                hint, as in the paper's Algorithm 1); 0 = automatic, 33 = off, max 32    */
 } amk_config;
 
 /*
@@ -123,6 +124,7 @@ typedef struct amk_plan {
   uint32_t threads;           /* threads per block (one producer warp + consumer warps)                */
   uint32_t smem_bytes;        /* dynamic shared memory per block                                       */
   uint32_t stage_bytes, n_stages, max_inflight;
+  uint32_t l2_ahead;          /* ring tiles requested into L2 ahead of the ring                        */
   uint32_t n_gemv_ops;        /* 4 per layer + LM head                                                 */
   uint32_t n_phases;          /* dependency joins per token                                            */
   uint64_t packed_bytes, workspace_bytes, kv_bytes;

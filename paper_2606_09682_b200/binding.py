@@ -33,8 +33,7 @@ class amk_config(C.Structure):
                                           "tied_embeddings")] + [
         ("rms_eps", C.c_float), ("rope_theta", C.c_float)] + [
         (n, C.c_uint32) for n in ("wdtype", "group_size", "quantize_lm_head", "wait_timeout_us", "flags",
-                                  "stage_bytes", "n_stages", "max_inflight", "sync_mode", "n_blocks")] + [
-        ("reserved", C.c_uint32 * 1)]
+                                  "stage_bytes", "n_stages", "max_inflight", "sync_mode", "n_blocks", "l2_ahead")]
 
 
 _PP = C.POINTER(C.c_void_p)
@@ -48,7 +47,7 @@ class amk_weights(C.Structure):
 
 class amk_plan(C.Structure):
     _fields_ = [(n, C.c_uint32) for n in ("n_blocks", "threads", "smem_bytes", "stage_bytes", "n_stages",
-                                          "max_inflight", "n_gemv_ops", "n_phases")] + [
+                                          "max_inflight", "l2_ahead", "n_gemv_ops", "n_phases")] + [
         (n, C.c_uint64) for n in ("packed_bytes", "workspace_bytes", "kv_bytes", "weight_stream_bytes")]
 
 
@@ -102,7 +101,7 @@ def _check(code: int, what: str):
 
 def make_config(shape, wdtype: str = "bf16", flags: int = 0, wait_timeout_us: int = 0, stage_bytes: int = 0,
                 n_stages: int = 0, max_inflight: int = 0, group_size: int = 128, sync_mode: int = 1,
-                n_blocks: int = 0) -> amk_config:
+                n_blocks: int = 0, l2_ahead: int = 0) -> amk_config:
     """``shape``: any object with hidden, n_layers, n_q_heads, n_kv_heads, head_dim, mlp, vocab, max_seq,
     tied, rms_eps, rope_theta attributes."""
     c = amk_config()
@@ -115,7 +114,7 @@ def make_config(shape, wdtype: str = "bf16", flags: int = 0, wait_timeout_us: in
     c.group_size = group_size if wdtype == "int4" else 0
     c.wait_timeout_us, c.flags = wait_timeout_us, flags
     c.stage_bytes, c.n_stages, c.max_inflight = stage_bytes, n_stages, max_inflight
-    c.sync_mode, c.n_blocks = sync_mode, n_blocks
+    c.sync_mode, c.n_blocks, c.l2_ahead = sync_mode, n_blocks, l2_ahead
     return c
 
 
@@ -198,11 +197,11 @@ class Decoder:
 
     def __init__(self, shape, weights: Dict, wdtype: str = "bf16", flags: int = 0, wait_timeout_us: int = 0,
                  stage_bytes: int = 0, n_stages: int = 0, max_inflight: int = 0, sync_mode: int = 1,
-                 n_blocks: int = 0, device="cuda"):
+                 n_blocks: int = 0, l2_ahead: int = 0, device="cuda"):
         self.shape, self.wdtype = shape, wdtype
         self.device = torch.device(device)
         self.cfg = make_config(shape, wdtype, flags, wait_timeout_us, stage_bytes, n_stages, max_inflight,
-                               sync_mode=sync_mode, n_blocks=n_blocks)
+                               sync_mode=sync_mode, n_blocks=n_blocks, l2_ahead=l2_ahead)
         self.packed = torch.empty(amk_packed_bytes(self.cfg), dtype=torch.uint8, device=self.device)
         self.workspace = torch.empty(amk_workspace_bytes(self.cfg), dtype=torch.uint8, device=self.device)
         keep: List = []

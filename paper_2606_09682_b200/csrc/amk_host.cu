@@ -60,7 +60,7 @@ int resolve_blocks(const amk_config* c) {
 amk_status check_config(const amk_config* c) {
   if (!c) return AMK_ERR_INVALID_ARG;
   if (c->struct_size != sizeof(amk_config) || c->abi_version != AMK_ABI_VERSION) return AMK_ERR_INVALID_ARG;
-  for (uint32_t r : c->reserved) if (r) return AMK_ERR_INVALID_ARG;
+  if (c->l2_ahead > 33u) return AMK_ERR_INVALID_ARG;
   if (!c->hidden || !c->n_layers || !c->n_q_heads || !c->n_kv_heads || !c->mlp || !c->vocab || !c->max_seq)
     return AMK_ERR_INVALID_ARG;
   if (c->wdtype > AMK_W_INT4 || c->sync_mode > 1) return AMK_ERR_INVALID_ARG;
@@ -72,7 +72,7 @@ amk_status check_config(const amk_config* c) {
   const uint32_t kdiv = (c->wdtype == AMK_W_INT4) ? 128 : 64;
   const uint32_t qdim = c->n_q_heads * c->head_dim;
   if (c->hidden % kdiv || c->mlp % kdiv || qdim % kdiv) return AMK_ERR_UNSUPPORTED;
-  if (c->hidden > 7680u || c->mlp > 15360u || qdim > 15360u) return AMK_ERR_UNSUPPORTED;   // prologue register budget
+  if (c->hidden > 16u * kConsumerThreads) return AMK_ERR_UNSUPPORTED;   // a normed input is gathered in one batch
   if (c->wdtype == AMK_W_INT4 && c->group_size != 128) return AMK_ERR_UNSUPPORTED;
   if ((uint64_t)c->vocab * c->hidden > (1ull << 40)) return AMK_ERR_UNSUPPORTED;
   if (c->stage_bytes && (c->stage_bytes % 1024 || c->stage_bytes < 8192 || c->stage_bytes > 65536))
@@ -328,7 +328,7 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     if ((size_t)qd > kmax) kmax = qd;
     size_t act = kmax * (cfg->wdtype == AMK_W_BF16 ? 4 : 3);   // bf16 high + low halves, or three int8 digits
     if ((size_t)H * 4 > act) act = (size_t)H * 4;               // the LM head is always bf16
-    const size_t attn_need = ((size_t)n_rep * hd + (size_t)kConsumerWarps * 4 * (hd + 2)) * 4;
+    const size_t attn_need = ((size_t)n_rep * hd + (size_t)kConsumerWarps * 4 * (hd + 2)) * 4 + (size_t)hd * 4;
     if (attn_need > act) act = attn_need;
     act = (act + 127) & ~(size_t)127;
     const uint32_t stage_bytes = h->pl.stage_bytes;
@@ -346,7 +346,7 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     if (max_inflight > n_stages) max_inflight = n_stages;
     const size_t smem_bytes = hdr + act + (size_t)n_stages * stage_bytes;
     int per_sm = 0;
-    AMK_CUDA(decode_kernel_attrs(smem_bytes, &per_sm));
+    AMK_CUDA(decode_kernel_attrs((int)cfg->wdtype, hd, smem_bytes, &per_sm));
     if (per_sm < 1) {
       snprintf(h->errmsg, sizeof(h->errmsg), "decode kernel does not fit one block per SM");
       status = AMK_ERR_UNSUPPORTED;
@@ -445,6 +445,7 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     p.status = (DevStatus*)(h->ws + h->wl.status);
     p.trace = (cfg->flags & AMK_FLAG_TRACE) ? (unsigned long long*)(h->ws + h->wl.trace) : nullptr;
     p.stage_bytes = (int)stage_bytes; p.n_stages = (int)n_stages; p.max_inflight = (int)max_inflight;
+    p.l2_ahead = cfg->l2_ahead == 0 ? 6 : (cfg->l2_ahead > 32 ? 0 : (int)cfg->l2_ahead);
     p.act_bytes = (int)act;
     p.timeout_ns = 1000ull * (cfg->wait_timeout_us ? cfg->wait_timeout_us : 200000u);
     p.drop_phase = -1; p.drop_block = -1;
@@ -452,6 +453,7 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     amk_plan& pn = h->plan;
     pn.n_blocks = n_blocks; pn.threads = kThreads; pn.smem_bytes = (uint32_t)smem_bytes;
     pn.stage_bytes = stage_bytes; pn.n_stages = n_stages; pn.max_inflight = max_inflight;
+    pn.l2_ahead = (uint32_t)p.l2_ahead;
     pn.n_gemv_ops = (uint32_t)h->pl.ops.size(); pn.n_phases = 5 * L;
     pn.packed_bytes = h->pl.packed_total; pn.workspace_bytes = h->wl.total; pn.kv_bytes = kv_bytes_of(cfg);
     pn.weight_stream_bytes = h->pl.weight_stream_bytes;

@@ -87,6 +87,7 @@ struct KParams {
   unsigned long long* trace;              // [n_blocks][5 L + 1][8] or null
   // plan
   int stage_bytes, n_stages, max_inflight;
+  int l2_ahead;                           // ring tiles requested into L2 ahead of the ring (0..32)
   int act_bytes;                          // activation / attention scratch area in shared memory
   unsigned long long timeout_ns;
   int drop_phase, drop_block;             // test hook: this block does not publish this task's output
@@ -94,7 +95,7 @@ struct KParams {
 
 // Launchers implemented in the .cu files.
 cudaError_t launch_decode(const KParams& p, int n_blocks, size_t smem_bytes, cudaStream_t stream);
-cudaError_t decode_kernel_attrs(size_t smem_bytes, int* max_blocks_per_sm);
+cudaError_t decode_kernel_attrs(int wdtype, int hd, size_t smem_bytes, int* max_blocks_per_sm);
 
 // One op to pack: its shape, rotation and region, plus where the canonical rows come from.
 struct PackOp {

@@ -35,9 +35,8 @@ namespace {
 
 constexpr int kBarCons = 1;                          // named barrier of the consumer warps
 constexpr int kOutWarps = (kPassRows + 31) / 32;     // warps that hold a pass's output rows
-constexpr int kLines = 16;                           // 16-byte activation lines per thread (K <= 2 * 480 * 16)
-constexpr int kBatch = 8;                            // lines gathered at a time
-constexpr int kNormLines = 8;                        // lines per thread of a normed input (H <= 7680)
+constexpr int kBatch = 8;                            // 16-byte activation lines a thread gathers at a time
+                                                     // (a normed input must fit one batch per thread)
 constexpr float kDigitScale = 1048575.0f;            // int8 / int4 activations: 3 signed base-128 digits
 
 struct Ctx {
@@ -151,44 +150,48 @@ __device__ __forceinline__ float warp_max(float v) {
   return v;
 }
 
-// Spin until both elements of the line at `addr` carry `seq`; bounded.
-__device__ __noinline__ bool poll_pair2_slow(const KParams& p, const void* addr, unsigned seq, int task, uint4* out) {
+// Spin until both elements of the line at `addr` carry `seq`; bounded.  On failure the returned line does
+// not carry `seq` (values are returned, not written through a pointer, so callers' arrays stay in registers).
+__device__ __noinline__ uint4 poll_pair2_slow(const KParams& p, const void* addr, unsigned seq, int task) {
   const unsigned long long t0 = globaltimer_ns();
   unsigned spins = 0;
   for (;;) {
-    const uint4 v = ld_pair2(addr);
-    if (v.y == seq && v.w == seq) { *out = v; return true; }
+    uint4 v = ld_pair2(addr);
+    if (v.y == seq && v.w == seq) return v;
     if ((++spins & 15u) == 0u) {
-      if (ld_relaxed_gpu(&p.status->abort)) return false;
-      if (globaltimer_ns() - t0 > p.timeout_ns) {
+      bool give_up = ld_relaxed_gpu(&p.status->abort) != 0u;
+      if (!give_up && globaltimer_ns() - t0 > p.timeout_ns) {
         report_failure(p, (unsigned)AMK_ERR_TIMEOUT, task, v.y == seq ? v.w : v.y, seq);
-        return false;
+        give_up = true;
       }
+      if (give_up) { v.y = seq + 1u; return v; }
     }
   }
 }
-__device__ __noinline__ bool poll_pair_slow(const KParams& p, const void* addr, unsigned seq, int task, float* out) {
+__device__ __noinline__ uint2 poll_pair_slow(const KParams& p, const void* addr, unsigned seq, int task) {
   const unsigned long long t0 = globaltimer_ns();
   unsigned spins = 0;
   for (;;) {
-    const uint2 v = ld_pair(addr);
-    if (v.y == seq) { *out = __uint_as_float(v.x); return true; }
+    uint2 v = ld_pair(addr);
+    if (v.y == seq) return v;
     if ((++spins & 15u) == 0u) {
-      if (ld_relaxed_gpu(&p.status->abort)) return false;
-      if (globaltimer_ns() - t0 > p.timeout_ns) {
+      bool give_up = ld_relaxed_gpu(&p.status->abort) != 0u;
+      if (!give_up && globaltimer_ns() - t0 > p.timeout_ns) {
         report_failure(p, (unsigned)AMK_ERR_TIMEOUT, task, v.y, seq);
-        return false;
+        give_up = true;
       }
+      if (give_up) { v.y = seq + 1u; return v; }
     }
   }
 }
 // One activation element written by `task` in this step.
-__device__ __forceinline__ float read_act(Ctx& c, const ActPair* a, unsigned seq, int task) {
-  const uint2 v = ld_pair(a);
-  if (v.y == seq) return __uint_as_float(v.x);
-  float r = 0.f;
-  if (!poll_pair_slow(c.p, a, seq, task, &r)) c.bad = true;
-  return r;
+__device__ __forceinline__ float read_act(const KParams& p, bool& bad, const ActPair* a, unsigned seq, int task) {
+  uint2 v = ld_pair(a);
+  if (v.y != seq) {
+    v = poll_pair_slow(p, a, seq, task);
+    if (v.y != seq) bad = true;
+  }
+  return __uint_as_float(v.x);
 }
 
 __device__ __forceinline__ float silu_f(float z) { return z / (1.0f + expf(-z)); }
@@ -199,116 +202,153 @@ __device__ __forceinline__ float silu_f(float z) { return z / (1.0f + expf(-z));
 //   bf16 weights: X0[K] = bf16(a), X1[K] = bf16(a - X0): two B columns whose sum is a to ~2^-17.
 //   int8 / int4 : a / scale as three signed base-128 digits D2, D1, D0 (three B columns), exact integers.
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ bool load_input(Ctx& c, int wd, int K, const ActPair* src, unsigned seq, int src_task,
-                                           const unsigned short* embed_row, const unsigned short* normw, int task) {
-  const KParams& p = c.p;
-  const int n2 = K >> 1;                               // lines of two elements
-  float2 v[kLines];
-  unsigned gw[kNormLines];
-  if (normw) {
-#pragma unroll
-    for (int i = 0; i < kNormLines; i++) {
-      const int ln = c.tid + i * kConsumerThreads;
-      gw[i] = (ln < n2) ? __ldg(reinterpret_cast<const unsigned*>(normw) + ln) : 0u;
-    }
-  }
-  float ss = 0.f, amax = 0.f;
-#pragma unroll
-  for (int i0 = 0; i0 < kLines; i0 += kBatch) {
-    if (i0 * kConsumerThreads >= n2) break;
-    // issue a batch of loads first, then settle the ones that had not arrived
-    uint4 raw[kBatch];
-#pragma unroll
-    for (int i = 0; i < kBatch; i++) {
-      const int ln = c.tid + (i0 + i) * kConsumerThreads;
-      if (ln < n2) {
-        if (embed_row) {
-          const unsigned w = __ldg(reinterpret_cast<const unsigned*>(embed_row) + ln);
-          raw[i] = make_uint4(w << 16, seq, w & 0xffff0000u, seq);
-        } else {
-          raw[i] = ld_pair2(src + 2 * ln);
-        }
-      }
-    }
-#pragma unroll
-    for (int i = 0; i < kBatch; i++) {
-      const int ln = c.tid + (i0 + i) * kConsumerThreads;
-      if (ln < n2) {
-        if (raw[i].y != seq || raw[i].w != seq) {
-          if (!poll_pair2_slow(p, src + 2 * ln, seq, src_task, &raw[i])) c.bad = true;
-        }
-        float a = __uint_as_float(raw[i].x), b = __uint_as_float(raw[i].z);
-        if (normw) {
-          ss = fmaf(a, a, ss);
-          ss = fmaf(b, b, ss);
-          if (embed_row && c.cta == 0 && (p.flags & AMK_FLAG_DEBUG_HIDDEN))
-            reinterpret_cast<float2*>(p.hidden)[ln] = make_float2(a, b);
-          if (i0 + i < kNormLines) { a *= bf16_lo(gw[(i0 + i) % kNormLines]); b *= bf16_hi(gw[(i0 + i) % kNormLines]); }
-        }
-        v[i0 + i] = make_float2(a, b);                 // norm weight applied; 1/rms follows the sum
-        amax = fmaxf(amax, fmaxf(fabsf(a), fabsf(b)));
-      }
-    }
-  }
-  if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_JOINED);
-  float r = 1.0f;
-  if (normw || wd != W_BF16) {
-    ss = warp_sum(ss);
-    amax = warp_max(amax);
-    if (c.lane == 0) { c.sh->warp_part[0][c.warp] = ss; c.sh->warp_part[1][c.warp] = amax; }
-    c.bad = cons_sync_or(c.bad);
-    if (c.bad) return false;
-    float tot = 0.f, mx = 0.f;
-#pragma unroll
-    for (int w = 0; w < kConsumerWarps; w++) { tot += c.sh->warp_part[0][w]; mx = fmaxf(mx, c.sh->warp_part[1][w]); }
-    if (normw) r = 1.0f / sqrtf(tot / (float)K + p.eps);
-    amax = mx * r;
-  }
-  if (wd == W_BF16) {
-    unsigned* X0 = reinterpret_cast<unsigned*>(c.xs);
+
+// two input elements -> their shared-memory form (line `ln` = elements 2 ln, 2 ln + 1)
+template <int WD>
+__device__ __forceinline__ void store_line(unsigned char* xs, int n2, int ln, float a, float b, float inv) {
+  if (WD == W_BF16) {
+    unsigned* X0 = reinterpret_cast<unsigned*>(xs);
     unsigned* X1 = X0 + n2;
-#pragma unroll
-    for (int i = 0; i < kLines; i++) {
-      const int ln = c.tid + i * kConsumerThreads;
-      if (ln < n2) {
-        const float a = v[i].x * r, b = v[i].y * r;
-        const unsigned ha = f32_to_bf16_rne(a), hb = f32_to_bf16_rne(b);
-        const unsigned la = f32_to_bf16_rne(a - __uint_as_float(ha << 16));
-        const unsigned lb = f32_to_bf16_rne(b - __uint_as_float(hb << 16));
-        X0[ln] = ha | (hb << 16);
-        X1[ln] = la | (lb << 16);
-      }
-    }
+    const unsigned ha = f32_to_bf16_rne(a), hb = f32_to_bf16_rne(b);
+    const unsigned la = f32_to_bf16_rne(a - __uint_as_float(ha << 16));
+    const unsigned lb = f32_to_bf16_rne(b - __uint_as_float(hb << 16));
+    X0[ln] = ha | (hb << 16);
+    X1[ln] = la | (lb << 16);
   } else {
-    const float inv = amax > 0.f ? kDigitScale / amax : 0.f;
-    c.xscale = amax / kDigitScale;
-    unsigned short* D2 = reinterpret_cast<unsigned short*>(c.xs);
+    unsigned short* D2 = reinterpret_cast<unsigned short*>(xs);
     unsigned short* D1 = D2 + n2;
     unsigned short* D0 = D1 + n2;
+    unsigned d2 = 0, d1 = 0, d0 = 0;
 #pragma unroll
-    for (int i = 0; i < kLines; i++) {
-      const int ln = c.tid + i * kConsumerThreads;
+    for (int e = 0; e < 2; e++) {
+      const int X = __float2int_rn((e ? b : a) * inv);
+      const int e0 = ((X + 64) & 127) - 64;
+      const int X1 = (X - e0) >> 7;
+      const int e1 = ((X1 + 64) & 127) - 64;
+      const int e2 = (X1 - e1) >> 7;
+      d0 |= (unsigned)(e0 & 0xff) << (8 * e);
+      d1 |= (unsigned)(e1 & 0xff) << (8 * e);
+      d2 |= (unsigned)(e2 & 0xff) << (8 * e);
+    }
+    D2[ln] = (unsigned short)d2;
+    D1[ln] = (unsigned short)d1;
+    D0[ln] = (unsigned short)d0;
+  }
+}
+
+// Gather one batch of lines (line0, line0 + T, ...): request them all, and if any has not arrived yet request
+// the whole batch again until all carry `seq` (bounded).  Returns true on failure.
+__device__ __forceinline__ bool gather_batch(const KParams& p, uint4 (&raw)[kBatch], int line0, int n2,
+                                             const ActPair* src, unsigned seq, int src_task,
+                                             const unsigned short* embed_row) {
+  if (embed_row) {
+#pragma unroll
+    for (int i = 0; i < kBatch; i++) {
+      const int ln = line0 + i * kConsumerThreads;
       if (ln < n2) {
-        unsigned d2 = 0, d1 = 0, d0 = 0;
+        const unsigned w = __ldg(reinterpret_cast<const unsigned*>(embed_row) + ln);
+        raw[i] = make_uint4(w << 16, seq, w & 0xffff0000u, seq);
+      }
+    }
+    return false;
+  }
+  unsigned long long t0 = 0;
+  for (unsigned spins = 0;; spins++) {
+    bool all = true;
 #pragma unroll
-        for (int e = 0; e < 2; e++) {
-          const int X = __float2int_rn((e ? v[i].y : v[i].x) * r * inv);
-          const int e0 = ((X + 64) & 127) - 64;
-          const int X1 = (X - e0) >> 7;
-          const int e1 = ((X1 + 64) & 127) - 64;
-          const int e2 = (X1 - e1) >> 7;
-          d0 |= (unsigned)(e0 & 0xff) << (8 * e);
-          d1 |= (unsigned)(e1 & 0xff) << (8 * e);
-          d2 |= (unsigned)(e2 & 0xff) << (8 * e);
-        }
-        D2[ln] = (unsigned short)d2;
-        D1[ln] = (unsigned short)d1;
-        D0[ln] = (unsigned short)d0;
+    for (int i = 0; i < kBatch; i++) {
+      const int ln = line0 + i * kConsumerThreads;
+      if (ln < n2) raw[i] = ld_pair2(src + 2 * ln);
+    }
+#pragma unroll
+    for (int i = 0; i < kBatch; i++) {
+      const int ln = line0 + i * kConsumerThreads;
+      if (ln < n2) all = all && (raw[i].y == seq) && (raw[i].w == seq);
+    }
+    if (all) return false;
+    if (spins == 0) t0 = globaltimer_ns();
+    if ((spins & 15u) == 15u) {
+      if (ld_relaxed_gpu(&p.status->abort)) return true;
+      if (globaltimer_ns() - t0 > p.timeout_ns) {
+        report_failure(p, (unsigned)AMK_ERR_TIMEOUT, src_task, 0u, seq);
+        return true;
       }
     }
   }
-  c.bad = cons_sync_or(c.bad);
-  return !c.bad;
+}
+
+struct LoadResult {
+  float xscale;      // int8 / int4: scale of the digit representation
+  bool bad;
+};
+
+// A vector short enough for one batch per thread (every normed input) is held in registers across the
+// reduction; longer vectors are never normed: they are converted as they arrive (bf16) or read twice
+// (integer inputs need their maximum first).
+template <int WD>
+__device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* sh, unsigned char* xs, int cta, int K,
+                                                 const ActPair* src, unsigned seq, int src_task,
+                                                 const unsigned short* embed_row, const unsigned short* normw,
+                                                 int task) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n2 = K >> 1;                               // lines of two elements
+  LoadResult res{1.0f, false};
+  uint4 raw[kBatch];
+  const bool reduce = (normw != nullptr) || (WD != W_BF16);
+  const bool held = n2 <= kBatch * kConsumerThreads;
+  float r = 1.0f, inv = 0.f;
+  if (reduce) {
+    float ss = 0.f, amax = 0.f;
+#pragma unroll 1
+    for (int l0 = tid; l0 < n2; l0 += kBatch * kConsumerThreads) {
+      res.bad |= gather_batch(p, raw, l0, n2, src, seq, src_task, embed_row);
+#pragma unroll
+      for (int i = 0; i < kBatch; i++) {
+        const int ln = l0 + i * kConsumerThreads;
+        if (ln < n2) {
+          float a = __uint_as_float(raw[i].x), b = __uint_as_float(raw[i].z);
+          if (normw) {                                 // (normed inputs are always held)
+            ss = fmaf(a, a, ss);
+            ss = fmaf(b, b, ss);
+            if (embed_row && cta == 0 && (p.flags & AMK_FLAG_DEBUG_HIDDEN))
+              reinterpret_cast<float2*>(p.hidden)[ln] = make_float2(a, b);
+            const unsigned gw = __ldg(reinterpret_cast<const unsigned*>(normw) + ln);
+            a *= bf16_lo(gw);                          // norm weight now, 1/rms after the sum
+            b *= bf16_hi(gw);
+            raw[i].x = __float_as_uint(a);
+            raw[i].z = __float_as_uint(b);
+          }
+          amax = fmaxf(amax, fmaxf(fabsf(a), fabsf(b)));
+        }
+      }
+    }
+    if (tid == 0) stamp(p, cta, task, AMK_TR_JOINED);
+    ss = warp_sum(ss);
+    amax = warp_max(amax);
+    if (lane == 0) { sh->warp_part[0][warp] = ss; sh->warp_part[1][warp] = amax; }
+    res.bad = cons_sync_or(res.bad);
+    float tot = 0.f, mx = 0.f;
+#pragma unroll
+    for (int w = 0; w < kConsumerWarps; w++) { tot += sh->warp_part[0][w]; mx = fmaxf(mx, sh->warp_part[1][w]); }
+    if (normw) r = 1.0f / sqrtf(tot / (float)K + p.eps);
+    mx *= r;
+    if (WD != W_BF16) {
+      inv = mx > 0.f ? kDigitScale / mx : 0.f;
+      res.xscale = mx / kDigitScale;
+    }
+  }
+#pragma unroll 1
+  for (int l0 = tid; l0 < n2; l0 += kBatch * kConsumerThreads) {
+    if (!(reduce && held)) res.bad |= gather_batch(p, raw, l0, n2, src, seq, src_task, embed_row);
+#pragma unroll
+    for (int i = 0; i < kBatch; i++) {
+      const int ln = l0 + i * kConsumerThreads;
+      if (ln < n2) store_line<WD>(xs, n2, ln, __uint_as_float(raw[i].x) * r, __uint_as_float(raw[i].z) * r, inv);
+    }
+  }
+  if (!reduce && tid == 0) stamp(p, cta, task, AMK_TR_JOINED);
+  res.bad = cons_sync_or(res.bad);
+  return res;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -444,7 +484,8 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int K, f
 // ------------------------------------------------------------------------------------------------
 // One matrix-vector product with its fused prologue (gather / RMSNorm) and epilogue.
 // ------------------------------------------------------------------------------------------------
-__device__ __noinline__ bool gemv_op(Ctx& c, int kind, int l) {
+template <int WDL>
+__device__ __forceinline__ bool gemv_op(Ctx& c, int kind, int l) {
   const KParams& p = c.p;
   const OpShape d = p.shape[kind];
   const int op_idx = (kind == OP_LMHEAD) ? 4 * p.L : 4 * l + kind;
@@ -477,9 +518,14 @@ __device__ __noinline__ bool gemv_op(Ctx& c, int kind, int l) {
 
   if (!from_embed && !wait_phase(c, src_task)) return false;
   if (np > 0) {
-    if (!load_input(c, d.wdtype, K, src, from_embed ? 1u : seq_of(p, src_task), src_task,
-                    from_embed ? embed_row : nullptr, normw, task))
-      return false;
+    const unsigned in_seq = from_embed ? 1u : seq_of(p, src_task);
+    const unsigned short* erow = from_embed ? embed_row : nullptr;
+    const LoadResult lr = (WDL == W_BF16 || kind == OP_LMHEAD)
+                              ? load_input<W_BF16>(p, c.sh, c.xs, c.cta, K, src, in_seq, src_task, erow, normw, task)
+                              : load_input<WDL>(p, c.sh, c.xs, c.cta, K, src, in_seq, src_task, erow, normw, task);
+    c.xscale = lr.xscale;
+    c.bad = lr.bad;
+    if (c.bad) return false;
   }
   if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_LOADED);
 
@@ -501,9 +547,9 @@ __device__ __noinline__ bool gemv_op(Ctx& c, int kind, int l) {
       const int vrow = vrow0 + c.tid;
       if (kind == OP_O) {
         resid = first_layer ? bf16_lo((unsigned)__ldg(embed_row + vrow))
-                            : read_act(c, p.x_a + vrow, seq_of(p, 5 * (l - 1) + 4), 5 * (l - 1) + 4);
+                            : read_act(p, c.bad, p.x_a + vrow, seq_of(p, 5 * (l - 1) + 4), 5 * (l - 1) + 4);
       } else if (kind == OP_DOWN) {
-        resid = read_act(c, p.x_b + vrow, seq_of(p, 5 * l + 2), 5 * l + 2);
+        resid = read_act(p, c.bad, p.x_b + vrow, seq_of(p, 5 * l + 2), 5 * l + 2);
       }
       if (d.wdtype == W_INT8) {
         const __half* scales = reinterpret_cast<const __half*>(
@@ -518,9 +564,9 @@ __device__ __noinline__ bool gemv_op(Ctx& c, int kind, int l) {
       if (d.wdtype != W_BF16) { sc0 *= c.xscale; sc1 *= c.xscale; }
     }
 
-    if (d.wdtype == W_BF16) consume_pass<W_BF16>(c, g, K, red);
-    else if (d.wdtype == W_INT8) consume_pass<W_INT8>(c, g, K, red);
-    else consume_pass<W_INT4>(c, g, K, red);
+    if (WDL == W_BF16 || kind == OP_LMHEAD) consume_pass<W_BF16>(c, g, K, red);     // the LM head is always bf16
+    else consume_pass<WDL>(c, g, K, red);
+    if (c.tid == 0 && ps == np - 1) stamp(p, c.cta, task, 7);
     c.bad = cons_sync_or(c.bad);
     if (c.bad) return false;
 
@@ -629,11 +675,24 @@ __device__ __noinline__ bool gemv_op(Ctx& c, int kind, int l) {
 // Scores are kept in the log2 domain: q is pre-scaled by log2(e) / sqrt(hd).
 // ------------------------------------------------------------------------------------------------
 template <int HD>
-__device__ __forceinline__ void attn_task(Ctx& c, int l, int g, int ch, int Lc, int C) {
-  const KParams& p = c.p;
+__device__ __noinline__ bool attn_general(const KParams& p, SmemHeader* sh, unsigned char* xs, int cta, int l, int g,
+                                          int ch, int Lc, int C, bool bad_in);
+
+// (Not inlined and called with scalars only: its many accumulators would otherwise push the per-thread
+// state of the task loop out of registers for the whole kernel.)
+template <int HD>
+__device__ __forceinline__ bool attn_task(const KParams& p, SmemHeader* sh, unsigned char* xs, int cta, int l, int g,
+                                       int ch, int Lc, int C, bool bad_in) {
+  struct {
+    const KParams& p;
+    SmemHeader* sh;
+    unsigned char* xs;
+    int tid, warp, lane, cta;
+    bool bad;
+  } c{p, sh, xs, (int)threadIdx.x, (int)(threadIdx.x >> 5), (int)(threadIdx.x & 31), cta, bad_in};
   constexpr int LG = HD / 8;            // lanes per cache position (8 bf16 each)
   constexpr int PPW = 32 / LG;          // positions per warp per step
-  constexpr int U = 4;                  // positions in flight per lane group
+  constexpr int U = 2;                  // positions in flight per lane group
   const int n_rep = p.n_rep, half = HD / 2;
   const int n_pos = p.pos + 1;
   const int j0 = ch * Lc, j1 = min(n_pos, j0 + Lc);
@@ -646,30 +705,78 @@ __device__ __forceinline__ void attn_task(Ctx& c, int l, int g, int ch, int Lc, 
   const unsigned in_seq = seq_of(p, 5 * l), out_seq = seq_of(p, 5 * l + 1);
   const bool drop = (5 * l + 1 == p.drop_phase && c.cta == p.drop_block);
 
-  for (int i = c.tid; i < n_rep * half; i += kConsumerThreads) {
+  // ---- gather q (all heads of the group) and, in the chunk that owns the new position, k and v ----------
+  // items: [0, n_rep*half) = q pairs (head h, dims e and e + half); then k pairs; then v pairs.
+  // Both elements and the rotation are requested before anything is checked, so one round trip serves all.
+  unsigned short* knew = reinterpret_cast<unsigned short*>(wp + (size_t)kConsumerWarps * 4 * (HD + 2));   // [HD] bf16
+  unsigned short* vnew = knew + HD;
+  const int n_items = (n_rep + (owns_new ? 2 : 0)) * half;
+  for (int i = c.tid; i < n_items; i += kConsumerThreads) {
     const int h = i / half, e = i - h * half;
-    const ActPair* q = p.qkv + (size_t)(g * n_rep + h) * HD;
-    const float a = read_act(c, q + e, in_seq, 5 * l), b = read_act(c, q + e + half, in_seq, 5 * l);
+    const ActPair* base = (h < n_rep) ? p.qkv + (size_t)(g * n_rep + h) * HD
+                        : (h == n_rep) ? p.qkv + (size_t)p.nq * HD + (size_t)g * HD
+                                       : p.qkv + (size_t)(p.nq + p.nkv) * HD + (size_t)g * HD;
+    uint2 ra = ld_pair(base + e), rb = ld_pair(base + e + half);
     const float2 cs = __ldg(rope + e);
-    qs[h * HD + e] = (a * cs.x - b * cs.y) * qscale;
-    qs[h * HD + e + half] = (b * cs.x + a * cs.y) * qscale;
-  }
-  if (owns_new) {
-    if (c.tid < half) {
-      const ActPair* k = p.qkv + (size_t)p.nq * HD + (size_t)g * HD;
-      const float a = read_act(c, k + c.tid, in_seq, 5 * l), b = read_act(c, k + c.tid + half, in_seq, 5 * l);
-      const float2 cs = __ldg(rope + c.tid);
+    if (ra.y != in_seq) { ra = poll_pair_slow(p, base + e, in_seq, 5 * l); if (ra.y != in_seq) c.bad = true; }
+    if (rb.y != in_seq) { rb = poll_pair_slow(p, base + e + half, in_seq, 5 * l); if (rb.y != in_seq) c.bad = true; }
+    const float a = __uint_as_float(ra.x), b = __uint_as_float(rb.x);
+    if (h < n_rep) {
+      qs[h * HD + e] = (a * cs.x - b * cs.y) * qscale;
+      qs[h * HD + e + half] = (b * cs.x + a * cs.y) * qscale;
+    } else if (h == n_rep) {
+      const unsigned short k0 = f32_to_bf16_rne(a * cs.x - b * cs.y), k1 = f32_to_bf16_rne(b * cs.x + a * cs.y);
       unsigned short* dst = p.kcache + (kvrow + p.pos) * HD;
-      dst[c.tid] = f32_to_bf16_rne(a * cs.x - b * cs.y);
-      dst[c.tid + half] = f32_to_bf16_rne(b * cs.x + a * cs.y);
-    } else if (c.tid >= 64 && c.tid < 64 + HD) {
-      const int e = c.tid - 64;
-      const ActPair* v = p.qkv + (size_t)(p.nq + p.nkv) * HD + (size_t)g * HD;
-      p.vcache[(kvrow + p.pos) * HD + e] = f32_to_bf16_rne(read_act(c, v + e, in_seq, 5 * l));
+      dst[e] = k0; dst[e + half] = k1;
+      knew[e] = k0; knew[e + half] = k1;
+    } else {
+      const unsigned short v0 = f32_to_bf16_rne(a), v1 = f32_to_bf16_rne(b);
+      unsigned short* dst = p.vcache + (kvrow + p.pos) * HD;
+      dst[e] = v0; dst[e + half] = v1;
+      vnew[e] = v0; vnew[e + half] = v1;
     }
   }
-  c.bad = cons_sync_or(c.bad);           // q in shared memory; the new cache row is visible to this block
+  c.bad = cons_sync_or(c.bad);           // q and the new cache row are in shared memory
   if (c.tid == 0) stamp(p, c.cta, 5 * l + 1, AMK_TR_LOADED);
+  if (c.bad) return true;
+
+  if (C == 1 && n_pos == 1) {
+    // one position: its softmax weight is exactly 1, the output is the cached (rounded) v row
+    if (!drop)
+      for (int i = c.tid; i < n_rep * HD; i += kConsumerThreads) {
+        const int h = i / HD, dd = i - h * HD;
+        st_pair(p.o + (size_t)(g * n_rep + h) * HD + dd, bf16_lo((unsigned)vnew[dd]), out_seq);
+      }
+    return c.bad;
+  }
+  return attn_general<HD>(p, sh, xs, cta, l, g, ch, Lc, C, c.bad);
+}
+
+// The general case (more than one cache position): kept out of line so that the code every task runs at
+// short contexts stays small; everything it needs is passed as scalars or recomputed.
+template <int HD>
+__device__ __noinline__ bool attn_general(const KParams& p, SmemHeader* sh, unsigned char* xs, int cta, int l, int g,
+                                          int ch, int Lc, int C, bool bad_in) {
+  struct {
+    SmemHeader* sh;
+    int tid, warp, lane, cta;
+    bool bad;
+  } c{sh, (int)threadIdx.x, (int)(threadIdx.x >> 5), (int)(threadIdx.x & 31), cta, bad_in};
+  constexpr int LG = HD / 8;            // lanes per cache position (8 bf16 each)
+  constexpr int PPW = 32 / LG;          // positions per warp per step
+  constexpr int U = 2;                  // positions in flight per lane group
+  const int n_rep = p.n_rep;
+  const int n_pos = p.pos + 1;
+  const int j0 = ch * Lc, j1 = min(n_pos, j0 + Lc);
+  const bool owns_new = (j1 == n_pos);
+  float* qs = reinterpret_cast<float*>(xs);            // [n_rep][HD]
+  float* wp = qs + n_rep * HD;                         // [warps][4][HD + 2]
+  unsigned short* knew = reinterpret_cast<unsigned short*>(wp + (size_t)kConsumerWarps * 4 * (HD + 2));
+  unsigned short* vnew = knew + HD;
+  const size_t kvrow = ((size_t)l * p.nkv + g) * p.S;
+  const unsigned out_seq = seq_of(p, 5 * l + 1);
+  const bool drop = (5 * l + 1 == p.drop_phase && cta == p.drop_block);
+  const int j_new = owns_new ? p.pos : -1;           // this position is taken from shared memory
 
   const int n_hb = (n_rep + 3) >> 2;     // blocks of four q heads
   const int wph = kConsumerWarps / n_hb; // warps per head block
@@ -692,8 +799,13 @@ __device__ __forceinline__ void attn_task(Ctx& c, int l, int g, int ch, int Lc, 
 #pragma unroll
       for (int u = 0; u < U; u++) {
         const int j = min(jb + u * stride, j1 - 1);
-        kq[u] = __ldcg(Kb + (size_t)j * LG + dl);
-        vq[u] = __ldcg(Vb + (size_t)j * LG + dl);
+        if (j == j_new) {
+          kq[u] = reinterpret_cast<const uint4*>(knew)[dl];
+          vq[u] = reinterpret_cast<const uint4*>(vnew)[dl];
+        } else {
+          kq[u] = __ldcg(Kb + (size_t)j * LG + dl);
+          vq[u] = __ldcg(Vb + (size_t)j * LG + dl);
+        }
       }
 #pragma unroll
       for (int u = 0; u < U; u++) {
@@ -761,7 +873,7 @@ __device__ __forceinline__ void attn_task(Ctx& c, int l, int g, int ch, int Lc, 
     }
   }
   c.bad = cons_sync_or(c.bad);
-  if (c.bad) return;
+  if (c.bad) return true;
 
   // merge the warps of each head block, in warp order
   for (int i = c.tid; i < n_rep * HD; i += kConsumerThreads) {
@@ -785,7 +897,7 @@ __device__ __forceinline__ void attn_task(Ctx& c, int l, int g, int ch, int Lc, 
       if (dd == 0) { pt[0] = M; pt[1] = Z; }
     }
   }
-  if (C == 1) return;
+  if (C == 1) return c.bad;
 
   // several chunks: the chunk that arrives last for this kv group combines all of them
   c.bad = cons_sync_or(c.bad);
@@ -814,9 +926,11 @@ __device__ __forceinline__ void attn_task(Ctx& c, int l, int g, int ch, int Lc, 
     }
     if (c.tid == 0) *gctr = 0u;          // next used by the next launch
   }
+  return c.bad;
 }
 
-__device__ __noinline__ bool attention_phase(Ctx& c, int l) {
+template <int HD>
+__device__ __forceinline__ bool attention_phase(Ctx& c, int l) {
   const KParams& p = c.p;
   int Lc, C;
   attn_chunks(p.pos + 1, c.nblk, p.nkv, &Lc, &C);
@@ -830,8 +944,7 @@ __device__ __noinline__ bool attention_phase(Ctx& c, int l) {
   if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_JOINED);
   if (t < n_tasks) {
     const int g = t / C, ch = t - g * C;
-    if (p.hd == 64) attn_task<64>(c, l, g, ch, Lc, C);
-    else attn_task<128>(c, l, g, ch, Lc, C);
+    c.bad = attn_task<HD>(p, c.sh, c.xs, c.cta, l, g, ch, Lc, C, c.bad);
   }
   c.bad = cons_sync_or(c.bad);
   if (c.bad) return false;
@@ -849,19 +962,30 @@ __device__ __noinline__ void producer(const KParams& p, SmemHeader* sh, unsigned
   const uint64_t pol = policy_evict_first();
   const unsigned S = (unsigned)p.n_stages;
   const unsigned inflight = (unsigned)p.max_inflight;
+  const unsigned ahead = (unsigned)p.l2_ahead;      // tiles kept requested into L2 beyond the ring (<= 32)
   const unsigned begin = __ldg(p.tile_begin + cta), end = __ldg(p.tile_begin + cta + 1);
   unsigned t = 0;                                   // tiles issued so far
   unsigned stage = 0, lap = 0;
   int cur_task = -1;
   int ok = 1;
-  unsigned long long e_next = (begin + lane < end) ? __ldg(p.tiles + begin + lane) : 0ull;
+  // the warp holds 64 consecutive table entries: [base, base + 32) in e_cur, [base + 32, base + 64) in e_next
+  unsigned long long e_cur = (begin + lane < end) ? __ldg(p.tiles + begin + lane) : 0ull;
+  unsigned long long e_next = (begin + 32 + lane < end) ? __ldg(p.tiles + begin + 32 + lane) : 0ull;
+  // the first `ahead` tiles are requested right away
+  for (unsigned j = 0; j < ahead && begin + j < end; j++) {
+    const unsigned long long e = __shfl_sync(0xffffffffu, e_cur, (int)j);
+    if (lane == 0) bulk_prefetch_l2(p.packed + ((e & ((1ull << 40) - 1)) << 4), (unsigned)((e >> 40) & 0x1fffu) << 4);
+  }
   for (unsigned base = begin; base < end && ok; base += 32) {
-    const unsigned long long e_cur = e_next;
-    if (base + 32 + lane < end) e_next = __ldg(p.tiles + base + 32 + lane);
     const int n = (int)min(32u, end - base);
     for (int j = 0; j < n; j++) {
       const unsigned long long e = __shfl_sync(0xffffffffu, e_cur, j);
+      // the tile `ahead` places further on: request it into L2 now
+      const int ja = j + (int)ahead;
+      const unsigned long long ea = __shfl_sync(0xffffffffu, ja < 32 ? e_cur : e_next, ja & 31);
       if (lane == 0) {
+        if (ahead && base + (unsigned)ja < end)
+          bulk_prefetch_l2(p.packed + ((ea & ((1ull << 40) - 1)) << 4), (unsigned)((ea >> 40) & 0x1fffu) << 4);
         const unsigned long long off = (e & ((1ull << 40) - 1)) << 4;
         const unsigned bytes = (unsigned)((e >> 40) & 0x1fffu) << 4;
         const int task = (int)(e >> 53);
@@ -884,6 +1008,8 @@ __device__ __noinline__ void producer(const KParams& p, SmemHeader* sh, unsigned
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
     }
+    e_cur = e_next;
+    e_next = (base + 64 + lane < end) ? __ldg(p.tiles + base + 64 + lane) : 0ull;
   }
   if (!ok && lane == 0) {
     // leaving early: every copy already issued must land before the block's shared memory is released
@@ -898,6 +1024,9 @@ __device__ __noinline__ void producer(const KParams& p, SmemHeader* sh, unsigned
 
 }  // namespace
 
+// One instantiation per (layer weight dtype, head dimension): only the code a model needs is resident,
+// which matters because every task runs its code once and instruction-cache misses cost like L2 misses.
+template <int WDL, int HD>
 __global__ void __launch_bounds__(kThreads, 1) amk_decode_kernel(const __grid_constant__ KParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   SmemHeader* sh = reinterpret_cast<SmemHeader*>(smem);
@@ -925,27 +1054,41 @@ __global__ void __launch_bounds__(kThreads, 1) amk_decode_kernel(const __grid_co
   int token = p.token_ptr ? __ldcg(p.token_ptr) : p.token;
   token = min(max(token, 0), p.V - 1);
   Ctx c{p, sh, xs, ring, tid, warp, lane, cta, nblk, 0, 0u, token, 1.0f, false};
-  bool ok = true;
-  for (int l = 0; l < p.L && ok; l++) {
-    ok = gemv_op(c, OP_QKV, l);
-    ok = ok && attention_phase(c, l);
-    ok = ok && gemv_op(c, OP_O, l);
-    ok = ok && gemv_op(c, OP_GATEUP, l);
-    ok = ok && gemv_op(c, OP_DOWN, l);
+  // the block's queue: tasks 5 l + {0..4} = QKV, attention, O, gate/up, down of layer l, then the LM head
+  // (one call site each, so that the per-thread state stays in registers)
+  const int n_tasks = 5 * p.L + 1;
+  for (int task = 0; task < n_tasks; task++) {
+    const int l = task / 5, k = task - 5 * l;
+    bool ok;
+    if (k == 1) ok = attention_phase<HD>(c, l);
+    else ok = gemv_op<WDL>(c, task == n_tasks - 1 ? (int)OP_LMHEAD : (k == 0 ? (int)OP_QKV : k - 1), l);
+    if (!ok) break;
   }
-  if (ok) gemv_op(c, OP_LMHEAD, p.L);
 }
 
-cudaError_t decode_kernel_attrs(size_t smem_bytes, int* max_blocks_per_sm) {
-  cudaError_t e = cudaFuncSetAttribute(amk_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+typedef void (*DecodeKernel)(const KParams);
+static DecodeKernel pick_kernel(int wdtype, int hd) {
+  if (hd == 64) {
+    if (wdtype == W_BF16) return amk_decode_kernel<W_BF16, 64>;
+    if (wdtype == W_INT8) return amk_decode_kernel<W_INT8, 64>;
+    return amk_decode_kernel<W_INT4, 64>;
+  }
+  if (wdtype == W_BF16) return amk_decode_kernel<W_BF16, 128>;
+  if (wdtype == W_INT8) return amk_decode_kernel<W_INT8, 128>;
+  return amk_decode_kernel<W_INT4, 128>;
+}
+
+cudaError_t decode_kernel_attrs(int wdtype, int hd, size_t smem_bytes, int* max_blocks_per_sm) {
+  DecodeKernel k = pick_kernel(wdtype, hd);
+  cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
   if (e != cudaSuccess) return e;
-  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(max_blocks_per_sm, amk_decode_kernel, kThreads, smem_bytes);
+  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(max_blocks_per_sm, k, kThreads, smem_bytes);
 }
 
 cudaError_t launch_decode(const KParams& p, int n_blocks, size_t smem_bytes, cudaStream_t stream) {
   void* args[] = {const_cast<KParams*>(&p)};
-  return cudaLaunchCooperativeKernel((const void*)amk_decode_kernel, dim3(n_blocks), dim3(kThreads), args, smem_bytes,
-                                     stream);
+  return cudaLaunchCooperativeKernel((const void*)pick_kernel(p.shape[OP_QKV].wdtype, p.hd), dim3(n_blocks),
+                                     dim3(kThreads), args, smem_bytes, stream);
 }
 
 }  // namespace amk

@@ -27,7 +27,7 @@
 
 namespace amk {
 
-constexpr int kConsumerWarps = 15;            // consumer warps per block (+1 producer warp = 512 threads)
+constexpr int kConsumerWarps = 11;            // consumer warps per block (+1 producer warp = 384 threads, 168 registers each)
 constexpr int kThreads = 32 * (kConsumerWarps + 1);
 constexpr int kConsumerThreads = 32 * kConsumerWarps;
 constexpr int kGMax = 16;                     // rows per row-warp: one m16n8 tile
