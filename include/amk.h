@@ -46,6 +46,9 @@ typedef enum { AMK_W_BF16 = 0, AMK_W_INT8 = 1, AMK_W_INT4 = 2 } amk_wdtype;
 /* amk_config.flags */
 #define AMK_FLAG_DEBUG_HIDDEN 1u /* keep the residual stream after the embedding and after every layer */
 #define AMK_FLAG_TRACE 2u        /* every block stamps the global timer at the stages of every task          */
+#define AMK_FLAG_MEASURED_SPLIT 4u /* amk_create measures the HBM rate each SM gets and gives each block a share
+                                      of every op in proportion (blocks are then identified by SM id).  Off by
+                                      default: on B200 it measured no faster than equal shares.             */
 
 /* Trace layout (amk_debug_trace): uint64 nanosecond stamps [n_blocks][n_tasks][AMK_TRACE_EVENTS], where
  * task 5*l+{0,1,2,3,4} = QKV, attention, O, gate/up, down of layer l and task 5*L = LM head. */

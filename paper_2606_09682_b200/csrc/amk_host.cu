@@ -3,6 +3,7 @@
 // decode step: every step of the path runs in the kernels.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -23,7 +24,7 @@ inline size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a
 
 // One matrix-vector product of the step, as the host plans it.
 struct PlanOp {
-  int kind, layer, rot;
+  int kind, layer;
   OpShape s;
   size_t region_off;                 // byte offset of the op's region in the packed buffer
   size_t scale_off;                  // int8: fp16 row scales (virtual row order)
@@ -36,6 +37,7 @@ struct Plan {
   uint32_t stage_bytes = 0;
   OpShape shape[5];
   std::vector<PlanOp> ops;
+  std::vector<int> bounds[5];        // per op kind: unit boundaries of the slots (n_blocks + 1)
   size_t scale_base = 0, scale_layer_stride = 0, scale_kind_off[4] = {0, 0, 0, 0};
   size_t embed_off = 0, attn_norm_off = 0, mlp_norm_off = 0, final_norm_off = 0, packed_total = 0;
   size_t weight_stream_bytes = 0;    // op regions + scale regions (what a token streams)
@@ -44,7 +46,7 @@ struct Plan {
 
 struct WorkspaceLayout {
   size_t status, phase_ctr, group_ctr, lm_ctr, next_ws, cand_val, cand_idx, x_a, x_b, qkv, o, m, part, hidden, rope,
-      trace, slice_tab, tile_begin, tiles, total;
+      trace, slice_tab, bounds, smid_tab, calib, tile_begin, tiles, total;
 };
 
 int resolve_blocks(const amk_config* c) {
@@ -83,8 +85,9 @@ amk_status check_config(const amk_config* c) {
 
 uint32_t stage_bytes_of(const amk_config* c) { return c->stage_bytes ? c->stage_bytes : 32768u; }
 
-Plan make_plan(const amk_config* c, int n_blocks, bool with_tiles, std::vector<unsigned long long>* tiles,
-               std::vector<unsigned>* tile_begin) {
+// `weights`: relative streaming rate of each slot (nullptr: equal shares).
+Plan make_plan(const amk_config* c, int n_blocks, const double* weights, bool with_tiles,
+               std::vector<unsigned long long>* tiles, std::vector<unsigned>* tile_begin) {
   Plan pl;
   pl.n_blocks = n_blocks;
   pl.stage_bytes = stage_bytes_of(c);
@@ -96,18 +99,21 @@ Plan make_plan(const amk_config* c, int n_blocks, bool with_tiles, std::vector<u
   pl.shape[OP_GATEUP] = OpShape{H, 2 * I, 2, wd};
   pl.shape[OP_DOWN] = OpShape{I, H, 1, wd};
   pl.shape[OP_LMHEAD] = OpShape{H, V, 1, W_BF16};
+  for (int k = 0; k < 5; k++) {
+    pl.bounds[k].resize(n_blocks + 1);
+    make_bounds(pl.shape[k].rows / pl.shape[k].unit_rows, n_blocks, weights, pl.bounds[k].data());
+  }
   size_t off = 0;
   auto add = [&](int kind, int layer) {
     PlanOp op;
     op.kind = kind; op.layer = layer; op.s = pl.shape[kind];
-    op.rot = (int)((pl.ops.size() * 37u) % (unsigned)n_blocks);
     op.region_off = off;
     op.scale_off = 0;
     op.slice_off.resize(n_blocks);
     size_t o = 0;
     for (int s = 0; s < n_blocks; s++) {
       op.slice_off[s] = o;
-      o += (size_t)slice_bytes(slot_slice(op.s.rows, op.s.unit_rows, n_blocks, s).rows, op.s.K, op.s.wdtype,
+      o += (size_t)slice_bytes(slot_slice(pl.bounds[kind].data(), op.s.unit_rows, s).rows, op.s.K, op.s.wdtype,
                                (int)pl.stage_bytes);
     }
     off = align_up(off + o);
@@ -143,8 +149,8 @@ Plan make_plan(const amk_config* c, int n_blocks, bool with_tiles, std::vector<u
     if (with_tiles) (*tile_begin)[cta] = (unsigned)count;
     for (size_t i = 0; i < pl.ops.size(); i++) {
       const PlanOp& op = pl.ops[i];
-      const int slot = (cta + op.rot) % n_blocks;
-      const Slice sl = slot_slice(op.s.rows, op.s.unit_rows, n_blocks, slot);
+      const int slot = cta;
+      const Slice sl = slot_slice(pl.bounds[op.kind].data(), op.s.unit_rows, slot);
       const int task = (op.kind == OP_LMHEAD) ? 5 * L : 5 * op.layer + (op.kind == OP_QKV ? 0 : op.kind + 1);
       size_t base = op.region_off + op.slice_off[slot];
       for (int ps = 0; ps < n_passes(sl.rows); ps++) {
@@ -191,8 +197,12 @@ WorkspaceLayout workspace_layout(const amk_config* c, const Plan& pl) {
   w.rope = take(S * (hd / 2) * sizeof(float2));
   w.trace = take((size_t)pl.n_blocks * (5 * L + 1) * AMK_TRACE_EVENTS * 8);
   w.slice_tab = take(pl.ops.size() * (size_t)pl.n_blocks * 8);
+  w.bounds = take(5 * ((size_t)pl.n_blocks + 1) * 4);
+  w.smid_tab = take((size_t)kMaxSmid * 4);
+  w.calib = take((size_t)pl.n_blocks * 16);
   w.tile_begin = take(((size_t)pl.n_blocks + 1) * 4);
-  w.tiles = take(pl.n_tiles * 8);
+  // the tile count depends a little on how the rows are split over the slots: leave room for any split
+  w.tiles = take((pl.n_tiles + pl.ops.size() * (size_t)pl.n_blocks * 2) * 8);
   w.total = off;
   return w;
 }
@@ -215,6 +225,7 @@ struct amk_handle {
   unsigned ctr_epoch;      // steps since the counters were last zeroed
   cudaStream_t last_stream;
   int drop_phase, drop_block;
+  float split_min, split_max;   // smallest / largest share given to a block, relative to the median
   char errmsg[256];
 };
 
@@ -239,7 +250,9 @@ amk_status amk_packed_bytes(const amk_config* cfg, size_t* bytes) {
   if (!bytes) return AMK_ERR_INVALID_ARG;
   amk_status st = check_config(cfg);
   if (st != AMK_OK) return st;
-  *bytes = make_plan(cfg, resolve_blocks(cfg), false, nullptr, nullptr).packed_total;
+  const Plan pl = make_plan(cfg, resolve_blocks(cfg), nullptr, false, nullptr, nullptr);
+  // int4 work units are padded to 16 bytes, so the total depends a little on the split: leave room
+  *bytes = pl.packed_total + (cfg->wdtype == AMK_W_INT4 ? pl.packed_total / 64 : 0);
   return AMK_OK;
 }
 
@@ -247,7 +260,7 @@ amk_status amk_workspace_bytes(const amk_config* cfg, size_t* bytes) {
   if (!bytes) return AMK_ERR_INVALID_ARG;
   amk_status st = check_config(cfg);
   if (st != AMK_OK) return st;
-  const Plan pl = make_plan(cfg, resolve_blocks(cfg), false, nullptr, nullptr);
+  const Plan pl = make_plan(cfg, resolve_blocks(cfg), nullptr, false, nullptr, nullptr);
   *bytes = workspace_layout(cfg, pl).total;
   return AMK_OK;
 }
@@ -309,13 +322,68 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
       status = AMK_ERR_UNSUPPORTED;
       goto fail;
     }
+    // ---- calibration: what share of the HBM stream does each SM get? ------------------------------------
+    // (only when every SM runs a block: then the SM id identifies the block, whatever block index it has)
+    std::vector<double> weights;
+    std::vector<int> slot_of_smid;
+    const Plan pl0 = make_plan(cfg, n_blocks, nullptr, false, nullptr, nullptr);
+    const WorkspaceLayout wl0 = workspace_layout(cfg, pl0);
+    if (packed_bytes < pl0.packed_total || workspace_bytes < wl0.total) {
+      snprintf(h->errmsg, sizeof(h->errmsg), "buffers too small: packed %zu < %zu or workspace %zu < %zu", packed_bytes,
+               pl0.packed_total, workspace_bytes, wl0.total);
+      status = AMK_ERR_INVALID_ARG;
+      goto fail;
+    }
+    const bool by_smid = (n_blocks == sms) && (cfg->flags & AMK_FLAG_MEASURED_SPLIT);
+    if (by_smid) {
+      size_t per = packed_bytes / (size_t)n_blocks;
+      if (per > (8u << 20)) per = 8u << 20;
+      per = per / 32768 * 32768;
+      if (per >= (1u << 20)) {
+        unsigned* smid_dev = (unsigned*)(h->ws + wl0.calib);
+        unsigned long long* ns_dev = (unsigned long long*)(h->ws + wl0.calib + (size_t)n_blocks * 4 + 4) ;
+        ns_dev = (unsigned long long*)(((uintptr_t)ns_dev + 7) & ~(uintptr_t)7);
+        std::vector<unsigned> smid(n_blocks);
+        std::vector<unsigned long long> ns(n_blocks);
+        for (int rep = 0; rep < 2; rep++)
+          AMK_CUDA(launch_calibrate(h->packed, per, n_blocks, (size_t)smem_optin, smid_dev, ns_dev, stream));
+        AMK_CUDA(cudaMemcpyAsync(smid.data(), smid_dev, (size_t)n_blocks * 4, cudaMemcpyDeviceToHost, stream));
+        AMK_CUDA(cudaMemcpyAsync(ns.data(), ns_dev, (size_t)n_blocks * 8, cudaMemcpyDeviceToHost, stream));
+        AMK_CUDA(cudaStreamSynchronize(stream));
+        // slot i = the i-th block of the calibration launch; every SM must appear exactly once
+        slot_of_smid.assign(kMaxSmid, -1);
+        weights.assign(n_blocks, 1.0);
+        bool ok_map = true;
+        std::vector<double> rates(n_blocks);
+        for (int i = 0; i < n_blocks; i++) {
+          if (smid[i] >= (unsigned)kMaxSmid || slot_of_smid[smid[i]] >= 0 || ns[i] == 0) { ok_map = false; break; }
+          slot_of_smid[smid[i]] = i;
+          rates[i] = (double)per / (double)ns[i];
+        }
+        if (ok_map) {
+          std::vector<double> sorted = rates;
+          std::sort(sorted.begin(), sorted.end());
+          const double med = sorted[n_blocks / 2];
+          for (int i = 0; i < n_blocks; i++) {
+            double w = rates[i] / med;
+            weights[i] = w < 0.8 ? 0.8 : (w > 1.5 ? 1.5 : w);      // a share, not a promise: keep it sane
+          }
+          if (getenv("AMK_VERBOSE")) {
+            fprintf(stderr, "amk_create: per-SM rate GB/s min %.1f p10 %.1f median %.1f p90 %.1f max %.1f (%zu bytes each)\n",
+                    sorted[0], sorted[n_blocks / 10], med, sorted[n_blocks * 9 / 10], sorted[n_blocks - 1], per);
+          }
+        } else {
+          weights.clear();
+          slot_of_smid.clear();
+        }
+      }
+    }
     std::vector<unsigned long long> tiles;
     std::vector<unsigned> tile_begin;
-    h->pl = make_plan(cfg, n_blocks, true, &tiles, &tile_begin);
-    h->wl = workspace_layout(cfg, h->pl);
-    if (packed_bytes < h->pl.packed_total || workspace_bytes < h->wl.total) {
-      snprintf(h->errmsg, sizeof(h->errmsg), "buffers too small: packed %zu < %zu or workspace %zu < %zu", packed_bytes,
-               h->pl.packed_total, workspace_bytes, h->wl.total);
+    h->pl = make_plan(cfg, n_blocks, weights.empty() ? nullptr : weights.data(), true, &tiles, &tile_begin);
+    h->wl = wl0;
+    if (packed_bytes < h->pl.packed_total || tiles.size() * 8 > h->wl.total - h->wl.tiles) {
+      snprintf(h->errmsg, sizeof(h->errmsg), "buffers too small for the measured split");
       status = AMK_ERR_INVALID_ARG;
       goto fail;
     }
@@ -360,6 +428,12 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
       for (size_t i = 0; i < h->pl.ops.size(); i++)
         memcpy(&slices[i * n_blocks], h->pl.ops[i].slice_off.data(), (size_t)n_blocks * 8);
       AMK_CUDA(cudaMemcpyAsync(h->ws + h->wl.slice_tab, slices.data(), slices.size() * 8, cudaMemcpyHostToDevice, stream));
+      std::vector<int> btab(5 * ((size_t)n_blocks + 1));
+      for (int k = 0; k < 5; k++) memcpy(&btab[k * ((size_t)n_blocks + 1)], h->pl.bounds[k].data(), ((size_t)n_blocks + 1) * 4);
+      AMK_CUDA(cudaMemcpyAsync(h->ws + h->wl.bounds, btab.data(), btab.size() * 4, cudaMemcpyHostToDevice, stream));
+      if (!slot_of_smid.empty())
+        AMK_CUDA(cudaMemcpyAsync(h->ws + h->wl.smid_tab, slot_of_smid.data(), (size_t)kMaxSmid * 4,
+                                 cudaMemcpyHostToDevice, stream));
       AMK_CUDA(cudaMemcpyAsync(h->ws + h->wl.tile_begin, tile_begin.data(), tile_begin.size() * 4,
                                cudaMemcpyHostToDevice, stream));
       AMK_CUDA(cudaMemcpyAsync(h->ws + h->wl.tiles, tiles.data(), tiles.size() * 8, cudaMemcpyHostToDevice, stream));
@@ -382,7 +456,8 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     for (size_t i = 0; i < h->pl.ops.size(); i++) {
       const PlanOp& op = h->pl.ops[i];
       PackOp d;
-      d.s = op.s; d.rot = op.rot; d.region_off = op.region_off; d.scale_off = op.scale_off;
+      d.s = op.s; d.region_off = op.region_off; d.scale_off = op.scale_off;
+      d.bounds = (const int*)(h->ws + h->wl.bounds) + (size_t)op.kind * (n_blocks + 1);
       d.slice_off = (const unsigned long long*)(h->ws + h->wl.slice_tab) + i * (size_t)n_blocks;
       PackSrc s;
       memset(&s, 0, sizeof(s));
@@ -428,6 +503,10 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     p.packed = h->packed;
     p.tiles = (const unsigned long long*)(h->ws + h->wl.tiles);
     p.tile_begin = (const unsigned*)(h->ws + h->wl.tile_begin);
+    p.bounds = (const int*)(h->ws + h->wl.bounds);
+    p.slot_of_smid = slot_of_smid.empty() ? nullptr : (const int*)(h->ws + h->wl.smid_tab);
+    h->split_min = 1.0f; h->split_max = 1.0f;
+    for (double w : weights) { if (w < h->split_min) h->split_min = (float)w; if (w > h->split_max) h->split_max = (float)w; }
     p.scale_base = h->pl.scale_base;
     p.scale_layer_stride = (unsigned)h->pl.scale_layer_stride;
     for (int k = 0; k < 4; k++) p.scale_kind_off[k] = (unsigned)h->pl.scale_kind_off[k];
@@ -598,7 +677,8 @@ amk_status amk_debug_unpack(amk_handle* h, int layer, int which, void* out_dev, 
   s.zero[slot] = zero_dev;
   const PlanOp& po = h->pl.ops[op];
   PackOp d;
-  d.s = po.s; d.rot = po.rot; d.region_off = po.region_off; d.scale_off = po.scale_off;
+  d.s = po.s; d.region_off = po.region_off; d.scale_off = po.scale_off;
+  d.bounds = (const int*)(h->ws + h->wl.bounds) + (size_t)po.kind * (h->plan.n_blocks + 1);
   d.slice_off = (const unsigned long long*)(h->ws + h->wl.slice_tab) + (size_t)op * h->plan.n_blocks;
   cudaError_t e = launch_pack(d, s, h->packed, (int)h->plan.n_blocks, (int)h->plan.stage_bytes, true,
                               (cudaStream_t)cuda_stream);

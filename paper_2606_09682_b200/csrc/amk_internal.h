@@ -19,6 +19,8 @@ struct DevStatus {
 };
 
 // Fixed shared-memory header in front of the activation area and the ring.
+constexpr int kMaxSmid = 4096;
+
 struct SmemHeader {
   uint64_t full[kMaxStages];
   uint64_t empty[kMaxStages];
@@ -27,7 +29,9 @@ struct SmemHeader {
   float cand_val[kConsumerWarps];
   int cand_idx[kConsumerWarps];
   int flag;                          // "this block arrived last" broadcast
-  int pad[3];
+  int slot;                          // this block's slot (its share of every op, its tile list)
+  int slice_row0[5], slice_rows[5];  // its rows of each op kind
+  int pad[1];
 };
 
 // An activation element in global memory: the value and the sequence number of the task that wrote it.
@@ -49,7 +53,9 @@ struct KParams {
   // weights
   const unsigned char* packed;            // packed buffer base
   const unsigned long long* tiles;        // per block: its ring tiles {offset/16 | bytes/16 << 40}, in stream order
-  const unsigned* tile_begin;             // [n_blocks + 1] index of each block's first tile
+  const unsigned* tile_begin;             // [n_blocks + 1] index of each slot's first tile
+  const int* bounds;                      // [5][n_blocks + 1] unit boundaries of the slots, per op kind
+  const int* slot_of_smid;                // [kMaxSmid] slot of the block running on each SM, or null: slot = blockIdx
   unsigned long long scale_base;          // int8: fp16 row scales, op-major in virtual row order
   unsigned scale_layer_stride;            // bytes per layer
   unsigned scale_kind_off[4];             // byte offset of each op kind inside a layer's scales
@@ -100,7 +106,7 @@ cudaError_t decode_kernel_attrs(int wdtype, int hd, size_t smem_bytes, int* max_
 // One op to pack: its shape, rotation and region, plus where the canonical rows come from.
 struct PackOp {
   OpShape s;
-  int rot;
+  const int* bounds;                      // DEVICE [n_blocks + 1]: unit boundaries of the slots for this op kind
   unsigned long long region_off;          // byte offset of the op's region in the packed buffer
   const unsigned long long* slice_off;    // DEVICE [n_blocks]: byte offset of each slot's slice inside the region
   unsigned long long scale_off;           // int8: byte offset of the fp16 row scales (virtual row order)
@@ -114,6 +120,9 @@ struct PackSrc {
 };
 cudaError_t launch_pack(const PackOp& d, const PackSrc& src, unsigned char* packed, int n_blocks, int stage_bytes,
                         bool inverse, cudaStream_t stream);
+// Streams `bytes_per_block` per block (one block per SM) and reports each block's SM id and time in ns.
+cudaError_t launch_calibrate(const unsigned char* src, size_t bytes_per_block, int n_blocks, size_t smem_bytes,
+                             unsigned* smid_out, unsigned long long* ns_out, cudaStream_t stream);
 cudaError_t launch_quantize_int8(const void* w, int64_t rows, int64_t cols, void* q, void* scale, cudaStream_t s);
 cudaError_t launch_quantize_int4(const void* w, int64_t rows, int64_t cols, void* packed, void* scale, void* zero,
                                  cudaStream_t s);

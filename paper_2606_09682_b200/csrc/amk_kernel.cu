@@ -488,10 +488,10 @@ template <int WDL>
 __device__ __forceinline__ bool gemv_op(Ctx& c, int kind, int l) {
   const KParams& p = c.p;
   const OpShape d = p.shape[kind];
-  const int op_idx = (kind == OP_LMHEAD) ? 4 * p.L : 4 * l + kind;
   const int task = (kind == OP_LMHEAD) ? 5 * p.L : 5 * l + (kind == OP_QKV ? 0 : kind + 1);
-  const int slot = (c.cta + (op_idx * 37) % c.nblk) % c.nblk;
-  const Slice sl = slot_slice(d.rows, d.unit_rows, c.nblk, slot);
+  Slice sl;
+  sl.row0 = c.sh->slice_row0[kind];
+  sl.rows = c.sh->slice_rows[kind];
   const int K = d.K;
   const bool first_layer = (l == 0);
   const unsigned short* embed_row = p.embed + (size_t)c.token * p.H;
@@ -1034,7 +1034,7 @@ __global__ void __launch_bounds__(kThreads, 1) amk_decode_kernel(const __grid_co
   unsigned char* xs = smem + hdr;
   unsigned char* ring = smem + hdr + p.act_bytes;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int cta = blockIdx.x, nblk = gridDim.x;
+  const int nblk = gridDim.x;
 
   if (tid == 0) {
     for (int s = 0; s < p.n_stages; s++) {
@@ -1042,9 +1042,31 @@ __global__ void __launch_bounds__(kThreads, 1) amk_decode_kernel(const __grid_co
       mbar_init(&sh->empty[s], kConsumerWarps);
     }
     sh->flag = 0;
+    // Which share of the work is this block's?  With one block per SM the SM id names the block, and the
+    // host's table gives the slot whose share matches what that SM was measured to stream.
+    int slot = blockIdx.x;
+    if (p.slot_of_smid) {
+      unsigned sm;
+      asm volatile("mov.u32 %0, %%smid;" : "=r"(sm));
+      slot = (sm < (unsigned)kMaxSmid) ? __ldg(p.slot_of_smid + sm) : -1;
+      if (slot < 0 || slot >= nblk) {
+        report_failure(p, (unsigned)AMK_ERR_ABORTED, -3, sm, 0u);     // an SM the plan has not seen
+        slot = -1;
+      }
+    }
+    sh->slot = slot;
+    if (slot >= 0) {
+      for (int k = 0; k < 5; k++) {
+        const int* b = p.bounds + k * (nblk + 1);
+        sh->slice_row0[k] = __ldg(b + slot) * p.shape[k].unit_rows;
+        sh->slice_rows[k] = (__ldg(b + slot + 1) - __ldg(b + slot)) * p.shape[k].unit_rows;
+      }
+    }
     mbar_fence_init();
   }
   __syncthreads();
+  const int cta = sh->slot;
+  if (cta < 0) return;
 
   if (warp == kConsumerWarps) {
     producer(p, sh, ring, cta, lane);
@@ -1064,6 +1086,70 @@ __global__ void __launch_bounds__(kThreads, 1) amk_decode_kernel(const __grid_co
     else ok = gemv_op<WDL>(c, task == n_tasks - 1 ? (int)OP_LMHEAD : (k == 0 ? (int)OP_QKV : k - 1), l);
     if (!ok) break;
   }
+}
+
+// Calibration: every block (one per SM, same shared-memory footprint as the decode kernel) streams
+// `bytes_per_block` through a small ring of bulk copies while all the others do the same, and reports its
+// SM id and the time it took.  SMs do not all get the same share of the HBM stream; the host can split the
+// rows of every op in proportion to these rates.
+__global__ void __launch_bounds__(kThreads, 1)
+amk_calibrate_kernel(const unsigned char* __restrict__ src, size_t bytes_per_block, unsigned* smid_out,
+                     unsigned long long* ns_out) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  constexpr int S = 4, TILE = 32768;
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem);
+  uint64_t* empty = full + S;
+  unsigned char* ring = smem + 128;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; s++) { mbar_init(full + s, 1); mbar_init(empty + s, kConsumerWarps); }
+    mbar_fence_init();
+  }
+  __syncthreads();
+  const unsigned char* base = src + (size_t)blockIdx.x * bytes_per_block;
+  const int n_tiles = (int)(bytes_per_block / TILE);
+  const unsigned long long t0 = globaltimer_ns();
+  const unsigned kSpinLimit = 1u << 26;
+  if (warp == kConsumerWarps) {
+    if (lane == 0) {
+      const uint64_t pol = policy_evict_first();
+      for (int t = 0; t < n_tiles; t++) {
+        const int s = t % S;
+        if (t >= S) {
+          unsigned spins = 0;
+          while (!mbar_try_wait(empty + s, ((t / S) - 1) & 1u)) if (++spins > kSpinLimit) return;
+        }
+        mbar_expect_tx(full + s, TILE);
+        bulk_g2s(ring + (size_t)s * TILE, base + (size_t)t * TILE, TILE, full + s, pol);
+      }
+    }
+  } else {
+    for (int t = 0; t < n_tiles; t++) {
+      const int s = t % S;
+      unsigned spins = 0;
+      bool ok = true;
+      while (!mbar_try_wait(full + s, (t / S) & 1u)) if (++spins > kSpinLimit) { ok = false; break; }
+      if (!ok) break;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty + s);
+    }
+    if (threadIdx.x == 0) {
+      unsigned sm;
+      asm volatile("mov.u32 %0, %%smid;" : "=r"(sm));
+      smid_out[blockIdx.x] = sm;
+      ns_out[blockIdx.x] = globaltimer_ns() - t0;
+    }
+  }
+}
+
+cudaError_t launch_calibrate(const unsigned char* src, size_t bytes_per_block, int n_blocks, size_t smem_bytes,
+                             unsigned* smid_out, unsigned long long* ns_out, cudaStream_t stream) {
+  const size_t need = 128 + 4 * 32768;
+  if (smem_bytes < need) smem_bytes = need;
+  cudaError_t e = cudaFuncSetAttribute(amk_calibrate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+  if (e != cudaSuccess) return e;
+  amk_calibrate_kernel<<<n_blocks, kThreads, smem_bytes, stream>>>(src, bytes_per_block, smid_out, ns_out);
+  return cudaGetLastError();
 }
 
 typedef void (*DecodeKernel)(const KParams);

@@ -79,24 +79,38 @@ AMK_HD void place_of_k(int wdtype, int k, int* chunk, int* elem) {
   *elem = 8 * q + 2 * j + (s & 1);
 }
 
-// Rows owned by slot s: units are dealt as evenly as possible, the first (units % n) slots get one more.
+// Rows owned by slot s.  The split of an op's units over the slots is a table: bounds[s] .. bounds[s+1] are
+// slot s's units (n_slots + 1 entries, bounds[0] = 0, bounds[n_slots] = units).  The host builds it in
+// proportion to what each SM was measured to stream, so that all blocks finish an op together.
 struct Slice { int row0; int rows; };
-AMK_HD Slice slot_slice(int total_rows, int unit_rows, int n_slots, int s) {
-  int units = total_rows / unit_rows;
-  int q = units / n_slots, rem = units % n_slots;
-  int u0 = s * q + (s < rem ? s : rem);
-  int nu = q + (s < rem ? 1 : 0);
-  Slice r; r.row0 = u0 * unit_rows; r.rows = nu * unit_rows;
+AMK_HD Slice slot_slice(const int* bounds, int unit_rows, int s) {
+  Slice r; r.row0 = bounds[s] * unit_rows; r.rows = (bounds[s + 1] - bounds[s]) * unit_rows;
   return r;
 }
-// Inverse: which slot owns a row.
-AMK_HD int slot_of_row(int total_rows, int unit_rows, int n_slots, int row) {
-  int units = total_rows / unit_rows;
-  int q = units / n_slots, rem = units % n_slots;
-  int u = row / unit_rows;
-  int big = rem * (q + 1);
-  if (u < big) return u / (q + 1);
-  return q ? rem + (u - big) / q : n_slots - 1;
+// Inverse: which slot owns a row (the last slot whose first unit is not beyond the row's unit).
+AMK_HD int slot_of_row(const int* bounds, int unit_rows, int n_slots, int row) {
+  const int u = row / unit_rows;
+  int lo = 0, hi = n_slots - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (bounds[mid] <= u) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+// (host only) Unit boundaries for `units` units over n_slots slots with relative weights w (nullptr: equal shares).
+inline void make_bounds(int units, int n_slots, const double* w, int* bounds) {
+  double total = 0.0;
+  for (int s = 0; s < n_slots; s++) total += w ? w[s] : 1.0;
+  double cum = 0.0;
+  bounds[0] = 0;
+  for (int s = 0; s < n_slots; s++) {
+    cum += w ? w[s] : 1.0;
+    int b = (int)(units * (cum / total) + 0.5);
+    if (b < bounds[s]) b = bounds[s];
+    if (b > units) b = units;
+    bounds[s + 1] = b;
+  }
+  bounds[n_slots] = units;
 }
 
 // Geometry of one pass of R rows over K columns.

@@ -46,8 +46,8 @@ __global__ void pack_kernel(const PackOp d, const PackSrc s, unsigned char* pack
                             int inverse) {
   const int vrow = blockIdx.x;
   const int wd = d.s.wdtype, K = d.s.K;
-  const int slot = slot_of_row(d.s.rows, d.s.unit_rows, n_blocks, vrow);
-  const Slice sl = slot_slice(d.s.rows, d.s.unit_rows, n_blocks, slot);
+  const int slot = slot_of_row(d.bounds, d.s.unit_rows, n_blocks, vrow);
+  const Slice sl = slot_slice(d.bounds, d.s.unit_rows, slot);
   const int local = vrow - sl.row0;
   const int ps = local / kPassRows, rp = local - ps * kPassRows;
   int64_t pass_off = 0;

@@ -7,7 +7,8 @@
 //     columns one lane quad supplies to the tensor core for a block are one contiguous run,
 //   * every ring tile is 16-byte aligned, fits the stage, and the tiles of a pass are contiguous and cover it,
 //   * every work unit a consumer warp touches lies inside the tile it waits for.
-// Usage: layout_check rows K wdtype unit_rows n_blocks stage_bytes   -> prints "ok" or a diagnostic.
+// Usage: layout_check rows K wdtype unit_rows n_blocks stage_bytes [skew]  -> prints "ok" or a diagnostic.
+// skew > 0 gives the slots unequal weights (1 + skew * (slot % 7) / 7), as a measured-bandwidth split would.
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -20,6 +21,12 @@ int main(int argc, char** argv) {
   if (argc < 7) return 2;
   const int rows = atoi(argv[1]), K = atoi(argv[2]), wd = atoi(argv[3]), unit_rows = atoi(argv[4]);
   const int N = atoi(argv[5]), stage = atoi(argv[6]);
+  const double skew = argc > 7 ? atof(argv[7]) : 0.0;
+  std::vector<double> wts(N);
+  for (int i = 0; i < N; i++) wts[i] = 1.0 + skew * (i % 7) / 7.0;
+  std::vector<int> bounds(N + 1);
+  make_bounds(rows / unit_rows, N, wts.data(), bounds.data());
+  if (bounds[0] != 0 || bounds[N] != rows / unit_rows) { printf("bad bounds\n"); return 1; }
   const int bc = block_cols(wd), cpb = block_chunks(wd);
   const int epc = bc / cpb;                     // elements per 16-byte chunk
   if (K % bc) { printf("K not a multiple of the column block\n"); return 1; }
@@ -47,9 +54,9 @@ int main(int argc, char** argv) {
   std::vector<int> seen((size_t)rows * K, 0);
   long long covered = 0;
   for (int slot = 0; slot < N; slot++) {
-    const Slice sl = slot_slice(rows, unit_rows, N, slot);
+    const Slice sl = slot_slice(bounds.data(), unit_rows, slot);
     for (int r = sl.row0; r < sl.row0 + sl.rows; r++)
-      if (slot_of_row(rows, unit_rows, N, r) != slot) { printf("slot_of_row mismatch row %d\n", r); return 1; }
+      if (slot_of_row(bounds.data(), unit_rows, N, r) != slot) { printf("slot_of_row mismatch row %d\n", r); return 1; }
     const int np = n_passes(sl.rows);
     long long sbytes = 0;
     for (int ps = 0; ps < np; ps++) {
