@@ -214,6 +214,12 @@ __device__ __forceinline__ void store_line(unsigned char* xs, int n2, int ln, fl
     const unsigned lb = f32_to_bf16_rne(b - __uint_as_float(hb << 16));
     X0[ln] = ha | (hb << 16);
     X1[ln] = la | (lb << 16);
+    if (inv > 0.f) {                                   // third column: what the first two still miss
+      unsigned* X2 = X1 + n2;
+      const unsigned ra = f32_to_bf16_rne((a - __uint_as_float(ha << 16)) - __uint_as_float(la << 16));
+      const unsigned rb = f32_to_bf16_rne((b - __uint_as_float(hb << 16)) - __uint_as_float(lb << 16));
+      X2[ln] = ra | (rb << 16);
+    }
   } else {
     unsigned short* D2 = reinterpret_cast<unsigned short*>(xs);
     unsigned short* D1 = D2 + n2;
@@ -337,6 +343,7 @@ __device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* s
       res.xscale = mx / kDigitScale;
     }
   }
+  if (WD == W_BF16) inv = (6 * K <= p.act_bytes) ? 1.f : 0.f;     // room for a third bf16 column of the input?
 #pragma unroll 1
   for (int l0 = tid; l0 < n2; l0 += kBatch * kConsumerThreads) {
     if (!(reduce && held)) res.bad |= gather_batch(p, raw, l0, n2, src, seq, src_task, embed_row);
@@ -370,7 +377,9 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int K, f
   const unsigned step_stride = (unsigned)(2 * urows * 16);                     // two chunks per k step
   const int S = p.n_stages;
   constexpr int BC = (WD == W_INT4) ? 128 : 64;
-  constexpr int NCOL = (WD == W_BF16) ? 2 : 3;                                  // B columns in use
+  // B columns in use: int8 / int4 three digits; bf16 high + low halves, plus a third term (fp32-exact
+  // input) whenever the input area has room for it
+  const int NCOL = (WD == W_BF16) ? ((6 * K <= p.act_bytes) ? 3 : 2) : 3;
   const unsigned char* xcol = c.xs + (size_t)min(gq, NCOL - 1) * K * (WD == W_BF16 ? 2 : 1);
 
   float facc[4] = {0.f, 0.f, 0.f, 0.f};
@@ -454,7 +463,7 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int K, f
   // per-row result: sum of the B columns in use, with the digit weights for integer inputs
   float y0, y1;
   if (WD == W_BF16) {
-    y0 = facc[0] + facc[1];
+    y0 = facc[0] + facc[1];                            // (columns not in use are zero; the sum over the quad follows)
     y1 = facc[2] + facc[3];
   } else {
     // columns 2q and 2q+1 of this lane: digit weights 16384 (col 0), 128 (col 1), 1 (col 2), 0 otherwise

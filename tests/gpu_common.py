@@ -10,6 +10,7 @@ HIDDEN_TOL = 5e-3      # rel-L2 per layer hidden state
 LOGITS_TOL = 1e-2      # rel-L2 on logits
 ARGMAX_GAP = 1e-2      # the greedy token must match bit-exactly when the oracle's top-2 gap exceeds this
 WD = {"bf16": orc.W_BF16, "int8": orc.W_INT8, "int4": orc.W_INT4}
+LAST = {}                # the last compared step's raw outputs, for callers that need them
 
 
 def rel_l2(a, b):
@@ -54,6 +55,7 @@ def compare_step(shape, dec, model, token, pos, kv_gpu, kv_cpu, check_hidden=Tru
     logits_o, tok_o, hidden_o = model.decode_step(token, pos, kv_cpu, want_hidden=check_hidden)
     logits_g = dec.logits.cpu().numpy()
     tok_g = int(dec.next_token.item())
+    LAST["logits_oracle"], LAST["logits_gpu"], LAST["token_gpu"] = logits_o, logits_g, tok_g
     out = {"logits": rel_l2(logits_g, logits_o)}
     assert np.isfinite(logits_g).all()
     if check_hidden:
