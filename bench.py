@@ -113,6 +113,21 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(x: float, device="cpu") -> float:
+    """Largest value of `x` over all ranks (the timing rule for anything multi-GPU); identity for one rank."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(x)
+    t = torch.tensor([x], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(us_per_step_max: float, replicas: int) -> float:
+    """Job-level microseconds per decoded token when `replicas` independent sequences decode side by side."""
+    return us_per_step_max / replicas
+
+
 def build_decoder(workload: str, device, flags: int = 0):
     from paper_2606_09682_b200 import binding as amk
     name, wd, pos = WORKLOADS[workload]
@@ -329,15 +344,9 @@ def main():
         raise SystemExit("decode step failed: " + msg)
     per = np.array([ev[i].elapsed_time(ev[i + 1]) * 1e3 for i in range(a.steps)])
     total_ms = ev[0].elapsed_time(ev[a.steps])
-    t = torch.tensor([total_ms], device=device, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, device)
     e2e_us, h2d, d2h = time_e2e(dec, shape, tok, pos, kv, max(5, a.steps // 4), 3)
-    te = torch.tensor([e2e_us], device=device, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(te, op=dist.ReduceOp.MAX)
-        e2e_us = float(te.item())
+    e2e_us = max_over_ranks(e2e_us, device)
 
     if rank == 0:
         peak, peak_src = measured_peak()
@@ -345,11 +354,11 @@ def main():
         us = total_ms * 1e3 / a.steps
         achieved = b["total"] / (us * 1e-6) / 1e9
         plan = dec.plan()
-        line = {"metric": METRIC, "value": us / world, "unit": "us/token", "n_gpus": world, "steps": a.steps,
+        line = {"metric": METRIC, "value": job_value(us, world), "unit": "us/token", "n_gpus": world, "steps": a.steps,
                 "warmup": a.warmup, "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak",
                 "vs_baseline": None, "dtype": wd if wd != "bf16" else "bf16 (fp32 accumulate)", "data": "synthetic",
                 "config": config, "clocks": clocks, "gpu_launches": a.steps,
-                "e2e": {"value": e2e_us / world, "unit": "us/token", "h2d_bytes_per_step": h2d,
+                "e2e": {"value": job_value(e2e_us, world), "unit": "us/token", "h2d_bytes_per_step": h2d,
                         "d2h_bytes_per_step": d2h},
                 "latency_us": {"median": float(np.median(per)), "p10": float(np.percentile(per, 10)),
                                "p90": float(np.percentile(per, 90))},
