@@ -230,6 +230,30 @@ amk_status amk_quantize_int8(const void* w_bf16, int64_t rows, int64_t cols, voi
 amk_status amk_quantize_int4(const void* w_bf16, int64_t rows, int64_t cols, void* packed_out, void* scale_out,
                              void* zero_out, void* cuda_stream);
 
+/*
+ * Greedy token of a logits vector, with scratch memory that is a fixed array inside the library image.
+ * The paper has no counterpart of this call: its kernel picks the token inside the decode step, as
+ * amk_decode_step does (the LM-head tail).  This is that tail alone -- every block of 2048 elements
+ * publishes its best {value, index}, the block that arrives last reduces them -- for callers that change
+ * the logits between the decode step and the choice of the token and want neither a workspace nor an
+ * allocation: the call allocates no host or device memory at all.
+ *   x      DEVICE in, n floats             token  DEVICE out, one int32 (lowest index among equal maxima)
+ *   n      1 .. AMK_ARGMAX_STATIC_MAX_N; larger n returns AMK_ERR_UNSUPPORTED, n < 1 or a NULL pointer
+ *          AMK_ERR_INVALID_ARG, a failed runtime call AMK_ERR_CUDA
+ *   msg    HOST out, msg_bytes bytes, may be NULL: the reason in words when the status is not AMK_OK
+ * The scratch (4352 bytes per device: an arrival counter and 512 candidates) belongs to the library.  The
+ * counter must be zero at the start of a call: it is zero when the library is loaded and the kernel puts it
+ * back to zero before it ends; the candidates need no initial value.  Because all calls on a device share
+ * the one scratch array, two calls that overlap in time (different streams, or different threads without
+ * an order between their streams) race and give wrong tokens: keep the calls of a device in one stream or
+ * order them with events.  The first call on each device looks up the scratch address (set-up, a
+ * synchronous runtime query under a lock), so make it before any stream capture that is to contain later
+ * calls.  Asynchronous on cuda_stream otherwise.
+ */
+#define AMK_ARGMAX_STATIC_MAX_N (1 << 20)
+amk_status amk_argmax_static(const float* x, int64_t n, int32_t* token, char* msg, size_t msg_bytes,
+                             void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

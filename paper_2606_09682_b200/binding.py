@@ -76,6 +76,7 @@ def _load() -> C.CDLL:
         "amk_destroy": (C.c_int, [vp]),
         "amk_quantize_int8": (C.c_int, [vp, i64, i64, vp, vp, vp]),
         "amk_quantize_int4": (C.c_int, [vp, i64, i64, vp, vp, vp, vp]),
+        "amk_argmax_static": (C.c_int, [vp, i64, vp, C.c_char_p, sz, vp]),
     }
     for name, (res, args) in sigs.items():
         fn = getattr(lib, name)
@@ -86,7 +87,8 @@ def _load() -> C.CDLL:
 lib = _load()
 EXPORTS = ("amk_status_str", "amk_packed_bytes", "amk_workspace_bytes", "amk_kv_bytes", "amk_create",
            "amk_decode_step", "amk_decode_greedy", "amk_last_status", "amk_plan_info", "amk_debug_hidden",
-           "amk_debug_trace", "amk_debug_unpack", "amk_debug_drop_signal", "amk_destroy", "amk_quantize_int8", "amk_quantize_int4")
+           "amk_debug_trace", "amk_debug_unpack", "amk_debug_drop_signal", "amk_destroy", "amk_quantize_int8", "amk_quantize_int4",
+           "amk_argmax_static")
 
 
 class AmkError(RuntimeError):
@@ -161,6 +163,20 @@ def amk_quantize_int4(w: torch.Tensor):
     _check(lib.amk_quantize_int4(w.data_ptr(), rows, cols, p.data_ptr(), s.data_ptr(), z.data_ptr(), _stream()),
            "amk_quantize_int4")
     return p, s, z
+
+
+AMK_ARGMAX_STATIC_MAX_N = 1 << 20
+
+
+def amk_argmax_static(x: torch.Tensor, token: torch.Tensor, n: int = -1) -> None:
+    """fp32 vector (cuda) -> token[0] (int32, cuda) = index of its maximum; library-owned scratch, no allocation.
+    ``n`` overrides the element count handed to the library (for argument-checking tests)."""
+    assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous()
+    assert token.is_cuda and token.dtype == torch.int32 and token.numel() >= 1
+    msg = C.create_string_buffer(256)
+    code = lib.amk_argmax_static(x.data_ptr(), x.numel() if n < 0 else n, token.data_ptr(), msg, 256, _stream())
+    if code != AMK_OK:
+        raise AmkError(code, msg.value.decode() or "amk_argmax_static")
 
 
 def quantize_weights(weights: Dict, wdtype: str) -> Dict:

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libamk.so")
-SOURCES = ["amk_host.cu", "amk_kernel.cu", "amk_pack.cu"]
+SOURCES = ["amk_host.cu", "amk_kernel.cu", "amk_pack.cu", "amk_static.cu"]
 HEADERS = ["amk_layout.h", "amk_internal.h", "amk_ptx.cuh", os.path.join(ROOT, "include", "amk.h")]
 
 
