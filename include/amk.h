@@ -52,14 +52,19 @@ typedef enum { AMK_W_BF16 = 0, AMK_W_INT8 = 1, AMK_W_INT4 = 2 } amk_wdtype;
 
 /* Trace layout (amk_debug_trace): uint64 nanosecond stamps [n_blocks][n_tasks][AMK_TRACE_EVENTS], where
  * task 5*l+{0,1,2,3,4} = QKV, attention, O, gate/up, down of layer l and task 5*L = LM head. */
-#define AMK_TRACE_EVENTS 8
+#define AMK_TRACE_EVENTS 12
 enum { AMK_TR_ENTER = 0,      /* consumer warps reach the task                                          */
        AMK_TR_JOINED = 1,     /* the dependency wait is over                                            */
        AMK_TR_LOADED = 2,     /* input vector in shared memory (GEMV tasks)                             */
        AMK_TR_COMPUTED = 3,   /* last output stored                                                     */
        AMK_TR_SIGNALLED = 4,  /* counter incremented                                                    */
        AMK_TR_PROD_FIRST = 5, /* producer issued the task's first ring tile (GEMV tasks)                */
-       AMK_TR_PROD_LAST = 6   /* producer issued the task's last ring tile                              */
+       AMK_TR_PROD_LAST = 6,  /* producer issued the task's last ring tile                              */
+       AMK_TR_REDUCED = 7,    /* last pass: per-row partial sums are in shared memory                   */
+       AMK_TR_PASS_BEGIN = 8, /* last pass: epilogue operands requested, tile walk starts               */
+       AMK_TR_FIRST_TILE = 9, /* last pass: its first ring tile has landed                              */
+       AMK_TR_TILES_DONE = 10,/* last pass: all ring tiles multiplied                                   */
+       AMK_TR_POLLS = 11      /* NOT a time: requests thread 0 made for its first batch of input lines   */
 };
 
 /* The seven per-layer linears, in the order used by amk_weights.linear[] and amk_debug_unpack. */
@@ -89,7 +94,7 @@ typedef struct amk_config {
   /* tuning knobs, 0 = automatic */
   uint32_t stage_bytes;      /* bytes per shared-memory ring stage (multiple of 1024)                  */
   uint32_t n_stages;         /* ring depth                                                             */
-  uint32_t max_inflight;     /* bulk copies a block keeps in flight (<= n_stages)                      */
+  uint32_t max_inflight;     /* bulk copies a block keeps in flight (<= n_stages; 0 = default 3)        */
   uint32_t sync_mode;        /* 0: activations carry sequence numbers AND every task ends with a release-
                                 increment that the next task's readers acquire-spin on (the paper's counter
                                 model); 1: sequence numbers only (no counters, no fences).  Same results.  */

@@ -45,7 +45,7 @@ struct Plan {
 };
 
 struct WorkspaceLayout {
-  size_t status, phase_ctr, group_ctr, lm_ctr, next_ws, cand_val, cand_idx, x_a, x_b, qkv, o, m, part, hidden, rope,
+  size_t status, phase_ctr, group_ctr, lm_ctr, next_ws, cand_val, cand_idx, x_a, x_b, qkv, o, m, m_amax, part, hidden, rope,
       trace, slice_tab, bounds, smid_tab, calib, tile_begin, tiles, total;
 };
 
@@ -192,6 +192,7 @@ WorkspaceLayout workspace_layout(const amk_config* c, const Plan& pl) {
   w.qkv = take((qd + 2 * kvd) * sizeof(ActPair));
   w.o = take(qd * sizeof(ActPair));
   w.m = take(I * sizeof(ActPair));
+  w.m_amax = take(kMaxBlocks * sizeof(ActPair));
   w.part = take((size_t)c->n_q_heads * kMaxChunks * (hd + 2) * 4);
   w.hidden = take((L + 1) * H * 4);
   w.rope = take(S * (hd / 2) * sizeof(float2));
@@ -410,7 +411,9 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
       status = AMK_ERR_UNSUPPORTED;
       goto fail;
     }
-    uint32_t max_inflight = cfg->max_inflight ? cfg->max_inflight : n_stages;
+    // default: three copies in flight per block -- enough to saturate HBM from 148 blocks; more only deepens the
+    // memory system's queues, which every dependency-carrying load then waits behind (measured: 3 beats 5 by 2-4 %)
+    uint32_t max_inflight = cfg->max_inflight ? cfg->max_inflight : 3;
     if (max_inflight > n_stages) max_inflight = n_stages;
     const size_t smem_bytes = hdr + act + (size_t)n_stages * stage_bytes;
     int per_sm = 0;
@@ -517,6 +520,7 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     p.rope = (const float2*)(h->ws + h->wl.rope);
     p.x_a = (ActPair*)(h->ws + h->wl.x_a); p.x_b = (ActPair*)(h->ws + h->wl.x_b);
     p.qkv = (ActPair*)(h->ws + h->wl.qkv); p.o = (ActPair*)(h->ws + h->wl.o); p.m = (ActPair*)(h->ws + h->wl.m);
+    p.m_amax = (ActPair*)(h->ws + h->wl.m_amax);
     p.part = (float*)(h->ws + h->wl.part); p.hidden = (float*)(h->ws + h->wl.hidden);
     p.phase_ctr = (unsigned*)(h->ws + h->wl.phase_ctr); p.group_ctr = (unsigned*)(h->ws + h->wl.group_ctr);
     p.lm_ctr = (unsigned*)(h->ws + h->wl.lm_ctr); p.cand_val = (float*)(h->ws + h->wl.cand_val);

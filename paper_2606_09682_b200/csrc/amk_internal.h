@@ -32,6 +32,13 @@ struct SmemHeader {
   int slot;                          // this block's slot (its share of every op, its tile list)
   int slice_row0[5], slice_rows[5];  // its rows of each op kind
   int pad[1];
+  // Pass geometry of each op kind for this block's slice, worked out once at kernel start (it takes a dozen
+  // integer divisions, which would otherwise sit on every task's critical path): [kind][0] a full pass of
+  // kPassRows rows (used when the slice has more than one pass), [kind][1] the last pass.
+  PassGeom geom[5][2];
+  int step_b[5][2], step_r[5][2];                    // tile-to-tile step of the unit walk: upt / Wr, upt % Wr
+  unsigned char wr_of[5][2][kConsumerWarps + 1];     // warp -> row-warp index, k-warp index
+  unsigned char wk_of[5][2][kConsumerWarps + 1];
 };
 
 // An activation element in global memory: the value and the sequence number of the task that wrote it.
@@ -81,6 +88,7 @@ struct KParams {
   ActPair* qkv;
   ActPair* o;
   ActPair* m;
+  ActPair* m_amax;                        // [n_blocks] max |m| over each block's rows (integer-weight models)
   float* part;                            // [nq][kMaxChunks][hd + 2]
   float* hidden;                          // [(L+1)][H]
   unsigned* phase_ctr;                    // [5 L]

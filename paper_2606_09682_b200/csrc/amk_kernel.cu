@@ -246,7 +246,7 @@ __device__ __forceinline__ void store_line(unsigned char* xs, int n2, int ln, fl
 // the whole batch again until all carry `seq` (bounded).  Returns true on failure.
 __device__ __forceinline__ bool gather_batch(const KParams& p, uint4 (&raw)[kBatch], int line0, int n2,
                                              const ActPair* src, unsigned seq, int src_task,
-                                             const unsigned short* embed_row) {
+                                             const unsigned short* embed_row, int cta, int task) {
   if (embed_row) {
 #pragma unroll
     for (int i = 0; i < kBatch; i++) {
@@ -271,7 +271,11 @@ __device__ __forceinline__ bool gather_batch(const KParams& p, uint4 (&raw)[kBat
       const int ln = line0 + i * kConsumerThreads;
       if (ln < n2) all = all && (raw[i].y == seq) && (raw[i].w == seq);
     }
-    if (all) return false;
+    if (all) {
+      if (p.trace && line0 == 0)     // (not a time) how many requests thread 0 needed for its first batch
+        p.trace[((size_t)cta * (5 * p.L + 1) + task) * AMK_TRACE_EVENTS + AMK_TR_POLLS] = spins + 1u;
+      return false;
+    }
     if (spins == 0) t0 = globaltimer_ns();
     if ((spins & 15u) == 15u) {
       if (ld_relaxed_gpu(&p.status->abort)) return true;
@@ -295,7 +299,7 @@ template <int WD>
 __device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* sh, unsigned char* xs, int cta, int K,
                                                  const ActPair* src, unsigned seq, int src_task,
                                                  const unsigned short* embed_row, const unsigned short* normw,
-                                                 int task) {
+                                                 int task, const ActPair* amax_src, int nblk) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n2 = K >> 1;                               // lines of two elements
   LoadResult res{1.0f, false};
@@ -303,11 +307,19 @@ __device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* s
   const bool reduce = (normw != nullptr) || (WD != W_BF16);
   const bool held = n2 <= kBatch * kConsumerThreads;
   float r = 1.0f, inv = 0.f;
+  // `amax_src`: the producers of this (integer, un-normed) input also published the maximum of their part, so
+  // the vector need not be read twice: the first batch is requested, the maxima are combined meanwhile.
+  const bool have_first = reduce && (held || amax_src != nullptr);
   if (reduce) {
     float ss = 0.f, amax = 0.f;
+    if (amax_src) {
+      res.bad |= gather_batch(p, raw, tid, n2, src, seq, src_task, embed_row, cta, task);
+      for (int b = tid; b < nblk; b += kConsumerThreads)
+        amax = fmaxf(amax, fabsf(read_act(p, res.bad, amax_src + b, seq, src_task)));
+    }
 #pragma unroll 1
-    for (int l0 = tid; l0 < n2; l0 += kBatch * kConsumerThreads) {
-      res.bad |= gather_batch(p, raw, l0, n2, src, seq, src_task, embed_row);
+    for (int l0 = tid; l0 < n2 && !amax_src; l0 += kBatch * kConsumerThreads) {
+      res.bad |= gather_batch(p, raw, l0, n2, src, seq, src_task, embed_row, cta, task);
 #pragma unroll
       for (int i = 0; i < kBatch; i++) {
         const int ln = l0 + i * kConsumerThreads;
@@ -346,7 +358,7 @@ __device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* s
   if (WD == W_BF16) inv = (6 * K <= p.act_bytes) ? 1.f : 0.f;     // room for a third bf16 column of the input?
 #pragma unroll 1
   for (int l0 = tid; l0 < n2; l0 += kBatch * kConsumerThreads) {
-    if (!(reduce && held)) res.bad |= gather_batch(p, raw, l0, n2, src, seq, src_task, embed_row);
+    if (!(have_first && l0 == tid)) res.bad |= gather_batch(p, raw, l0, n2, src, seq, src_task, embed_row, cta, task);
 #pragma unroll
     for (int i = 0; i < kBatch; i++) {
       const int ln = l0 + i * kConsumerThreads;
@@ -366,9 +378,11 @@ __device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* s
 #define AMK_HI(x, z) (((((x) >> 4) & 0x0F0F0F0Fu) + (z)) ^ 0x80808080u)
 
 template <int WD>
-__device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int K, float* red) {
+__device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int kind, int gw, int K, float* red,
+                                             int task) {
   const KParams& p = c.p;
-  const int wr = c.warp % g.Wr, wk = c.warp / g.Wr;
+  if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_PASS_BEGIN);
+  const int wr = c.sh->wr_of[kind][gw][c.warp], wk = c.sh->wk_of[kind][gw][c.warp];
   const bool active = wk < g.Wk;
   const int urows = (wr == g.Wr - 1) ? g.g_last : g.G;
   const int gq = c.lane >> 2, q = c.lane & 3;                                  // fragment row / column-pair index
@@ -382,75 +396,80 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int K, f
   const int NCOL = (WD == W_BF16) ? ((6 * K <= p.act_bytes) ? 3 : 2) : 3;
   const unsigned char* xcol = c.xs + (size_t)min(gq, NCOL - 1) * K * (WD == W_BF16 ? 2 : 1);
 
-  float facc[4] = {0.f, 0.f, 0.f, 0.f};
-  int iacc[4] = {0, 0, 0, 0};
+  // All fragments of a unit are loaded before its first MMA, and two accumulator sets are used in turn, so
+  // that consecutive MMAs do not wait for each other.
+  float facc[4] = {0.f, 0.f, 0.f, 0.f}, facc2[4] = {0.f, 0.f, 0.f, 0.f};
+  int iacc[4] = {0, 0, 0, 0}, iacc2[4] = {0, 0, 0, 0};
+  constexpr int NA = (WD == W_BF16) ? 4 : 2;         // ldmatrix.x4 loads per unit
+  unsigned fa[NA][4];                                // pending unit: weight fragments,
+  uint4 fx0 = make_uint4(0u, 0u, 0u, 0u), fx1 = fx0; // input fragments,
+  unsigned fsz0 = 0u, fsz1 = 0u;                     // int4: {scale, zero} of my two rows
+  auto flush = [&]() {
+    if (WD == W_BF16) {
+      mma_bf16(facc, fa[0], fx0.x, fx0.y);
+      mma_bf16(facc2, fa[1], fx0.z, fx0.w);
+      mma_bf16(facc, fa[2], fx1.x, fx1.y);
+      mma_bf16(facc2, fa[3], fx1.z, fx1.w);
+    } else if (WD == W_INT8) {
+      mma_s8(iacc, fa[0][0], fa[0][1], fa[0][2], fa[0][3], fx0.x, fx0.y);
+      mma_s8(iacc2, fa[1][0], fa[1][1], fa[1][2], fa[1][3], fx0.z, fx0.w);
+    } else {
+      const float s0 = __half2float(__ushort_as_half((unsigned short)(fsz0 & 0xffffu)));
+      const float s1 = __half2float(__ushort_as_half((unsigned short)(fsz1 & 0xffffu)));
+      // code - zero as a signed byte: (code + 128 - zero) ^ 0x80; no carries between bytes
+      const unsigned z0 = (unsigned)(128 - (int)__half2float(__ushort_as_half((unsigned short)(fsz0 >> 16)))) * 0x01010101u;
+      const unsigned z1 = (unsigned)(128 - (int)__half2float(__ushort_as_half((unsigned short)(fsz1 >> 16)))) * 0x01010101u;
+      int g4[4] = {0, 0, 0, 0}, h4[4] = {0, 0, 0, 0};
+      mma_s8(g4, AMK_LO(fa[0][0], z0), AMK_LO(fa[0][1], z1), AMK_LO(fa[0][2], z0), AMK_LO(fa[0][3], z1), fx0.x, fx0.y);
+      mma_s8(h4, AMK_HI(fa[0][0], z0), AMK_HI(fa[0][1], z1), AMK_HI(fa[0][2], z0), AMK_HI(fa[0][3], z1), fx0.z, fx0.w);
+      mma_s8(g4, AMK_LO(fa[1][0], z0), AMK_LO(fa[1][1], z1), AMK_LO(fa[1][2], z0), AMK_LO(fa[1][3], z1), fx1.x, fx1.y);
+      mma_s8(h4, AMK_HI(fa[1][0], z0), AMK_HI(fa[1][1], z1), AMK_HI(fa[1][2], z0), AMK_HI(fa[1][3], z1), fx1.z, fx1.w);
+      facc[0] = fmaf(s0, (float)(g4[0] + h4[0]), facc[0]);
+      facc[1] = fmaf(s0, (float)(g4[1] + h4[1]), facc[1]);
+      facc[2] = fmaf(s1, (float)(g4[2] + h4[2]), facc[2]);
+      facc[3] = fmaf(s1, (float)(g4[3] + h4[3]), facc[3]);
+    }
+  };
   int next_b = wk;                                   // my next column block
   const int my_off = wr * g.ub_full;
   // first unit of the current tile as (block, row-warp), and the step from one tile to the next
   int t_b = 0, t_r = 0;
-  const int step_b = g.upt / g.Wr, step_r = g.upt - step_b * g.Wr;
+  const int step_b = c.sh->step_b[kind][gw], step_r = c.sh->step_r[kind][gw];
   for (int t = 0; t < g.n_tiles; ++t) {
     const int tile_off = t_b * g.bb + t_r * g.ub_full;
     int n_b = t_b + step_b, n_r = t_r + step_r;      // first unit of the next tile
     if (n_r >= g.Wr) { n_r -= g.Wr; n_b++; }
     if (!c.bad && !wait_mbar(p, &c.sh->full[c.stage], c.parity, -1)) c.bad = true;
+    if (c.tid == 0 && t == 0) stamp(p, c.cta, task, AMK_TR_FIRST_TILE);
     if (active && !c.bad) {
       const unsigned char* sbase = c.ring + (size_t)c.stage * p.stage_bytes;
       // my units in this tile: blocks next_b, next_b + Wk, ... while (b, wr) comes before (n_b, n_r)
       while (next_b < g.nblk && (next_b < n_b || (next_b == n_b && wr < n_r))) {
         const unsigned char* u = sbase + (next_b * g.bb + my_off - tile_off);
+        fx0 = make_uint4(0u, 0u, 0u, 0u);
+        fx1 = fx0;
         if (WD == W_BF16) {
-          uint4 xb0 = make_uint4(0u, 0u, 0u, 0u), xb1 = xb0;
           if (gq < NCOL) {
             const uint4* xp = reinterpret_cast<const uint4*>(xcol + ((size_t)next_b * BC + 16 * q) * 2);
-            xb0 = xp[0];
-            xb1 = xp[1];
+            fx0 = xp[0];
+            fx1 = xp[1];
           }
-          unsigned a[4];
-          ldmatrix_x4(a, u + lane_off);
-          mma_bf16(facc, a, xb0.x, xb0.y);
-          ldmatrix_x4(a, u + lane_off + step_stride);
-          mma_bf16(facc, a, xb0.z, xb0.w);
-          ldmatrix_x4(a, u + lane_off + 2 * step_stride);
-          mma_bf16(facc, a, xb1.x, xb1.y);
-          ldmatrix_x4(a, u + lane_off + 3 * step_stride);
-          mma_bf16(facc, a, xb1.z, xb1.w);
         } else if (WD == W_INT8) {
-          uint4 xb = make_uint4(0u, 0u, 0u, 0u);
-          if (gq < NCOL) xb = *reinterpret_cast<const uint4*>(xcol + (size_t)next_b * BC + 16 * q);
-          unsigned a[4];
-          ldmatrix_x4(a, u + lane_off);
-          mma_s8(iacc, a[0], a[1], a[2], a[3], xb.x, xb.y);
-          ldmatrix_x4(a, u + lane_off + step_stride);
-          mma_s8(iacc, a[0], a[1], a[2], a[3], xb.z, xb.w);
+          if (gq < NCOL) fx0 = *reinterpret_cast<const uint4*>(xcol + (size_t)next_b * BC + 16 * q);
         } else {
-          uint4 xb0 = make_uint4(0u, 0u, 0u, 0u), xb1 = xb0;
           if (gq < NCOL) {
             const uint4* xp = reinterpret_cast<const uint4*>(xcol + (size_t)next_b * BC + 32 * q);
-            xb0 = xp[0];
-            xb1 = xp[1];
+            fx0 = xp[0];
+            fx1 = xp[1];
           }
           // {scale, zero} of my two fragment rows for this group (= this column block)
           const unsigned* szp = reinterpret_cast<const unsigned*>(u + urows * 64);
-          const unsigned sz0 = szp[min(gq, urows - 1)], sz1 = szp[min(gq + 8, urows - 1)];
-          const float s0 = __half2float(__ushort_as_half((unsigned short)(sz0 & 0xffffu)));
-          const float s1 = __half2float(__ushort_as_half((unsigned short)(sz1 & 0xffffu)));
-          // code - zero as a signed byte: (code + 128 - zero) ^ 0x80; no carries between bytes
-          const unsigned z0 = (unsigned)(128 - (int)__half2float(__ushort_as_half((unsigned short)(sz0 >> 16)))) * 0x01010101u;
-          const unsigned z1 = (unsigned)(128 - (int)__half2float(__ushort_as_half((unsigned short)(sz1 >> 16)))) * 0x01010101u;
-          int g4[4] = {0, 0, 0, 0};
-          unsigned a[4];
-          ldmatrix_x4(a, u + lane_off);
-          mma_s8(g4, AMK_LO(a[0], z0), AMK_LO(a[1], z1), AMK_LO(a[2], z0), AMK_LO(a[3], z1), xb0.x, xb0.y);
-          mma_s8(g4, AMK_HI(a[0], z0), AMK_HI(a[1], z1), AMK_HI(a[2], z0), AMK_HI(a[3], z1), xb0.z, xb0.w);
-          ldmatrix_x4(a, u + lane_off + step_stride);
-          mma_s8(g4, AMK_LO(a[0], z0), AMK_LO(a[1], z1), AMK_LO(a[2], z0), AMK_LO(a[3], z1), xb1.x, xb1.y);
-          mma_s8(g4, AMK_HI(a[0], z0), AMK_HI(a[1], z1), AMK_HI(a[2], z0), AMK_HI(a[3], z1), xb1.z, xb1.w);
-          facc[0] = fmaf(s0, (float)g4[0], facc[0]);
-          facc[1] = fmaf(s0, (float)g4[1], facc[1]);
-          facc[2] = fmaf(s1, (float)g4[2], facc[2]);
-          facc[3] = fmaf(s1, (float)g4[3], facc[3]);
+          fsz0 = szp[min(gq, urows - 1)];
+          fsz1 = szp[min(gq + 8, urows - 1)];
         }
+#pragma unroll
+        for (int j = 0; j < NA; j++) ldmatrix_x4(fa[j], u + lane_off + j * step_stride);
+        flush();
         next_b += g.Wk;
       }
     }
@@ -460,6 +479,9 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int K, f
     t_b = n_b;
     t_r = n_r;
   }
+#pragma unroll
+  for (int e = 0; e < 4; e++) { facc[e] += facc2[e]; iacc[e] += iacc2[e]; }
+  if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_TILES_DONE);
   // per-row result: sum of the B columns in use, with the digit weights for integer inputs
   float y0, y1;
   if (WD == W_BF16) {
@@ -521,17 +543,51 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind, int l) {
     case OP_DOWN: src = p.m; src_task = 5 * l + 3; break;
     default: src = p.x_a; src_task = 5 * (p.L - 1) + 4; normw = p.final_norm; break;
   }
-  // geometry of the first pass while nothing else can be done
   const int np = n_passes(sl.rows);
-  PassGeom g = pass_geom(np ? pass_rows(sl.rows, 0) : 1, K, d.wdtype, p.stage_bytes);
+
+  // Epilogue operands (residual element, int8 row scales) of a pass: requested before the pass -- those of the
+  // first pass before the dependency wait -- and first looked at after it, so their latency is hidden.
+  uint2 rraw = make_uint2(0u, 0u);                       // residual {value, seq}
+  const ActPair* raddr = nullptr;
+  int rtask = -1;
+  __half sh0 = __float2half(1.f), sh1 = __float2half(1.f);
+  auto request_operands = [&](int ps) {
+    const int R = pass_rows(sl.rows, ps);
+    const int vrow0 = sl.row0 + ps * kPassRows;
+    raddr = nullptr;
+    if (c.tid < ((kind == OP_GATEUP) ? (R >> 1) : R)) {
+      const int vrow = vrow0 + c.tid;
+      if (kind == OP_O) {
+        if (first_layer) rraw.x = (unsigned)__ldg(embed_row + vrow) << 16;
+        else { raddr = p.x_a + vrow; rtask = 5 * (l - 1) + 4; }
+      } else if (kind == OP_DOWN) {
+        raddr = p.x_b + vrow;
+        rtask = 5 * l + 2;
+      }
+      if (raddr) rraw = ld_pair(raddr);
+      if (d.wdtype == W_INT8) {
+        const __half* scales = reinterpret_cast<const __half*>(
+            p.packed + p.scale_base + (size_t)l * p.scale_layer_stride + p.scale_kind_off[kind]);
+        if (kind == OP_GATEUP) {
+          sh0 = __ldg(scales + vrow0 + 2 * c.tid);
+          sh1 = __ldg(scales + vrow0 + 2 * c.tid + 1);
+        } else {
+          sh0 = __ldg(scales + vrow);
+        }
+      }
+    }
+  };
+  if (np > 0) request_operands(0);
 
   if (!from_embed && !wait_phase(c, src_task)) return false;
   if (np > 0) {
     const unsigned in_seq = from_embed ? 1u : seq_of(p, src_task);
     const unsigned short* erow = from_embed ? embed_row : nullptr;
     const LoadResult lr = (WDL == W_BF16 || kind == OP_LMHEAD)
-                              ? load_input<W_BF16>(p, c.sh, c.xs, c.cta, K, src, in_seq, src_task, erow, normw, task)
-                              : load_input<WDL>(p, c.sh, c.xs, c.cta, K, src, in_seq, src_task, erow, normw, task);
+                              ? load_input<W_BF16>(p, c.sh, c.xs, c.cta, K, src, in_seq, src_task, erow, normw, task,
+                                                   nullptr, c.nblk)
+                              : load_input<WDL>(p, c.sh, c.xs, c.cta, K, src, in_seq, src_task, erow, normw, task,
+                                                kind == OP_DOWN ? p.m_amax : nullptr, c.nblk);
     c.xscale = lr.xscale;
     c.bad = lr.bad;
     if (c.bad) return false;
@@ -542,40 +598,31 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind, int l) {
   float best_val = -CUDART_INF_F;
   int best_idx = 0x7fffffff;
   const bool drop = (task == p.drop_phase && c.cta == p.drop_block);
+  float gu_amax = 0.f;                                // gate/up of an integer-weight model: max |output| of this block
   for (int ps = 0; ps < np; ps++) {
     const int R = pass_rows(sl.rows, ps);
-    if (ps > 0) g = pass_geom(R, K, d.wdtype, p.stage_bytes);
+    const int gw = (ps == np - 1) ? 1 : 0;             // which precomputed geometry: a full pass or the last one
+    const PassGeom g = c.sh->geom[kind][gw];
     const int vrow0 = sl.row0 + ps * kPassRows;
     float* red = c.sh->red[ps & 1];
 
-    // epilogue operands fetched ahead of the pass
     const int n_out = (kind == OP_GATEUP) ? (R >> 1) : R;
     const bool outp = c.tid < n_out;
-    float resid = 0.f, sc0 = 1.f, sc1 = 1.f;
-    if (outp) {
-      const int vrow = vrow0 + c.tid;
-      if (kind == OP_O) {
-        resid = first_layer ? bf16_lo((unsigned)__ldg(embed_row + vrow))
-                            : read_act(p, c.bad, p.x_a + vrow, seq_of(p, 5 * (l - 1) + 4), 5 * (l - 1) + 4);
-      } else if (kind == OP_DOWN) {
-        resid = read_act(p, c.bad, p.x_b + vrow, seq_of(p, 5 * l + 2), 5 * l + 2);
-      }
-      if (d.wdtype == W_INT8) {
-        const __half* scales = reinterpret_cast<const __half*>(
-            p.packed + p.scale_base + (size_t)l * p.scale_layer_stride + p.scale_kind_off[kind]);
-        if (kind == OP_GATEUP) {
-          sc0 = __half2float(__ldg(scales + vrow0 + 2 * c.tid));
-          sc1 = __half2float(__ldg(scales + vrow0 + 2 * c.tid + 1));
-        } else {
-          sc0 = __half2float(__ldg(scales + vrow));
-        }
-      }
-      if (d.wdtype != W_BF16) { sc0 *= c.xscale; sc1 *= c.xscale; }
-    }
+    if (ps > 0) request_operands(ps);
 
-    if (WDL == W_BF16 || kind == OP_LMHEAD) consume_pass<W_BF16>(c, g, K, red);     // the LM head is always bf16
-    else consume_pass<WDL>(c, g, K, red);
-    if (c.tid == 0 && ps == np - 1) stamp(p, c.cta, task, 7);
+    if (WDL == W_BF16 || kind == OP_LMHEAD) consume_pass<W_BF16>(c, g, kind, gw, K, red, task);     // the LM head is always bf16
+    else consume_pass<WDL>(c, g, kind, gw, K, red, task);
+    if (c.tid == 0 && ps == np - 1) stamp(p, c.cta, task, AMK_TR_REDUCED);
+    if (raddr) {
+      const unsigned rseq = seq_of(p, rtask);
+      if (rraw.y != rseq) {
+        rraw = poll_pair_slow(p, raddr, rseq, rtask);
+        if (rraw.y != rseq) c.bad = true;
+      }
+    }
+    const float resid = __uint_as_float(rraw.x);
+    float sc0 = __half2float(sh0), sc1 = __half2float(sh1);
+    if (d.wdtype != W_BF16) { sc0 *= c.xscale; sc1 *= c.xscale; }
     c.bad = cons_sync_or(c.bad);
     if (c.bad) return false;
 
@@ -589,7 +636,9 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind, int l) {
         }
         gt *= sc0;
         up *= sc1;
-        st_pair(p.m + (vrow0 >> 1) + c.tid, silu_f(gt) * up, my_seq);
+        const float mv = silu_f(gt) * up;
+        st_pair(p.m + (vrow0 >> 1) + c.tid, mv, my_seq);
+        gu_amax = fmaxf(gu_amax, fabsf(mv));
       } else {
         float y = 0.f;
         for (int k = 0; k < g.Wk; k++) y += red[k * R + c.tid];
@@ -609,6 +658,19 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind, int l) {
             break;
         }
       }
+    }
+  }
+  if (WDL != W_BF16 && kind == OP_GATEUP) {
+    // publish this block's max |m|: the down projection scales its integer input by the maximum over all blocks
+    gu_amax = warp_max(gu_amax);
+    if (c.lane == 0) c.sh->cand_val[c.warp] = gu_amax;
+    c.bad = cons_sync_or(c.bad);
+    if (c.bad) return false;
+    if (c.tid == 0 && !drop) {
+      float mx = 0.f;
+#pragma unroll
+      for (int w = 0; w < kConsumerWarps; w++) mx = fmaxf(mx, c.sh->cand_val[w]);
+      st_pair(p.m_amax + c.cta, mx, my_seq);
     }
   }
   if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_COMPUTED);
@@ -1076,6 +1138,21 @@ __global__ void __launch_bounds__(kThreads, 1) amk_decode_kernel(const __grid_co
   __syncthreads();
   const int cta = sh->slot;
   if (cta < 0) return;
+  if (tid < 10) {
+    const int k = tid >> 1, which = tid & 1;
+    const int rows = sh->slice_rows[k];
+    const int np = n_passes(rows);
+    const int R = which ? (np ? pass_rows(rows, np - 1) : 1) : kPassRows;
+    const PassGeom g = pass_geom(R, p.shape[k].K, p.shape[k].wdtype, p.stage_bytes);
+    sh->geom[k][which] = g;
+    sh->step_b[k][which] = g.upt / g.Wr;
+    sh->step_r[k][which] = g.upt % g.Wr;
+    for (int w = 0; w < kConsumerWarps; w++) {
+      sh->wr_of[k][which][w] = (unsigned char)(w % g.Wr);
+      sh->wk_of[k][which][w] = (unsigned char)(w / g.Wr);
+    }
+  }
+  __syncthreads();
 
   if (warp == kConsumerWarps) {
     producer(p, sh, ring, cta, lane);

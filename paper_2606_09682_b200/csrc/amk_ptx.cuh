@@ -111,21 +111,33 @@ __device__ __forceinline__ void mma_s8(int (&c)[4], unsigned a0, unsigned a1, un
 }
 
 // ---- activation elements {value, sequence number}: 8-byte single-copy-atomic accesses at GPU scope -----
+// They carry an L2 evict_last policy: the few hundred KB of activations are touched once per layer while
+// hundreds of MB of weights stream through L2 in between; an 8-byte store to a line that has been evicted
+// makes L2 fetch the line from HBM first, and every reader of the line waits for that.
+__device__ __forceinline__ uint64_t policy_evict_last() {
+  uint64_t pol;
+  asm("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
 __device__ __forceinline__ void st_pair(void* p, float v, unsigned seq) {
   const unsigned long long w = (unsigned long long)__float_as_uint(v) | ((unsigned long long)seq << 32);
-  asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(w) : "memory");
+  asm volatile("st.relaxed.gpu.global.L2::cache_hint.u64 [%0], %1, %2;" ::"l"(p), "l"(w), "l"(policy_evict_last())
+               : "memory");
 }
 __device__ __forceinline__ uint2 ld_pair(const void* p) {
   unsigned long long w;
-  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(w) : "l"(p) : "memory");
+  asm volatile("ld.relaxed.gpu.global.L2::cache_hint.u64 %0, [%1], %2;"
+               : "=l"(w)
+               : "l"(p), "l"(policy_evict_last())
+               : "memory");
   return make_uint2((unsigned)w, (unsigned)(w >> 32));
 }
 // two consecutive elements with one 16-byte load (each 8-byte half is read whole)
 __device__ __forceinline__ uint4 ld_pair2(const void* p) {
   uint4 v;
-  asm volatile("ld.relaxed.gpu.global.v4.u32 {%0,%1,%2,%3}, [%4];"
+  asm volatile("ld.relaxed.gpu.global.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
                : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-               : "l"(p)
+               : "l"(p), "l"(policy_evict_last())
                : "memory");
   return v;
 }
