@@ -317,6 +317,16 @@ __device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* s
       for (int b = tid; b < nblk; b += kConsumerThreads)
         amax = fmaxf(amax, fabsf(read_act(p, res.bad, amax_src + b, seq, src_task)));
     }
+    // norm weights of my lines: requested before the gather, so that their latency (they come from HBM, being
+    // read once per token) is not added to the join's (normed inputs are always held: one batch per thread)
+    unsigned gwt[kBatch];
+    if (normw) {
+#pragma unroll
+      for (int i = 0; i < kBatch; i++) {
+        const int ln = tid + i * kConsumerThreads;
+        gwt[i] = (ln < n2) ? __ldg(reinterpret_cast<const unsigned*>(normw) + ln) : 0u;
+      }
+    }
 #pragma unroll 1
     for (int l0 = tid; l0 < n2 && !amax_src; l0 += kBatch * kConsumerThreads) {
       res.bad |= gather_batch(p, raw, l0, n2, src, seq, src_task, embed_row, cta, task);
@@ -330,7 +340,7 @@ __device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* s
             ss = fmaf(b, b, ss);
             if (embed_row && cta == 0 && (p.flags & AMK_FLAG_DEBUG_HIDDEN))
               reinterpret_cast<float2*>(p.hidden)[ln] = make_float2(a, b);
-            const unsigned gw = __ldg(reinterpret_cast<const unsigned*>(normw) + ln);
+            const unsigned gw = gwt[i];
             a *= bf16_lo(gw);                          // norm weight now, 1/rms after the sum
             b *= bf16_hi(gw);
             raw[i].x = __float_as_uint(a);
