@@ -46,6 +46,8 @@ typedef enum { AMK_W_BF16 = 0, AMK_W_INT8 = 1, AMK_W_INT4 = 2 } amk_wdtype;
 /* amk_config.flags */
 #define AMK_FLAG_DEBUG_HIDDEN 1u /* keep the residual stream after the embedding and after every layer */
 #define AMK_FLAG_TRACE 2u        /* every block stamps the global timer at the stages of every task          */
+#define AMK_FLAG_TRACE_CYCLES 8u /* with AMK_FLAG_TRACE: stamps are the SM's cycle counter, not the global timer (whose
+                                    resolution is a quarter microsecond): only differences within one block mean anything */
 #define AMK_FLAG_MEASURED_SPLIT 4u /* amk_create measures the HBM rate each SM gets and gives each block a share
                                       of every op in proportion (blocks are then identified by SM id).  Off by
                                       default: on B200 it measured no faster than equal shares.             */

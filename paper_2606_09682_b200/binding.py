@@ -22,6 +22,7 @@ AMK_W_BF16, AMK_W_INT8, AMK_W_INT4 = 0, 1, 2
 AMK_FLAG_DEBUG_HIDDEN = 1
 AMK_FLAG_TRACE = 2
 AMK_FLAG_MEASURED_SPLIT = 4
+AMK_FLAG_TRACE_CYCLES = 8
 AMK_TRACE_EVENTS = 12
 AMK_LIN_Q, AMK_LIN_K, AMK_LIN_V, AMK_LIN_O, AMK_LIN_GATE, AMK_LIN_UP, AMK_LIN_DOWN, AMK_LIN_LM_HEAD = range(8)
 KINDS = ("wq", "wk", "wv", "wo", "wgate", "wup", "wdown")

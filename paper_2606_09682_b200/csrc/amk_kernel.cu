@@ -136,7 +136,9 @@ __device__ __forceinline__ void signal_phase(Ctx& c, int phase) {
 
 // One thread stamps the global timer for (task, event) of this block when tracing is on.
 __device__ __forceinline__ void stamp(const KParams& p, int cta, int task, int ev) {
-  if (p.trace) p.trace[((size_t)cta * (5 * p.L + 1) + task) * AMK_TRACE_EVENTS + ev] = globaltimer_ns();
+  if (p.trace)
+    p.trace[((size_t)cta * (5 * p.L + 1) + task) * AMK_TRACE_EVENTS + ev] =
+        (p.flags & AMK_FLAG_TRACE_CYCLES) ? (unsigned long long)clock64() : globaltimer_ns();
 }
 
 __device__ __forceinline__ float warp_sum(float v) {
