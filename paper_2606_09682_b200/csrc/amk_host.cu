@@ -167,6 +167,11 @@ Plan make_plan(const amk_config* c, int n_blocks, const double* weights, bool wi
         }
         base += (size_t)pass_bytes(g);
       }
+      if (op.kind == OP_QKV) {
+        // marker (no bytes) of the layer's attention task: the producer streams the chunk's cache rows here
+        if (with_tiles) tiles->push_back((unsigned long long)(5 * op.layer + 1) << 53);
+        count++;
+      }
     }
   }
   if (with_tiles) (*tile_begin)[n_blocks] = (unsigned)count;
@@ -193,7 +198,7 @@ WorkspaceLayout workspace_layout(const amk_config* c, const Plan& pl) {
   w.o = take(qd * sizeof(ActPair));
   w.m = take(I * sizeof(ActPair));
   w.m_amax = take(kMaxBlocks * sizeof(ActPair));
-  w.part = take((size_t)c->n_q_heads * kMaxChunks * (hd + 2) * 4);
+  w.part = take((size_t)c->n_q_heads * kMaxChunks * (hd + 2) * sizeof(ActPair));
   w.hidden = take((L + 1) * H * 4);
   w.rope = take(S * (hd / 2) * sizeof(float2));
   w.trace = take((size_t)pl.n_blocks * (5 * L + 1) * AMK_TRACE_EVENTS * 8);
@@ -397,7 +402,11 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     if ((size_t)qd > kmax) kmax = qd;
     size_t act = kmax * (cfg->wdtype == AMK_W_BF16 ? 4 : 3);   // bf16 high + low halves, or three int8 digits
     if ((size_t)H * 4 > act) act = (size_t)H * 4;               // the LM head is always bf16
-    const size_t attn_need = ((size_t)n_rep * hd + (size_t)kConsumerWarps * 4 * (hd + 2)) * 4 + (size_t)hd * 4;
+    // attention scratch: q vectors, per-warp partial outputs, the new K / V rows, the scores of the longest chunk
+    int lc_max = 0, c_max = 0;
+    attn_chunks((int)cfg->max_seq, (int)n_blocks, (int)cfg->n_kv_heads, &lc_max, &c_max);
+    const size_t attn_need = ((size_t)n_rep * hd + (size_t)kConsumerWarps * 4 * (hd + 2)) * 4 + (size_t)hd * 4 +
+                             (size_t)n_rep * lc_max * 4;
     if (attn_need > act) act = attn_need;
     act = (act + 127) & ~(size_t)127;
     const uint32_t stage_bytes = h->pl.stage_bytes;
@@ -521,7 +530,7 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     p.x_a = (ActPair*)(h->ws + h->wl.x_a); p.x_b = (ActPair*)(h->ws + h->wl.x_b);
     p.qkv = (ActPair*)(h->ws + h->wl.qkv); p.o = (ActPair*)(h->ws + h->wl.o); p.m = (ActPair*)(h->ws + h->wl.m);
     p.m_amax = (ActPair*)(h->ws + h->wl.m_amax);
-    p.part = (float*)(h->ws + h->wl.part); p.hidden = (float*)(h->ws + h->wl.hidden);
+    p.part = (ActPair*)(h->ws + h->wl.part); p.hidden = (float*)(h->ws + h->wl.hidden);
     p.phase_ctr = (unsigned*)(h->ws + h->wl.phase_ctr); p.group_ctr = (unsigned*)(h->ws + h->wl.group_ctr);
     p.lm_ctr = (unsigned*)(h->ws + h->wl.lm_ctr); p.cand_val = (float*)(h->ws + h->wl.cand_val);
     p.cand_idx = (int*)(h->ws + h->wl.cand_idx); p.next_ws = (int*)(h->ws + h->wl.next_ws);

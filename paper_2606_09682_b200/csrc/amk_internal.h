@@ -89,7 +89,7 @@ struct KParams {
   ActPair* o;
   ActPair* m;
   ActPair* m_amax;                        // [n_blocks] max |m| over each block's rows (integer-weight models)
-  float* part;                            // [nq][kMaxChunks][hd + 2]
+  ActPair* part;                          // [nq][kMaxChunks][hd + 2]: a chunk's max, sum, unnormalised output
   float* hidden;                          // [(L+1)][H]
   unsigned* phase_ctr;                    // [5 L]
   unsigned* group_ctr;                    // [L][nkv]

@@ -758,13 +758,15 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind, int l) {
 // Scores are kept in the log2 domain: q is pre-scaled by log2(e) / sqrt(hd).
 // ------------------------------------------------------------------------------------------------
 template <int HD>
-__device__ __noinline__ bool attn_general(const KParams& p, SmemHeader* sh, unsigned char* xs, int cta, int l, int g,
-                                          int ch, int Lc, int C, bool bad_in);
+__device__ __noinline__ unsigned attn_general(const KParams& p, SmemHeader* sh, unsigned char* xs,
+                                              const unsigned char* ring, int cta, int l, int g, int ch, int Lc, int C,
+                                              bool bad_in, int stage, unsigned parity);
 
 // (Not inlined and called with scalars only: its many accumulators would otherwise push the per-thread
 // state of the task loop out of registers for the whole kernel.)
 template <int HD>
-__device__ __forceinline__ bool attn_task(const KParams& p, SmemHeader* sh, unsigned char* xs, int cta, int l, int g,
+__device__ __forceinline__ bool attn_task(const KParams& p, SmemHeader* sh, unsigned char* xs,
+                                       const unsigned char* ring, int& stage, unsigned& parity, int cta, int l, int g,
                                        int ch, int Lc, int C, bool bad_in) {
   struct {
     const KParams& p;
@@ -832,184 +834,225 @@ __device__ __forceinline__ bool attn_task(const KParams& p, SmemHeader* sh, unsi
       }
     return c.bad;
   }
-  return attn_general<HD>(p, sh, xs, cta, l, g, ch, Lc, C, c.bad);
+  const unsigned r = attn_general<HD>(p, sh, xs, ring, cta, l, g, ch, Lc, C, c.bad, stage, parity);
+  stage = (int)((r >> 1) & 0x7fu);
+  parity = (r >> 8) & 1u;
+  return (r & 1u) != 0u;
 }
 
 // The general case (more than one cache position): kept out of line so that the code every task runs at
 // short contexts stays small; everything it needs is passed as scalars or recomputed.
+// The chunk's cache rows [j0, min(j1, pos)) arrive through the weight ring: the producer streams the K rows,
+// then the V rows, as ring tiles between the QKV and the O projection's weights (see `producer`), so the
+// consumers never wait for a load from HBM.  Three phases, with the chunk's scores in shared memory:
+//   1. scores: the lanes of a group hold 8 dims each of a K row and of four q vectors; dot products are
+//      completed by shuffles;
+//   2. softmax within the chunk: one warp per head takes the maximum, exponentiates in place and sums;
+//   3. P V: lanes cover the 16-byte pieces of a V row, lane groups and warps cover row slices; the slices
+//      are summed by shuffles, then across warps through shared memory.
+// The chunk's (max, sum, unnormalised output) is the final output for a single chunk, else a partial.
+// Returns bad | stage << 1 | parity << 8 (the ring position moves on by the tiles walked).
 template <int HD>
-__device__ __noinline__ bool attn_general(const KParams& p, SmemHeader* sh, unsigned char* xs, int cta, int l, int g,
-                                          int ch, int Lc, int C, bool bad_in) {
+__device__ __noinline__ unsigned attn_general(const KParams& p, SmemHeader* sh, unsigned char* xs,
+                                              const unsigned char* ring, int cta, int l, int g, int ch, int Lc, int C,
+                                              bool bad_in, int stage, unsigned parity) {
   struct {
     SmemHeader* sh;
     int tid, warp, lane, cta;
     bool bad;
   } c{sh, (int)threadIdx.x, (int)(threadIdx.x >> 5), (int)(threadIdx.x & 31), cta, bad_in};
-  constexpr int LG = HD / 8;            // lanes per cache position (8 bf16 each)
-  constexpr int PPW = 32 / LG;          // positions per warp per step
-  constexpr int U = 2;                  // positions in flight per lane group
+  constexpr int NC = HD / 8;            // 16-byte pieces per cache row = lanes per row
+  constexpr int RPW = 32 / NC;          // rows a warp handles at a time
   const int n_rep = p.n_rep;
   const int n_pos = p.pos + 1;
   const int j0 = ch * Lc, j1 = min(n_pos, j0 + Lc);
   const bool owns_new = (j1 == n_pos);
+  const int rows = min(j1, p.pos) - j0;                // rows that come from the cache
+  const int n = j1 - j0;                               // + the new row, held in shared memory
+  const int rpt = p.stage_bytes / (HD * 2);            // cache rows per ring tile
+  const int n_t = (rows + rpt - 1) / rpt;              // ring tiles of K (and again of V)
   float* qs = reinterpret_cast<float*>(xs);            // [n_rep][HD]
   float* wp = qs + n_rep * HD;                         // [warps][4][HD + 2]
   unsigned short* knew = reinterpret_cast<unsigned short*>(wp + (size_t)kConsumerWarps * 4 * (HD + 2));
   unsigned short* vnew = knew + HD;
-  const size_t kvrow = ((size_t)l * p.nkv + g) * p.S;
+  float* S = reinterpret_cast<float*>(vnew + HD);      // [n_rep][Lc] scores, then softmax numerators
+  float* hmax = c.sh->red[0];                          // [n_rep] chunk maximum and sum per head
+  float* hsum = c.sh->red[1];
   const unsigned out_seq = seq_of(p, 5 * l + 1);
   const bool drop = (5 * l + 1 == p.drop_phase && cta == p.drop_block);
-  const int j_new = owns_new ? p.pos : -1;           // this position is taken from shared memory
-
   const int n_hb = (n_rep + 3) >> 2;     // blocks of four q heads
   const int wph = kConsumerWarps / n_hb; // warps per head block
   const int hb = c.warp / wph, wi = c.warp - hb * wph;
-  const int dl = c.lane % LG, sub = c.lane / LG;
-  float m[4], lsum[4], acc[4][8];
+  const bool busy = hb < n_hb;
+  const int dl = c.lane % NC, sub = c.lane / NC;
+  const int S_ = p.n_stages;
+
+  // ---- 1. scores -----------------------------------------------------------------------------------------
+  {
+    float q[4][8];                       // my 8 dims of my block's four q vectors
 #pragma unroll
-  for (int hh = 0; hh < 4; hh++) {
-    m[hh] = -CUDART_INF_F;
-    lsum[hh] = 0.f;
+    for (int hh = 0; hh < 4; hh++) {
+      const int h = min(hb * 4 + hh, n_rep - 1);
 #pragma unroll
-    for (int e = 0; e < 8; e++) acc[hh][e] = 0.f;
+      for (int e = 0; e < 8; e++) q[hh][e] = busy ? qs[h * HD + dl * 8 + e] : 0.f;
+    }
+    auto score_row = [&](const uint4 kq, int t) {
+      const float kf[8] = {bf16_lo(kq.x), bf16_hi(kq.x), bf16_lo(kq.y), bf16_hi(kq.y),
+                           bf16_lo(kq.z), bf16_hi(kq.z), bf16_lo(kq.w), bf16_hi(kq.w)};
+#pragma unroll
+      for (int hh = 0; hh < 4; hh++) {
+        float s = kf[0] * q[hh][0];
+#pragma unroll
+        for (int e = 1; e < 8; e++) s = fmaf(kf[e], q[hh][e], s);
+#pragma unroll
+        for (int o = NC / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (dl == 0 && hb * 4 + hh < n_rep && t >= 0) S[(hb * 4 + hh) * Lc + t] = s;
+      }
+    };
+    for (int k = 0; k < n_t; k++) {
+      if (!c.bad && !wait_mbar(p, &c.sh->full[stage], parity, -1)) c.bad = true;
+      c.bad = __any_sync(0xffffffffu, c.bad) != 0;                         // (shuffles below: the warp stays together)
+      if (busy && !c.bad) {
+        const unsigned char* tile = ring + (size_t)stage * p.stage_bytes;
+        const int r_t = min(rpt, rows - k * rpt);
+        for (int r0 = wi * RPW; r0 < r_t; r0 += wph * RPW) {            // (warp-uniform bounds: shuffles inside)
+          const int r = r0 + sub;
+          const uint4 kq = *reinterpret_cast<const uint4*>(tile + (size_t)min(r, r_t - 1) * (HD * 2) + dl * 16);
+          score_row(kq, r < r_t ? k * rpt + r : -1);
+        }
+      }
+      __syncwarp();
+      if (c.lane == 0 && !c.bad) mbar_arrive(&c.sh->empty[stage]);
+      if (++stage == S_) { stage = 0; parity ^= 1u; }
+    }
+    if (owns_new && busy && wi == 0 && !c.bad)                            // the new row, from shared memory
+      score_row(reinterpret_cast<const uint4*>(knew)[dl], sub == 0 ? n - 1 : -1);
   }
-  if (hb < n_hb && !c.bad) {
-    const uint4* Kb = reinterpret_cast<const uint4*>(p.kcache + kvrow * HD);
-    const uint4* Vb = reinterpret_cast<const uint4*>(p.vcache + kvrow * HD);
-    const int stride = wph * PPW;
-    for (int jb = j0 + wi * PPW + sub; jb - sub - wi * PPW < j1; jb += U * stride) {
-      uint4 kq[U], vq[U];
-#pragma unroll
-      for (int u = 0; u < U; u++) {
-        const int j = min(jb + u * stride, j1 - 1);
-        if (j == j_new) {
-          kq[u] = reinterpret_cast<const uint4*>(knew)[dl];
-          vq[u] = reinterpret_cast<const uint4*>(vnew)[dl];
-        } else {
-          kq[u] = __ldcg(Kb + (size_t)j * LG + dl);
-          vq[u] = __ldcg(Vb + (size_t)j * LG + dl);
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < U; u++) {
-        const bool valid = (jb + u * stride) < j1;
-        const float kf[8] = {bf16_lo(kq[u].x), bf16_hi(kq[u].x), bf16_lo(kq[u].y), bf16_hi(kq[u].y),
-                             bf16_lo(kq[u].z), bf16_hi(kq[u].z), bf16_lo(kq[u].w), bf16_hi(kq[u].w)};
-        const float vf[8] = {bf16_lo(vq[u].x), bf16_hi(vq[u].x), bf16_lo(vq[u].y), bf16_hi(vq[u].y),
-                             bf16_lo(vq[u].z), bf16_hi(vq[u].z), bf16_lo(vq[u].w), bf16_hi(vq[u].w)};
-#pragma unroll
-        for (int hh = 0; hh < 4; hh++) {
-          const int h = hb * 4 + hh;
-          if (h < n_rep) {
-            const float4 q0 = *reinterpret_cast<const float4*>(qs + h * HD + dl * 8);
-            const float4 q1 = *reinterpret_cast<const float4*>(qs + h * HD + dl * 8 + 4);
-            float s = kf[0] * q0.x;
-            s = fmaf(kf[1], q0.y, s);
-            s = fmaf(kf[2], q0.z, s);
-            s = fmaf(kf[3], q0.w, s);
-            s = fmaf(kf[4], q1.x, s);
-            s = fmaf(kf[5], q1.y, s);
-            s = fmaf(kf[6], q1.z, s);
-            s = fmaf(kf[7], q1.w, s);
-#pragma unroll
-            for (int o = LG / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-            if (valid) {
-              const float mn = fmaxf(m[hh], s);
-              const float corr = exp2f(m[hh] - mn);          // m = -inf gives 0
-              const float pw = exp2f(s - mn);
-              lsum[hh] = fmaf(lsum[hh], corr, pw);
-#pragma unroll
-              for (int e = 0; e < 8; e++) acc[hh][e] = fmaf(acc[hh][e], corr, pw * vf[e]);
-              m[hh] = mn;
-            }
-          }
-        }
-      }
+  c.bad = cons_sync_or(c.bad);
+
+  // ---- 2. softmax numerators within the chunk (log2 domain) -----------------------------------------------
+  for (int h = c.warp; h < n_rep && !c.bad; h += kConsumerWarps) {
+    float* sr = S + h * Lc;
+    float mx = -CUDART_INF_F;
+    for (int t = c.lane; t < n; t += 32) mx = fmaxf(mx, sr[t]);
+    mx = warp_max(mx);
+    float z = 0.f;
+    for (int t = c.lane; t < n; t += 32) {
+      const float pw = exp2f(sr[t] - mx);
+      sr[t] = pw;
+      z += pw;
     }
-    // merge the lane groups of the warp
+    z = warp_sum(z);
+    if (c.lane == 0) { hmax[h] = mx; hsum[h] = z; }
+  }
+  c.bad = cons_sync_or(c.bad);
+
+  // ---- 3. P V ---------------------------------------------------------------------------------------------
+  {
+    float acc[4][8];
 #pragma unroll
-    for (int o = LG; o < 32; o <<= 1) {
+    for (int hh = 0; hh < 4; hh++)
+#pragma unroll
+      for (int e = 0; e < 8; e++) acc[hh][e] = 0.f;
+    auto add_row = [&](const uint4 vq, int t) {
+      const float vf[8] = {bf16_lo(vq.x), bf16_hi(vq.x), bf16_lo(vq.y), bf16_hi(vq.y),
+                           bf16_lo(vq.z), bf16_hi(vq.z), bf16_lo(vq.w), bf16_hi(vq.w)};
 #pragma unroll
       for (int hh = 0; hh < 4; hh++) {
-        const float mo = __shfl_xor_sync(0xffffffffu, m[hh], o);
-        const float lo = __shfl_xor_sync(0xffffffffu, lsum[hh], o);
-        const float mn = fmaxf(m[hh], mo);
-        const float a = (m[hh] == -CUDART_INF_F) ? 0.f : exp2f(m[hh] - mn);
-        const float b = (mo == -CUDART_INF_F) ? 0.f : exp2f(mo - mn);
-        lsum[hh] = lsum[hh] * a + lo * b;
+        const float pw = S[min(hb * 4 + hh, n_rep - 1) * Lc + t];
 #pragma unroll
-        for (int e = 0; e < 8; e++) {
-          const float ao = __shfl_xor_sync(0xffffffffu, acc[hh][e], o);
-          acc[hh][e] = acc[hh][e] * a + ao * b;
-        }
-        m[hh] = mn;
+        for (int e = 0; e < 8; e++) acc[hh][e] = fmaf(pw, vf[e], acc[hh][e]);
       }
+    };
+    for (int k = 0; k < n_t; k++) {
+      if (!c.bad && !wait_mbar(p, &c.sh->full[stage], parity, -1)) c.bad = true;
+      c.bad = __any_sync(0xffffffffu, c.bad) != 0;                         // (shuffles below: the warp stays together)
+      if (busy && !c.bad) {
+        const unsigned char* tile = ring + (size_t)stage * p.stage_bytes;
+        const int r_t = min(rpt, rows - k * rpt);
+        for (int r = wi * RPW + sub; r < r_t; r += wph * RPW)
+          add_row(*reinterpret_cast<const uint4*>(tile + (size_t)r * (HD * 2) + dl * 16), k * rpt + r);
+      }
+      __syncwarp();
+      if (c.lane == 0 && !c.bad) mbar_arrive(&c.sh->empty[stage]);
+      if (++stage == S_) { stage = 0; parity ^= 1u; }
     }
-    if (sub == 0) {
+    if (owns_new && busy && wi == 0 && sub == 0 && !c.bad) add_row(reinterpret_cast<const uint4*>(vnew)[dl], n - 1);
+    // sum the lane groups of the warp, then leave the warp's partial in shared memory
 #pragma unroll
-      for (int hh = 0; hh < 4; hh++) {
-        float* w = wp + (size_t)(c.warp * 4 + hh) * (HD + 2);
-        if (dl == 0) { w[0] = m[hh]; w[1] = lsum[hh]; }
+    for (int o = NC; o < 32; o <<= 1)
 #pragma unroll
-        for (int e = 0; e < 8; e++) w[2 + dl * 8 + e] = acc[hh][e];
-      }
+      for (int hh = 0; hh < 4; hh++)
+#pragma unroll
+        for (int e = 0; e < 8; e++) acc[hh][e] += __shfl_xor_sync(0xffffffffu, acc[hh][e], o);
+    if (sub == 0 && busy) {
+#pragma unroll
+      for (int hh = 0; hh < 4; hh++)
+#pragma unroll
+        for (int e = 0; e < 8; e++) wp[(size_t)(c.warp * 4 + hh) * (HD + 2) + 2 + dl * 8 + e] = acc[hh][e];
     }
   }
   c.bad = cons_sync_or(c.bad);
-  if (c.bad) return true;
+  const unsigned ring_pos = ((unsigned)stage << 1) | (parity << 8);
+  if (c.bad) return 1u | ring_pos;
 
-  // merge the warps of each head block, in warp order
+  // sum the warps of each head block, in warp order
   for (int i = c.tid; i < n_rep * HD; i += kConsumerThreads) {
     const int h = i / HD, dd = i - h * HD;
     const int hbb = h >> 2, hh = h & 3;
-    float M = -CUDART_INF_F;
-    for (int w = 0; w < wph; w++) M = fmaxf(M, wp[(size_t)((hbb * wph + w) * 4 + hh) * (HD + 2)]);
-    float Z = 0.f, A = 0.f;
-    for (int w = 0; w < wph; w++) {
-      const float* ww = wp + (size_t)((hbb * wph + w) * 4 + hh) * (HD + 2);
-      const float a = (ww[0] == -CUDART_INF_F) ? 0.f : exp2f(ww[0] - M);
-      Z = fmaf(a, ww[1], Z);
-      A = fmaf(a, ww[2 + dd], A);
-    }
+    float A = 0.f;
+    for (int w = 0; w < wph; w++) A += wp[(size_t)((hbb * wph + w) * 4 + hh) * (HD + 2) + 2 + dd];
     const int hq = g * n_rep + h;
     if (C == 1) {
-      if (!drop) st_pair(p.o + (size_t)hq * HD + dd, A / Z, out_seq);
-    } else {
-      float* pt = p.part + ((size_t)hq * kMaxChunks + ch) * (HD + 2);
-      pt[2 + dd] = A;
-      if (dd == 0) { pt[0] = M; pt[1] = Z; }
+      if (!drop) st_pair(p.o + (size_t)hq * HD + dd, A / hsum[h], out_seq);
+    } else if (!drop) {
+      ActPair* pt = p.part + ((size_t)hq * kMaxChunks + ch) * (HD + 2);
+      st_pair(pt + 2 + dd, A, out_seq);
+      if (dd == 0) { st_pair(pt, hmax[h], out_seq); st_pair(pt + 1, hsum[h], out_seq); }
     }
   }
-  if (C == 1) return c.bad;
+  if (C == 1) return ring_pos;
 
-  // several chunks: the chunk that arrives last for this kv group combines all of them
-  c.bad = cons_sync_or(c.bad);
-  unsigned* gctr = p.group_ctr + (size_t)l * p.nkv + g;
-  if (c.tid == 0) {
-    __threadfence();
-    const unsigned old = atomicAdd(gctr, 1u);
-    __threadfence();
-    c.sh->flag = (old == (unsigned)(C - 1));
-  }
-  c.bad = cons_sync_or(c.bad);
-  if (c.sh->flag && !c.bad) {
-    for (int i = c.tid; i < n_rep * HD; i += kConsumerThreads) {
-      const int h = i / HD, dd = i - h * HD;
-      const int hq = g * n_rep + h;
-      const float* pt = p.part + (size_t)hq * kMaxChunks * (HD + 2);
-      float M = -CUDART_INF_F;
-      for (int k = 0; k < C; k++) M = fmaxf(M, __ldcg(pt + (size_t)k * (HD + 2)));
-      float Z = 0.f, A = 0.f;
-      for (int k = 0; k < C; k++) {
-        const float a = exp2f(__ldcg(pt + (size_t)k * (HD + 2)) - M);
-        Z = fmaf(a, __ldcg(pt + (size_t)k * (HD + 2) + 1), Z);
-        A = fmaf(a, __ldcg(pt + (size_t)k * (HD + 2) + 2 + dd), A);
+  // Several chunks: every chunk's block combines an equal share of the group's n_rep * HD outputs.  The partials
+  // carry sequence numbers like every other activation, so the exchange needs no counter and no fence: gather
+  // what my share needs from all chunks (waiting for it), then combine from shared memory.
+  c.bad = cons_sync_or(c.bad);                       // the warps' partial sums are no longer needed
+  const int E = n_rep * HD;
+  const int e0 = (int)((long long)E * ch / C), e1 = (int)((long long)E * (ch + 1) / C);
+  const int n_out = e1 - e0;
+  float* G = wp;                                     // [n_out][C] outputs' partials, then [heads touched][C][2] = M, Z
+  if (n_out > 0) {
+    const int h_lo = e0 / HD, h_hi = (e1 - 1) / HD;
+    const int n_a = n_out * C, n_mz = (h_hi - h_lo + 1) * C * 2;
+    for (int i = c.tid; i < n_a + n_mz; i += kConsumerThreads) {
+      const ActPair* src;
+      if (i < n_a) {
+        const int o = i / C, k = i - o * C, e = e0 + o;
+        const int h = e / HD, dd = e - h * HD;
+        src = p.part + ((size_t)(g * n_rep + h) * kMaxChunks + k) * (HD + 2) + 2 + dd;
+      } else {
+        const int r = i - n_a, hk = r >> 1, h = h_lo + hk / C, k = hk - (hk / C) * C;
+        src = p.part + ((size_t)(g * n_rep + h) * kMaxChunks + k) * (HD + 2) + (r & 1);
       }
-      if (!drop) st_pair(p.o + (size_t)hq * HD + dd, A / Z, out_seq);
+      G[i] = read_act(p, c.bad, src, out_seq, 5 * l + 1);
     }
-    if (c.tid == 0) *gctr = 0u;          // next used by the next launch
   }
-  return c.bad;
+  c.bad = cons_sync_or(c.bad);
+  if (c.bad) return 1u | ring_pos;
+  for (int o = c.tid; o < n_out; o += kConsumerThreads) {
+    const int e = e0 + o, h = e / HD, dd = e - h * HD;
+    const float* mz = G + n_out * C + (size_t)(h - e0 / HD) * C * 2;
+    float M = -CUDART_INF_F;
+    for (int k = 0; k < C; k++) M = fmaxf(M, mz[2 * k]);
+    float Z = 0.f, A = 0.f;
+    for (int k = 0; k < C; k++) {                      // fixed order: deterministic
+      const float a = exp2f(mz[2 * k] - M);
+      Z = fmaf(a, mz[2 * k + 1], Z);
+      A = fmaf(a, G[o * C + k], A);
+    }
+    if (!drop) st_pair(p.o + (size_t)(g * n_rep + h) * HD + dd, A / Z, out_seq);
+  }
+  return (c.bad ? 1u : 0u) | ring_pos;
 }
 
 template <int HD>
@@ -1027,7 +1070,7 @@ __device__ __forceinline__ bool attention_phase(Ctx& c, int l) {
   if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_JOINED);
   if (t < n_tasks) {
     const int g = t / C, ch = t - g * C;
-    c.bad = attn_task<HD>(p, c.sh, c.xs, c.cta, l, g, ch, Lc, C, c.bad);
+    c.bad = attn_task<HD>(p, c.sh, c.xs, c.ring, c.stage, c.parity, c.cta, l, g, ch, Lc, C, c.bad);
   }
   c.bad = cons_sync_or(c.bad);
   if (c.bad) return false;
@@ -1057,7 +1100,8 @@ __device__ __noinline__ void producer(const KParams& p, SmemHeader* sh, unsigned
   // the first `ahead` tiles are requested right away
   for (unsigned j = 0; j < ahead && begin + j < end; j++) {
     const unsigned long long e = __shfl_sync(0xffffffffu, e_cur, (int)j);
-    if (lane == 0) bulk_prefetch_l2(p.packed + ((e & ((1ull << 40) - 1)) << 4), (unsigned)((e >> 40) & 0x1fffu) << 4);
+    if (lane == 0 && ((e >> 40) & 0x1fffu))
+      bulk_prefetch_l2(p.packed + ((e & ((1ull << 40) - 1)) << 4), (unsigned)((e >> 40) & 0x1fffu) << 4);
   }
   for (unsigned base = begin; base < end && ok; base += 32) {
     const int n = (int)min(32u, end - base);
@@ -1067,25 +1111,51 @@ __device__ __noinline__ void producer(const KParams& p, SmemHeader* sh, unsigned
       const int ja = j + (int)ahead;
       const unsigned long long ea = __shfl_sync(0xffffffffu, ja < 32 ? e_cur : e_next, ja & 31);
       if (lane == 0) {
-        if (ahead && base + (unsigned)ja < end)
+        if (ahead && base + (unsigned)ja < end && ((ea >> 40) & 0x1fffu))
           bulk_prefetch_l2(p.packed + ((ea & ((1ull << 40) - 1)) << 4), (unsigned)((ea >> 40) & 0x1fffu) << 4);
         const unsigned long long off = (e & ((1ull << 40) - 1)) << 4;
         const unsigned bytes = (unsigned)((e >> 40) & 0x1fffu) << 4;
         const int task = (int)(e >> 53);
-        if (lap > 0 && !wait_mbar(p, &sh->empty[stage], (lap - 1) & 1u, -2)) ok = 0;
-        if (ok && inflight < S && t >= inflight) {
-          const unsigned tl = t - inflight;          // this older tile must have landed
-          if (!wait_mbar(p, &sh->full[tl % S], (tl / S) & 1u, -2)) ok = 0;
-        }
-        if (ok) {
-          mbar_expect_tx(&sh->full[stage], bytes);
-          bulk_g2s(ring + (size_t)stage * p.stage_bytes, p.packed + off, bytes, &sh->full[stage], pol);
-          if (p.trace) {
-            if (task != cur_task) { stamp(p, cta, task, AMK_TR_PROD_FIRST); cur_task = task; }
-            stamp(p, cta, task, AMK_TR_PROD_LAST);
+        // one ring tile: wait for a free stage (and for an older copy to have landed), then issue the copy
+        auto issue = [&](const unsigned char* src, unsigned nbytes) {
+          if (lap > 0 && !wait_mbar(p, &sh->empty[stage], (lap - 1) & 1u, -2)) ok = 0;
+          if (ok && inflight < S && t >= inflight) {
+            const unsigned tl = t - inflight;          // this older tile must have landed
+            if (!wait_mbar(p, &sh->full[tl % S], (tl / S) & 1u, -2)) ok = 0;
           }
-          t++;
-          if (++stage == S) { stage = 0; lap++; }
+          if (ok) {
+            mbar_expect_tx(&sh->full[stage], nbytes);
+            bulk_g2s(ring + (size_t)stage * p.stage_bytes, src, nbytes, &sh->full[stage], pol);
+            if (p.trace) {
+              if (task != cur_task) { stamp(p, cta, task, AMK_TR_PROD_FIRST); cur_task = task; }
+              stamp(p, cta, task, AMK_TR_PROD_LAST);
+            }
+            t++;
+            if (++stage == S) { stage = 0; lap++; }
+          }
+        };
+        if (bytes) {
+          issue(p.packed + off, bytes);
+        } else if (p.pos > 0) {
+          // Marker of an attention task: stream the cache rows of this block's chunk, K then V, cut into ring
+          // tiles -- the same rows, in the same tiles, that attn_general walks.  (Rows of earlier positions
+          // only: they were written by earlier launches.  The new row stays in the consumers' shared memory.)
+          const int l = task / 5, nblk = (int)gridDim.x;
+          int Lc, C;
+          attn_chunks(p.pos + 1, nblk, p.nkv, &Lc, &C);
+          const int tt = (cta + nblk - (l * 29) % nblk) % nblk;
+          if (tt < p.nkv * C) {
+            const int g = tt / C, ch = tt - g * C;
+            const int j0 = ch * Lc, rows = min(p.pos, j0 + Lc) - j0;
+            const int rpt = p.stage_bytes / (p.hd * 2);
+            const size_t first = (((size_t)l * p.nkv + g) * p.S + j0) * p.hd;      // in elements
+            for (int which = 0; which < 2 && ok; which++) {
+              const unsigned short* cache = which ? p.vcache : p.kcache;
+              for (int r0 = 0; r0 < rows && ok; r0 += rpt)
+                issue(reinterpret_cast<const unsigned char*>(cache + first + (size_t)r0 * p.hd),
+                      (unsigned)(min(rpt, rows - r0) * p.hd * 2));
+            }
+          }
         }
       }
       ok = __shfl_sync(0xffffffffu, ok, 0);
