@@ -66,6 +66,8 @@ enum { AMK_TR_ENTER = 0,      /* consumer warps reach the task                  
        AMK_TR_PASS_BEGIN = 8, /* last pass: epilogue operands requested, tile walk starts               */
        AMK_TR_FIRST_TILE = 9, /* last pass: its first ring tile has landed                              */
        AMK_TR_TILES_DONE = 10,/* last pass: all ring tiles multiplied                                   */
+       /* attention tasks over several positions use 8 = scores done, 9 = softmax done, 10 = P V done (partial
+          published), 7 = all chunks' partials gathered */
        AMK_TR_POLLS = 11      /* NOT a time: requests thread 0 made for its first batch of input lines   */
 };
 

@@ -929,6 +929,7 @@ __device__ __noinline__ unsigned attn_general(const KParams& p, SmemHeader* sh, 
       score_row(reinterpret_cast<const uint4*>(knew)[dl], sub == 0 ? n - 1 : -1);
   }
   c.bad = cons_sync_or(c.bad);
+  if (c.tid == 0) stamp(p, cta, 5 * l + 1, AMK_TR_PASS_BEGIN);
 
   // ---- 2. softmax numerators within the chunk (log2 domain) -----------------------------------------------
   for (int h = c.warp; h < n_rep && !c.bad; h += kConsumerWarps) {
@@ -946,6 +947,7 @@ __device__ __noinline__ unsigned attn_general(const KParams& p, SmemHeader* sh, 
     if (c.lane == 0) { hmax[h] = mx; hsum[h] = z; }
   }
   c.bad = cons_sync_or(c.bad);
+  if (c.tid == 0) stamp(p, cta, 5 * l + 1, AMK_TR_FIRST_TILE);
 
   // ---- 3. P V ---------------------------------------------------------------------------------------------
   {
@@ -995,6 +997,7 @@ __device__ __noinline__ unsigned attn_general(const KParams& p, SmemHeader* sh, 
   c.bad = cons_sync_or(c.bad);
   const unsigned ring_pos = ((unsigned)stage << 1) | (parity << 8);
   if (c.bad) return 1u | ring_pos;
+  if (c.tid == 0) stamp(p, cta, 5 * l + 1, AMK_TR_TILES_DONE);
 
   // sum the warps of each head block, in warp order
   for (int i = c.tid; i < n_rep * HD; i += kConsumerThreads) {
@@ -1039,6 +1042,7 @@ __device__ __noinline__ unsigned attn_general(const KParams& p, SmemHeader* sh, 
   }
   c.bad = cons_sync_or(c.bad);
   if (c.bad) return 1u | ring_pos;
+  if (c.tid == 0) stamp(p, cta, 5 * l + 1, AMK_TR_REDUCED);
   for (int o = c.tid; o < n_out; o += kConsumerThreads) {
     const int e = e0 + o, h = e / HD, dd = e - h * HD;
     const float* mz = G + n_out * C + (size_t)(h - e0 / HD) * C * 2;
