@@ -53,6 +53,21 @@ def test_prefilled_cache_split_k(name, pos):
     dec.close()
 
 
+@pytest.mark.parametrize("name,wdtype", [("mini", "bf16"), ("mini_hd128", "int8"), ("mini_ragged", "bf16"), ("mini_wide", "int4")])
+def test_chunk_boundaries_and_last_position(name, wdtype):
+    """Positions around the 32-position chunk boundary -- a last chunk that holds nothing but the new row
+    (pos = 32, 64), chunks that end exactly at the boundary (pos = 31, 63), one position only in the cache
+    (pos = 1) -- and the last position the cache has room for."""
+    shape, dec, model = _setup(name, wdtype, seed=24)
+    tok = inp.make_token(shape, 6)
+    for pos in (1, 31, 32, 33, 63, 64, shape.max_seq - 1):
+        kv_g = inp.make_kv_prefill(shape, 7, pos, device="cuda")
+        kv_c = inp.bits(kv_g).copy()
+        r = gc.compare_step(shape, dec, model, tok, pos, kv_g, kv_c)
+        print(name, wdtype, pos, r)
+    dec.close()
+
+
 def test_deterministic_repeat():
     shape, dec, model = _setup("mini_wide", "bf16", seed=23)
     kv = inp.make_kv_prefill(shape, 6, 77, device="cuda")
