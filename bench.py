@@ -34,6 +34,8 @@ WORKLOADS = {
     "llama3_8b_bf16_pos0": ("llama3_8b", "bf16", 0),
     "llama3_8b_int8_pos0": ("llama3_8b", "int8", 0),
     "llama3_8b_bf16_pos4096": ("llama3_8b", "bf16", 4096),
+    "llama3_8b_int8_pos4096": ("llama3_8b", "int8", 4096),
+    "tinyllama_1b_int8_pos512": ("tinyllama_1b", "int8", 512),
     "tinyllama_1b_bf16_pos0": ("tinyllama_1b", "bf16", 0),
     "tinyllama_1b_int8_pos0": ("tinyllama_1b", "int8", 0),
     "tinyllama_1b_int4_pos0": ("tinyllama_1b", "int4", 0),
@@ -42,7 +44,10 @@ WORKLOADS = {
 }
 DEFAULT_WORKLOAD = "llama3_8b_bf16_pos0"      # the largest single-GPU configuration
 OTHER = ["llama3_8b_int8_pos0", "tinyllama_1b_bf16_pos0", "tinyllama_1b_int8_pos0", "tinyllama_1b_int4_pos0",
-         "smollm2_135m_bf16_pos0", "tinyllama_1b_bf16_pos1024"]
+         "smollm2_135m_bf16_pos0", "tinyllama_1b_bf16_pos1024", "tinyllama_1b_int8_pos512", "llama3_8b_int8_pos4096",
+         "llama3_8b_bf16_pos4096"]
+# device-resident multi-token runs (amk_decode_greedy: the token is fed back on the device): (shape, dtype, steps)
+SUSTAINED = [("smollm2_135m", "bf16", 256), ("tinyllama_1b", "bf16", 256)]
 METRIC = "batch-1 decode us/token; achieved HBM GB/s vs B200 measured peak"
 SEED = 0xA3C0
 
@@ -253,6 +258,32 @@ def run_one(workload, device, steps, warmup, with_cpu):
     return res
 
 
+def run_sustained(name, wd, n_steps, device):
+    """n_steps greedy tokens from position 0 in one call: the launches are queued back to back and every step reads
+    its token from the previous step's output on the device; the KV cache grows as it goes."""
+    from paper_2606_09682_b200 import binding as amk
+    shape = inp.SHAPES[name]
+    w = inp.make_weights(shape, SEED, device=device)
+    wq = amk.quantize_weights(w, wd)
+    dec = amk.Decoder(shape, wq, wd, device=device)
+    del w, wq
+    kv = inp.make_kv_prefill(shape, SEED + 1, 0, device=device)
+    tok = inp.make_token(shape, SEED + 2)
+    dec.amk_decode_greedy(tok, 0, n_steps, kv)          # warm-up (same positions again below)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    toks = dec.amk_decode_greedy(tok, 0, n_steps, kv)
+    e1.record()
+    torch.cuda.synchronize()
+    st, msg = dec.amk_last_status()
+    ms = e0.elapsed_time(e1)
+    out = {"workload": f"{name}_{wd}_greedy{n_steps}", "steps": n_steps, "ms": ms, "us_per_token": ms * 1e3 / n_steps,
+           "tokens_per_s": n_steps / (ms * 1e-3), "status": st, "last_token": int(toks[-1].item())}
+    dec.close()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -401,6 +432,13 @@ def main():
                 except Exception as e:      # a side run must never take the headline line down
                     others.append({"workload": wl, "error": str(e)})
             line["other_configs"] = others
+            sustained = []
+            for sname, swd, n_steps in SUSTAINED:
+                try:
+                    sustained.append(run_sustained(sname, swd, n_steps, device))
+                except Exception as e:
+                    sustained.append({"workload": f"{sname}_{swd}_greedy{n_steps}", "error": str(e)})
+            line["sustained"] = sustained
         print(json.dumps(line))
     if world > 1:
         dist.barrier()
