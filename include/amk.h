@@ -240,6 +240,34 @@ amk_status amk_quantize_int4(const void* w_bf16, int64_t rows, int64_t cols, voi
                              void* zero_out, void* cuda_stream);
 
 /*
+ * Static check of the tables a decode step runs from -- the counterpart of the paper's validate() (Section 4,
+ * "The invariants validate() proves", Table 2), for this kernel's tables: the per-block queues of ring tiles,
+ * the row bounds that say which block produces which output rows, and the dependency model of a step.
+ * amk_plan_export writes them as one array of 64-bit words (HOST memory; call with out = NULL to learn the
+ * size); amk_plan_check accepts such an array or rejects it with the reason in msg.  amk_create runs the
+ * check on its own tables and refuses to go on (AMK_ERR_UNSUPPORTED) if it fails, so a rejected plan is never
+ * launched.  Neither call touches the GPU; set cfg->n_blocks when no device is present.
+ *   words: header {magic, blocks, layers, ops, stage bytes, weight bytes, tiles, schedule rows};
+ *          per op {kind, layer, K, rows, unit rows, dtype, region offset, region bytes};
+ *          row bounds [5][blocks + 1]; first tile of each block [blocks + 1];
+ *          tiles {offset / 16 | bytes / 16 << 40 | task << 53} (bytes = 0: attention marker);
+ *          schedule rows {task kind, buffers read, buffers written, flags | buffers read whole << 8}.
+ * What is checked (paper's check -> here):
+ *   referential integrity, capacity caps -> every tile inside the weight area, 16-byte aligned, non-empty, at most
+ *       one ring stage, task ids in range, section sizes consistent with the model;
+ *   wait satisfiability, output reachability -> the row bounds of every GEMV partition its rows (every element a
+ *       task waits for has exactly one producer); every buffer a task reads is written earlier in the step;
+ *   per-SM queue order -> each block's queue is exactly the sequence of tiles its consumers will wait for
+ *       (derived again from the pass geometry), one attention marker per layer after the QKV tiles;
+ *   DAG acyclicity, transitive happens-before, KV ordering -> in the step's fixed task order no task reads ahead
+ *       of its writer, and every overwrite of an activation buffer is ordered, through an all-to-all join, after
+ *       every block's read of the previous content.  (Shared-counter all-join does not arise: joins are
+ *       carried by the data or wait for all blocks.)
+ */
+amk_status amk_plan_export(const amk_config* cfg, uint64_t* out, size_t cap_words, size_t* need_words);
+amk_status amk_plan_check(const amk_config* cfg, const uint64_t* tables, size_t n_words, char* msg, size_t msg_bytes);
+
+/*
  * Greedy token of a logits vector, with scratch memory that is a fixed array inside the library image.
  * The paper has no counterpart of this call: its kernel picks the token inside the decode step, as
  * amk_decode_step does (the LM-head tail).  This is that tail alone -- every block of 2048 elements

@@ -78,6 +78,8 @@ def _load() -> C.CDLL:
         "amk_quantize_int8": (C.c_int, [vp, i64, i64, vp, vp, vp]),
         "amk_quantize_int4": (C.c_int, [vp, i64, i64, vp, vp, vp, vp]),
         "amk_argmax_static": (C.c_int, [vp, i64, vp, C.c_char_p, sz, vp]),
+        "amk_plan_export": (C.c_int, [C.POINTER(amk_config), vp, sz, C.POINTER(sz)]),
+        "amk_plan_check": (C.c_int, [C.POINTER(amk_config), vp, sz, C.c_char_p, sz]),
     }
     for name, (res, args) in sigs.items():
         fn = getattr(lib, name)
@@ -89,7 +91,7 @@ lib = _load()
 EXPORTS = ("amk_status_str", "amk_packed_bytes", "amk_workspace_bytes", "amk_kv_bytes", "amk_create",
            "amk_decode_step", "amk_decode_greedy", "amk_last_status", "amk_plan_info", "amk_debug_hidden",
            "amk_debug_trace", "amk_debug_unpack", "amk_debug_drop_signal", "amk_destroy", "amk_quantize_int8", "amk_quantize_int4",
-           "amk_argmax_static")
+           "amk_argmax_static", "amk_plan_export", "amk_plan_check")
 
 
 class AmkError(RuntimeError):
@@ -167,6 +169,25 @@ def amk_quantize_int4(w: torch.Tensor):
 
 
 AMK_ARGMAX_STATIC_MAX_N = 1 << 20
+
+
+def amk_plan_export(cfg: amk_config):
+    """The tables a step runs from, as a numpy uint64 array (host only; no GPU needed when cfg.n_blocks is set)."""
+    import numpy as np
+    need = C.c_size_t()
+    _check(lib.amk_plan_export(C.byref(cfg), None, 0, C.byref(need)), "amk_plan_export")
+    out = np.zeros(need.value, dtype=np.uint64)
+    _check(lib.amk_plan_export(C.byref(cfg), out.ctypes.data, out.size, C.byref(need)), "amk_plan_export")
+    return out
+
+
+def amk_plan_check(cfg: amk_config, tables):
+    """(status, reason) of the static check over an exported -- or tampered with -- table array."""
+    import numpy as np
+    t = np.ascontiguousarray(tables, dtype=np.uint64)
+    msg = C.create_string_buffer(256)
+    st = lib.amk_plan_check(C.byref(cfg), t.ctypes.data, t.size, msg, 256)
+    return st, msg.value.decode()
 
 
 def amk_argmax_static(x: torch.Tensor, token: torch.Tensor, n: int = -1) -> None:

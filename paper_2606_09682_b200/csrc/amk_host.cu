@@ -49,6 +49,9 @@ struct WorkspaceLayout {
       trace, slice_tab, bounds, smid_tab, calib, tile_begin, tiles, total;
 };
 
+void plan_to_words(const amk_config* cfg, const Plan& pl, const std::vector<unsigned long long>& tiles,
+                   const std::vector<unsigned>& tile_begin, std::vector<uint64_t>& out);
+
 int resolve_blocks(const amk_config* c) {
   if (c->n_blocks) return (int)c->n_blocks;
   int dev = 0, sms = 0;
@@ -387,6 +390,19 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     std::vector<unsigned long long> tiles;
     std::vector<unsigned> tile_begin;
     h->pl = make_plan(cfg, n_blocks, weights.empty() ? nullptr : weights.data(), true, &tiles, &tile_begin);
+    {
+      // the static check of the tables: a rejected plan is never launched
+      std::vector<uint64_t> words;
+      plan_to_words(cfg, h->pl, tiles, tile_begin, words);
+      amk_config ccfg = *cfg;
+      ccfg.n_blocks = (uint32_t)n_blocks;
+      char why[160];
+      if (amk_plan_check(&ccfg, words.data(), words.size(), why, sizeof(why)) != AMK_OK) {
+        snprintf(h->errmsg, sizeof(h->errmsg), "plan rejected by the static check: %s", why);
+        status = AMK_ERR_UNSUPPORTED;
+        goto fail;
+      }
+    }
     h->wl = wl0;
     if (packed_bytes < h->pl.packed_total || tiles.size() * 8 > h->wl.total - h->wl.tiles) {
       snprintf(h->errmsg, sizeof(h->errmsg), "buffers too small for the measured split");
@@ -732,3 +748,276 @@ amk_status amk_quantize_int4(const void* w_bf16, int64_t rows, int64_t cols, voi
 }
 
 }  // extern "C"
+
+// ====================================================================================================
+// Static check of the tables a step runs from (the counterpart of the paper's validate(), Table 2).
+// amk_plan_export writes them as one self-describing array of 64-bit words, amk_plan_check verifies such an
+// array -- the exported one, or one a test has tampered with -- and amk_create checks its own before upload.
+// ====================================================================================================
+namespace {
+
+constexpr unsigned long long kPlanMagic = 0x314E414C504B4D41ull;   // "AMKPLAN1"
+enum { PH_MAGIC, PH_BLOCKS, PH_LAYERS, PH_OPS, PH_STAGE, PH_WEIGHT_BYTES, PH_TILES, PH_SCHED, PH_WORDS };
+constexpr int kOpWords = 8;       // kind, layer, K, rows, unit_rows, wdtype, region_off, region_bytes
+constexpr int kSchedWords = 4;    // task kind, buffers read, buffers written, flags
+// buffers of the schedule model
+enum { B_XA = 1, B_QKV = 2, B_O = 4, B_XB = 8, B_M = 16, B_KVROW = 32, B_OUT = 64, B_MAX = 128, B_PART = 256 };
+// flags: every block takes part / the participants together write the whole of each buffer written /
+// each participant reads the whole of the buffers in `full_reads` (low 16 bits of word 3 >> 8)
+enum { SF_ALL = 1, SF_WRITES_WHOLE = 2 };
+
+struct SchedRow { unsigned kind, reads, writes, flags_fullreads; };
+// The per-layer cycle and the head.  `fullreads` = buffers a participant reads entirely (an all-to-all join);
+// the other reads are of elements the same block wrote (residual rows) or of another task's slice.
+const SchedRow kSchedule[6] = {
+    {0, B_XA, B_QKV, SF_ALL | SF_WRITES_WHOLE | (B_XA << 8)},                                   // QKV
+    {1, B_QKV | B_PART, B_O | B_KVROW | B_PART, SF_WRITES_WHOLE | (B_PART << 8)},               // attention
+    {2, B_O | B_XA, B_XB, SF_ALL | SF_WRITES_WHOLE | (B_O << 8)},                               // O + residual
+    {3, B_XB, B_M | B_MAX, SF_ALL | SF_WRITES_WHOLE | (B_XB << 8)},                             // gate/up
+    {4, B_M | B_MAX | B_XB, B_XA, SF_ALL | SF_WRITES_WHOLE | ((B_M | B_MAX) << 8)},             // down + residual
+    {5, B_XA, B_OUT, SF_ALL | SF_WRITES_WHOLE | (B_XA << 8)},                                   // LM head
+};
+
+struct Reject {
+  char* msg;
+  size_t n;
+  amk_status fail(const char* fmt, long long a = 0, long long b = 0, long long c = 0) {
+    if (msg && n) snprintf(msg, n, fmt, a, b, c);
+    return AMK_ERR_INVALID_ARG;
+  }
+};
+
+// Schedule model: one step = L cycles of rows 0..4, then row 5.  Checked over enough cycles to cross a
+// layer boundary twice.
+amk_status check_schedule(const uint64_t* sw, int n_sched, Reject& rj) {
+  if (n_sched != 6) return rj.fail("schedule: %lld rows, expected 6", n_sched);
+  struct T { unsigned reads, writes, flags, full; };
+  std::vector<T> seq;
+  const int cycles = 3;
+  for (int cyc = 0; cyc <= cycles; cyc++)
+    for (int r = 0; r < 6; r++) {
+      if ((cyc < cycles) != (r < 5)) continue;
+      const uint64_t* w = sw + (size_t)r * kSchedWords;
+      if (w[0] != (unsigned long long)r) return rj.fail("schedule: row %lld holds task kind %lld", r, (long long)w[0]);
+      seq.push_back(T{(unsigned)w[1], (unsigned)w[2], (unsigned)(w[3] & 0xffu), (unsigned)(w[3] >> 8)});
+    }
+  const int n = (int)seq.size();
+  for (int i = 0; i < n; i++) {
+    const T& t = seq[i];
+    if (t.full & ~t.reads) return rj.fail("schedule: task %lld reads whole a buffer it does not read", i);
+    // wait satisfiability: what a task reads was written earlier in the step (or enters the step from outside:
+    // the residual stream from the embedding, cache rows of earlier positions)
+    for (unsigned b = 1; b <= B_PART; b <<= 1) {
+      if (!(t.reads & b) || b == B_KVROW) continue;
+      bool found = (b == B_XA);     // the embedding row
+      for (int j = i; j >= 0 && !found; j--) found = (seq[j].writes & b) != 0 && (j < i || b == B_PART);
+      if (!found) return rj.fail("schedule: task %lld waits for buffer 0x%llx that nothing before it writes", i, b);
+    }
+  }
+  // output reachability
+  if (!(seq[n - 1].writes & B_OUT)) return rj.fail("schedule: no task produces the step's output");
+  // Overwrites: before task W overwrites buffer b, every block that read the previous content must be done.
+  // after[a][c]: every block of task c starts after every block of task a has finished.  It holds if c reads
+  // whole a buffer that a's participants together write (c waits for all of it), and it carries over through
+  // program order on either side when the other task runs on at least the same blocks (on all of them, or it
+  // is the same task), through chains, and to a task whose every block reads part of what the other wrote.
+  std::vector<std::vector<char>> after(n, std::vector<char>(n, 0));
+  for (int a = 0; a < n; a++)
+    for (int c2 = a + 1; c2 < n; c2++)
+      if ((seq[a].flags & SF_WRITES_WHOLE) && (seq[c2].full & seq[a].writes)) after[a][c2] = 1;
+  for (bool changed = true; changed;) {
+    changed = false;
+    for (int a = 0; a < n; a++)
+      for (int c2 = a + 1; c2 < n; c2++) {
+        if (after[a][c2]) continue;
+        bool hold = false;
+        for (int m = a; m <= c2 && !hold; m++) {
+          // a ..(program order).. m => c2, with m on every block a runs on
+          if (m > a && m < c2 && (seq[m].flags & SF_ALL) && after[m][c2]) hold = true;
+          // a => m ..(program order).. c2, with m on every block c2 runs on
+          if (m > a && m < c2 && (seq[m].flags & SF_ALL) && after[a][m]) hold = true;
+          // chains
+          if (m > a && m < c2 && after[a][m] && after[m][c2]) hold = true;
+          // a => m, and every block of c2 reads something m's blocks wrote last (so each waits for one of them)
+          if (m > a && m < c2 && after[a][m]) {
+            for (unsigned b = 1; b <= B_PART && !hold; b <<= 1) {
+              if (!(seq[m].writes & b) || !(seq[c2].reads & b) || b == B_KVROW) continue;
+              bool latest = true;
+              for (int j = m + 1; j < c2; j++) latest = latest && !(seq[j].writes & b);
+              if (latest) hold = true;
+            }
+          }
+        }
+        if (hold) { after[a][c2] = 1; changed = true; }
+      }
+  }
+  for (int w = 0; w < n; w++) {
+    for (unsigned b = 1; b <= B_PART; b <<= 1) {
+      if (!(seq[w].writes & b) || b == B_KVROW || b == B_OUT) continue;
+      int prev = -1;
+      for (int j = w - 1; j >= 0; j--)
+        if (seq[j].writes & b) { prev = j; break; }
+      if (prev < 0) continue;
+      for (int r = prev; r < w; r++) {
+        if (!(seq[r].reads & b)) continue;
+        if (r == prev && b != B_PART) continue;          // (a task does not read what it writes, except the partials)
+        if (!after[r][w])
+          return rj.fail("schedule: task %lld overwrites buffer 0x%llx while task %lld may still read it", w, b, r);
+      }
+    }
+  }
+  return AMK_OK;
+}
+
+}  // namespace
+
+namespace {
+void plan_to_words(const amk_config* cfg, const Plan& pl, const std::vector<unsigned long long>& tiles,
+                   const std::vector<unsigned>& tile_begin, std::vector<uint64_t>& out) {
+  const int nb = pl.n_blocks;
+  const size_t n_ops = pl.ops.size();
+  out.assign(PH_WORDS, 0);
+  out[PH_MAGIC] = kPlanMagic; out[PH_BLOCKS] = (uint64_t)nb; out[PH_LAYERS] = cfg->n_layers; out[PH_OPS] = n_ops;
+  out[PH_STAGE] = pl.stage_bytes; out[PH_TILES] = tiles.size(); out[PH_SCHED] = 6;
+  size_t weight_end = 0;
+  for (size_t i = 0; i < n_ops; i++) {
+    const PlanOp& op = pl.ops[i];
+    size_t bytes = 0;
+    for (int s = 0; s < nb; s++)
+      bytes += (size_t)slice_bytes(slot_slice(pl.bounds[op.kind].data(), op.s.unit_rows, s).rows, op.s.K, op.s.wdtype,
+                                   (int)pl.stage_bytes);
+    const uint64_t row[kOpWords] = {(uint64_t)op.kind, (uint64_t)op.layer, (uint64_t)op.s.K, (uint64_t)op.s.rows,
+                                    (uint64_t)op.s.unit_rows, (uint64_t)op.s.wdtype, (uint64_t)op.region_off, (uint64_t)bytes};
+    out.insert(out.end(), row, row + kOpWords);
+    if (op.region_off + bytes > weight_end) weight_end = op.region_off + bytes;
+  }
+  out[PH_WEIGHT_BYTES] = weight_end;
+  for (int k = 0; k < 5; k++)
+    for (int s = 0; s <= nb; s++) out.push_back((uint64_t)pl.bounds[k][s]);
+  for (int s = 0; s <= nb; s++) out.push_back(tile_begin[s]);
+  for (size_t i = 0; i < tiles.size(); i++) out.push_back(tiles[i]);
+  for (int r = 0; r < 6; r++) {
+    out.push_back(kSchedule[r].kind); out.push_back(kSchedule[r].reads); out.push_back(kSchedule[r].writes);
+    out.push_back(kSchedule[r].flags_fullreads);
+  }
+}
+}  // namespace
+
+extern "C" amk_status amk_plan_export(const amk_config* cfg, uint64_t* out, size_t cap_words, size_t* need_words) {
+  if (!need_words) return AMK_ERR_INVALID_ARG;
+  amk_status st = check_config(cfg);
+  if (st != AMK_OK) return st;
+  std::vector<unsigned long long> tiles;
+  std::vector<unsigned> tile_begin;
+  const Plan pl = make_plan(cfg, resolve_blocks(cfg), nullptr, true, &tiles, &tile_begin);
+  std::vector<uint64_t> words;
+  plan_to_words(cfg, pl, tiles, tile_begin, words);
+  *need_words = words.size();
+  if (!out) return AMK_OK;
+  if (cap_words < words.size()) return AMK_ERR_INVALID_ARG;
+  memcpy(out, words.data(), words.size() * 8);
+  return AMK_OK;
+}
+
+extern "C" amk_status amk_plan_check(const amk_config* cfg, const uint64_t* t, size_t n_words, char* msg,
+                                     size_t msg_bytes) {
+  Reject rj{msg, msg_bytes};
+  if (msg && msg_bytes) msg[0] = 0;
+  if (!t) return rj.fail("no tables");
+  amk_status st = check_config(cfg);
+  if (st != AMK_OK) { rj.fail("configuration rejected"); return st; }
+  // ---- well-formedness of the container ------------------------------------------------------------------
+  if (n_words < PH_WORDS || t[PH_MAGIC] != kPlanMagic) return rj.fail("not a plan (magic / size)");
+  const long long nb = (long long)t[PH_BLOCKS], L = (long long)t[PH_LAYERS], n_ops = (long long)t[PH_OPS];
+  const long long stage = (long long)t[PH_STAGE], wbytes = (long long)t[PH_WEIGHT_BYTES], n_tiles = (long long)t[PH_TILES];
+  if (nb < 1 || nb > kMaxBlocks) return rj.fail("block count %lld out of range", nb);
+  if (cfg->n_blocks && nb != (long long)cfg->n_blocks) return rj.fail("block count %lld differs from the configuration's", nb);
+  if (L != (long long)cfg->n_layers || n_ops != 4 * L + 1) return rj.fail("layers %lld / ops %lld do not match the model", L, n_ops);
+  if (stage != (long long)stage_bytes_of(cfg)) return rj.fail("stage size %lld differs from the configuration's", stage);
+  if (n_tiles < 0 || n_tiles > (1ll << 32)) return rj.fail("tile count out of range");
+  const size_t need = PH_WORDS + (size_t)n_ops * kOpWords + 5 * ((size_t)nb + 1) + ((size_t)nb + 1) + (size_t)n_tiles +
+                      (size_t)t[PH_SCHED] * kSchedWords;
+  if (t[PH_SCHED] > 64 || need != n_words) return rj.fail("array length %lld, sections add up to %lld", (long long)n_words, (long long)need);
+  const uint64_t* ops = t + PH_WORDS;
+  const uint64_t* bounds = ops + (size_t)n_ops * kOpWords;
+  const uint64_t* tbeg = bounds + 5 * ((size_t)nb + 1);
+  const uint64_t* tiles = tbeg + (size_t)nb + 1;
+  const uint64_t* sched = tiles + (size_t)n_tiles;
+
+  // ---- op table: the model's GEMVs in step order, regions inside the weight area and disjoint -------------
+  const int H = cfg->hidden, I = cfg->mlp, V = cfg->vocab, wd = (int)cfg->wdtype;
+  const int qd = cfg->n_q_heads * cfg->head_dim, kvd = cfg->n_kv_heads * cfg->head_dim;
+  const OpShape want[5] = {{H, qd + 2 * kvd, 1, wd}, {qd, H, 1, wd}, {H, 2 * I, 2, wd}, {I, H, 1, wd}, {H, V, 1, W_BF16}};
+  long long prev_end = 0;
+  for (long long i = 0; i < n_ops; i++) {
+    const uint64_t* o = ops + (size_t)i * kOpWords;
+    const long long kind = (i == n_ops - 1) ? OP_LMHEAD : (i % 4), layer = i / 4;
+    if ((long long)o[0] != kind || (long long)o[1] != layer) return rj.fail("op %lld is not the step's op at that place", i);
+    const OpShape& s = want[kind];
+    if ((long long)o[2] != s.K || (long long)o[3] != s.rows || (long long)o[4] != s.unit_rows || (long long)o[5] != s.wdtype)
+      return rj.fail("op %lld: shape or dtype differs from the model's", i);
+    const long long off = (long long)o[6], bytes = (long long)o[7];
+    if (off < prev_end || (off & 15) || bytes < 0 || off + bytes > wbytes) return rj.fail("op %lld: region [%lld, +%lld) overlaps or leaves the weight area", i, off, bytes);
+    prev_end = off + bytes;
+  }
+  // ---- row bounds: every output row of every GEMV has exactly one producer block --------------------------
+  for (int k = 0; k < 5; k++) {
+    const uint64_t* b = bounds + (size_t)k * (nb + 1);
+    const long long units = want[k].rows / want[k].unit_rows;
+    if (b[0] != 0 || (long long)b[nb] != units) return rj.fail("op kind %lld: row bounds do not span [0, %lld]", k, units);
+    for (long long s = 0; s < nb; s++)
+      if ((long long)b[s + 1] < (long long)b[s]) return rj.fail("op kind %lld: row bounds decrease at block %lld", k, s);
+  }
+  // ---- per-block queues: exactly the tiles the consumers will wait for, in their order ---------------------
+  if (tbeg[0] != 0 || (long long)tbeg[nb] != n_tiles) return rj.fail("tile index does not span the tile list");
+  std::vector<int> bnd(nb + 1);
+  std::vector<long long> slice_off((size_t)nb);
+  for (long long s = 0; s < nb; s++)
+    if ((long long)tbeg[s + 1] < (long long)tbeg[s]) return rj.fail("tile index decreases at block %lld", s);
+  // offsets of each block's slice inside each op's region follow from the bounds
+  std::vector<long long> cursor((size_t)nb);
+  for (long long s = 0; s < nb; s++) cursor[s] = (long long)tbeg[s];
+  for (long long i = 0; i < n_ops; i++) {
+    const uint64_t* o = ops + (size_t)i * kOpWords;
+    const int kind = (int)o[0];
+    const long long layer = (long long)o[1];
+    for (long long s = 0; s <= nb; s++) bnd[s] = (int)bounds[(size_t)kind * (nb + 1) + s];
+    long long acc = 0;
+    for (long long s = 0; s < nb; s++) {
+      slice_off[s] = acc;
+      acc += slice_bytes(slot_slice(bnd.data(), want[kind].unit_rows, (int)s).rows, want[kind].K, want[kind].wdtype, (int)stage);
+    }
+    if (acc != (long long)o[7]) return rj.fail("op %lld: region holds %lld bytes, its slices need %lld", i, (long long)o[7], acc);
+    const long long task = (kind == OP_LMHEAD) ? 5 * L : 5 * layer + (kind == OP_QKV ? 0 : kind + 1);
+    for (long long s = 0; s < nb; s++) {
+      const Slice sl = slot_slice(bnd.data(), want[kind].unit_rows, (int)s);
+      long long base = (long long)o[6] + slice_off[s];
+      for (int ps = 0; ps < n_passes(sl.rows); ps++) {
+        const PassGeom g = pass_geom(pass_rows(sl.rows, ps), want[kind].K, want[kind].wdtype, (int)stage);
+        for (int k = 0; k < g.n_tiles; k++) {
+          const long long o0 = unit_off(g, k * g.upt), o1 = unit_off(g, (k + 1) * g.upt);
+          if (cursor[s] >= (long long)tbeg[s + 1]) return rj.fail("block %lld: queue ends before task %lld's tiles", s, task);
+          const uint64_t e = tiles[cursor[s]++];
+          const long long eoff = (long long)((e & ((1ull << 40) - 1)) << 4), ebytes = (long long)(((e >> 40) & 0x1fffu) << 4);
+          const long long etask = (long long)(e >> 53);
+          if (ebytes <= 0 || ebytes > stage) return rj.fail("block %lld: a tile of %lld bytes (stage %lld)", s, ebytes, stage);
+          if (eoff + ebytes > wbytes) return rj.fail("block %lld: tile [%lld, +%lld) leaves the weight area", s, eoff, ebytes);
+          if (etask != task) return rj.fail("block %lld: tile of task %lld where task %lld is walked", s, etask, task);
+          if (eoff != base + o0 || ebytes != o1 - o0)
+            return rj.fail("block %lld task %lld: tile is not the one the consumers wait for", s, task);
+        }
+        base += pass_bytes(g);
+      }
+      if (kind == OP_QKV) {       // the attention task's marker
+        if (cursor[s] >= (long long)tbeg[s + 1]) return rj.fail("block %lld: queue ends before layer %lld's attention marker", s, layer);
+        const uint64_t e = tiles[cursor[s]++];
+        if (((e >> 40) & 0x1fffu) != 0 || (long long)(e >> 53) != 5 * layer + 1)
+          return rj.fail("block %lld: layer %lld's attention marker is missing or misplaced", s, layer);
+      }
+    }
+  }
+  for (long long s = 0; s < nb; s++)
+    if (cursor[s] != (long long)tbeg[s + 1]) return rj.fail("block %lld: %lld tiles nobody waits for", s, (long long)tbeg[s + 1] - cursor[s]);
+  // ---- the dependency model of a step ------------------------------------------------------------------------
+  return check_schedule(sched, (int)t[PH_SCHED], rj);
+}
