@@ -315,8 +315,22 @@ __device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* s
   if (reduce) {
     float ss = 0.f, amax = 0.f;
     if (amax_src) {
+      // the blocks' maxima are requested before the gather (they were published with the values), looked at after
+      uint2 ar[2] = {make_uint2(0u, seq), make_uint2(0u, seq)};
+#pragma unroll
+      for (int j = 0; j < 2; j++)
+        if (tid + j * kConsumerThreads < nblk) ar[j] = ld_pair(amax_src + tid + j * kConsumerThreads);
       res.bad |= gather_batch(p, raw, tid, n2, src, seq, src_task, embed_row, cta, task);
-      for (int b = tid; b < nblk; b += kConsumerThreads)
+#pragma unroll
+      for (int j = 0; j < 2; j++) {
+        const int b = tid + j * kConsumerThreads;
+        if (b < nblk && ar[j].y != seq) {
+          ar[j] = poll_pair_slow(p, amax_src + b, seq, src_task);
+          if (ar[j].y != seq) res.bad = true;
+        }
+        amax = fmaxf(amax, fabsf(__uint_as_float(ar[j].x)));
+      }
+      for (int b = tid + 2 * kConsumerThreads; b < nblk; b += kConsumerThreads)
         amax = fmaxf(amax, fabsf(read_act(p, res.bad, amax_src + b, seq, src_task)));
     }
     // norm weights of my lines: requested before the gather, so that their latency (they come from HBM, being
