@@ -128,3 +128,20 @@ def test_greedy_loop_equals_single_steps(amk):
     assert torch.equal(kv1, kv2) and torch.equal(last_logits, dec.logits)
     assert dec.amk_last_status()[0] == amk.AMK_OK
     dec.close()
+
+
+def test_knob_search_on_a_small_grid(amk):
+    """The search with the real effects: every point passes the correctness gate (the knobs do not change the
+    arithmetic: logits bit-equal to the default configuration's), no latency is below the floor."""
+    from paper_2606_09682_b200 import autotune as at
+    shape = inp.SHAPES["mini_wide"]
+    w = inp.make_weights(shape, 51, device="cuda")
+    build, correct, measure, release, floor_us = at.gpu_effects(shape, w, "bf16", pos=3)
+    grid = [at.Knobs(16384, 2, 2), at.Knobs(24576, 3, 6), at.Knobs(65536, 2, 2)]
+    res = at.tune(build, correct, measure, release, floor_us, grid=grid, steps=10, ab_rounds=3)
+    assert len(res["trials"]) == 4
+    for t in res["trials"]:
+        assert t.verdict in ("kept", "reverted") or t.verdict.startswith("rejected: build"), t
+        if t.latency_us is not None:
+            assert t.latency_us >= floor_us
+    assert res["best_us"] >= floor_us
