@@ -41,11 +41,13 @@ WORKLOADS = {
     "tinyllama_1b_int4_pos0": ("tinyllama_1b", "int4", 0),
     "tinyllama_1b_bf16_pos1024": ("tinyllama_1b", "bf16", 1024),
     "smollm2_135m_bf16_pos0": ("smollm2_135m", "bf16", 0),
+    "llama32_1b_bf16_pos0": ("llama32_1b", "bf16", 0),
+    "llama32_1b_int8_pos0": ("llama32_1b", "int8", 0),
 }
 DEFAULT_WORKLOAD = "llama3_8b_bf16_pos0"      # the largest single-GPU configuration
 OTHER = ["llama3_8b_int8_pos0", "tinyllama_1b_bf16_pos0", "tinyllama_1b_int8_pos0", "tinyllama_1b_int4_pos0",
          "smollm2_135m_bf16_pos0", "tinyllama_1b_bf16_pos1024", "tinyllama_1b_int8_pos512", "llama3_8b_int8_pos4096",
-         "llama3_8b_bf16_pos4096"]
+         "llama3_8b_bf16_pos4096", "llama32_1b_bf16_pos0", "llama32_1b_int8_pos0"]
 # device-resident multi-token runs (amk_decode_greedy: the token is fed back on the device): (shape, dtype, steps)
 SUSTAINED = [("smollm2_135m", "bf16", 256), ("tinyllama_1b", "bf16", 256)]
 METRIC = "batch-1 decode us/token; achieved HBM GB/s vs B200 measured peak"

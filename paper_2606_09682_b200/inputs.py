@@ -63,6 +63,10 @@ SHAPES: Dict[str, ModelShape] = {
     "tinyllama_1b": ModelShape("tinyllama_1b", 2048, 22, 32, 4, 64, 5632, 32000, 2048, False),
     "llama3_8b": ModelShape("llama3_8b", 4096, 32, 32, 8, 128, 14336, 128256, 8192, False,
                             rope_theta=500000.0),
+    # the paper's 16-layer "b1" shape (Section 5, Tables 7-8: 2997.0 MB of bf16 weights): Llama-3.2-1B dimensions
+    # with an untied LM head
+    "llama32_1b": ModelShape("llama32_1b", 2048, 16, 32, 8, 64, 8192, 128256, 2048, False,
+                             rope_theta=500000.0),
 }
 
 

@@ -86,6 +86,18 @@ def test_tinyllama_shape(amk, wdtype, pos):
     dec.close()
 
 
+@pytest.mark.parametrize("wdtype,pos", [("bf16", 0), ("int8", 0), ("int4", 300)])
+def test_llama32_1b_shape(amk, wdtype, pos):
+    """The paper's 16-layer "b1" shape (Llama-3.2-1B dimensions, untied head): the whole step against the oracle."""
+    shape, w, _, dec = _build(amk, "llama32_1b", wdtype, 0xA3C5)
+    model, _ = gc.oracle_model(shape, w, wdtype)
+    kv_g = inp.make_kv_prefill(shape, 0xA3C5, pos, device="cuda")
+    kv_c = inp.bits(kv_g).copy()
+    r = gc.compare_step(shape, dec, model, inp.make_token(shape, 0xA3C5), pos, kv_g, kv_c)
+    print("llama32_1b", wdtype, pos, r)
+    dec.close()
+
+
 @pytest.mark.parametrize("wdtype,pos", [("bf16", 0), ("bf16", 4096), ("int8", 0), ("int8", 4096)])
 def test_llama3_8b_shape_sampled_layers(amk, wdtype, pos):
     shape, w, wq, dec = _build(amk, "llama3_8b", wdtype, 0xA3C4)
