@@ -113,6 +113,10 @@ __device__ __forceinline__ bool wait_mbar(const KParams& p, uint64_t* bar, unsig
   return wait_mbar_slow(p, bar, parity, kind);
 }
 
+// A step at position 0 with data-carried dependencies has no attention task: the QKV projection's epilogue
+// publishes the attention output and appends the cache rows itself (see gemv_op).
+__device__ __forceinline__ bool single_pos(const KParams& p) { return p.pos == 0 && p.sync_mode != 0; }
+
 // Sequence number carried by everything task `task` publishes in this step (never 0).
 __device__ __forceinline__ unsigned seq_of(const KParams& p, int task) {
   return p.epoch * (unsigned)(5 * p.L + 1) + (unsigned)task + 1u;
@@ -670,7 +674,29 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind, int l) {
         for (int k = 0; k < g.Wk; k++) y += red[k * R + c.tid];
         y *= sc0;
         switch (kind) {
-          case OP_QKV: st_pair(p.qkv + vrow, y, my_seq); break;
+          case OP_QKV:
+            st_pair(p.qkv + vrow, y, my_seq);
+            if (single_pos(p)) {
+              // Position 0: one cache position, softmax weight exactly 1, rotation by angle 0.  The attention
+              // output of every q head of a kv group is the rounded v row, and the rows to append are the
+              // rounded k and v themselves: the thread that owns the element does it all, and the layer has no
+              // attention task (one all-to-all join less on the chain).
+              const int qd = p.nq * p.hd, kvd = p.nkv * p.hd;
+              const int hs = (p.hd == 128) ? 7 : 6;
+              if (vrow >= qd) {
+                const bool is_v = vrow >= qd + kvd;
+                const int e = vrow - qd - (is_v ? kvd : 0);
+                const int g = e >> hs, dd = e & (p.hd - 1);
+                const unsigned short bits = f32_to_bf16_rne(y);
+                (is_v ? p.vcache : p.kcache)[((size_t)l * p.nkv + g) * p.S * p.hd + dd] = bits;
+                if (is_v) {
+                  const unsigned oseq = seq_of(p, 5 * l + 1);
+                  for (int h = g * p.n_rep; h < (g + 1) * p.n_rep; h++)
+                    st_pair(p.o + (size_t)h * p.hd + dd, bf16_lo((unsigned)bits), oseq);
+                }
+              }
+            }
+            break;
           case OP_O: st_pair(p.x_b + vrow, resid + y, my_seq); break;
           case OP_DOWN: {
             const float xn = resid + y;
@@ -1083,6 +1109,7 @@ __device__ __forceinline__ bool attention_phase(Ctx& c, int l) {
   const int t = (c.cta + c.nblk - rot) % c.nblk;
   const int task = 5 * l + 1;
   if (p.sync_mode != 0 && t >= n_tasks) return true;      // nothing to do here and nobody to tell
+  if (single_pos(p)) return true;                         // (the QKV projection has done it all)
   if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_ENTER);
   if (!wait_phase(c, 5 * l + 0)) return false;
   if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_JOINED);
