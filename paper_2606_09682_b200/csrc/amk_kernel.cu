@@ -156,24 +156,8 @@ __device__ __forceinline__ float warp_max(float v) {
   return v;
 }
 
-// Spin until both elements of the line at `addr` carry `seq`; bounded.  On failure the returned line does
-// not carry `seq` (values are returned, not written through a pointer, so callers' arrays stay in registers).
-__device__ __noinline__ uint4 poll_pair2_slow(const KParams& p, const void* addr, unsigned seq, int task) {
-  const unsigned long long t0 = globaltimer_ns();
-  unsigned spins = 0;
-  for (;;) {
-    uint4 v = ld_pair2(addr);
-    if (v.y == seq && v.w == seq) return v;
-    if ((++spins & 15u) == 0u) {
-      bool give_up = ld_relaxed_gpu(&p.status->abort) != 0u;
-      if (!give_up && globaltimer_ns() - t0 > p.timeout_ns) {
-        report_failure(p, (unsigned)AMK_ERR_TIMEOUT, task, v.y == seq ? v.w : v.y, seq);
-        give_up = true;
-      }
-      if (give_up) { v.y = seq + 1u; return v; }
-    }
-  }
-}
+// Spin until the element at `addr` carries `seq`; bounded.  On failure the returned element does not carry `seq`
+// (values are returned, not written through a pointer, so callers' arrays stay in registers).
 __device__ __noinline__ uint2 poll_pair_slow(const KParams& p, const void* addr, unsigned seq, int task) {
   const unsigned long long t0 = globaltimer_ns();
   unsigned spins = 0;
@@ -815,9 +799,6 @@ __device__ __forceinline__ bool attn_task(const KParams& p, SmemHeader* sh, unsi
     int tid, warp, lane, cta;
     bool bad;
   } c{p, sh, xs, (int)threadIdx.x, (int)(threadIdx.x >> 5), (int)(threadIdx.x & 31), cta, bad_in};
-  constexpr int LG = HD / 8;            // lanes per cache position (8 bf16 each)
-  constexpr int PPW = 32 / LG;          // positions per warp per step
-  constexpr int U = 2;                  // positions in flight per lane group
   const int n_rep = p.n_rep, half = HD / 2;
   const int n_pos = p.pos + 1;
   const int j0 = ch * Lc, j1 = min(n_pos, j0 + Lc);
