@@ -98,7 +98,7 @@ def test_llama32_1b_shape(amk, wdtype, pos):
     dec.close()
 
 
-@pytest.mark.parametrize("wdtype,pos", [("bf16", 0), ("bf16", 4096), ("int8", 0), ("int8", 4096)])
+@pytest.mark.parametrize("wdtype,pos", [("bf16", 0), ("bf16", 4096), ("int8", 0), ("int8", 4096), ("int4", 0), ("int4", 2500)])
 def test_llama3_8b_shape_sampled_layers(amk, wdtype, pos):
     shape, w, wq, dec = _build(amk, "llama3_8b", wdtype, 0xA3C4)
     kv_g = inp.make_kv_prefill(shape, 0xA3C4, pos, device="cuda")
