@@ -31,6 +31,7 @@ struct SmemHeader {
   int flag;                          // "this block arrived last" broadcast
   int slot;                          // this block's slot (its share of every op, its tile list)
   int slice_row0[5], slice_rows[5];  // its rows of each op kind
+  int attn_lc, attn_c;               // this step's split-K plan of the attention: chunk length, chunks per kv group
   int pad[1];
   // Pass geometry of each op kind for this block's slice, worked out once at kernel start (it takes a dozen
   // integer divisions, which would otherwise sit on every task's critical path): [kind][0] a full pass of

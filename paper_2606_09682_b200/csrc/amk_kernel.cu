@@ -1083,14 +1083,15 @@ __device__ __noinline__ unsigned attn_general(const KParams& p, SmemHeader* sh, 
 template <int HD>
 __device__ __forceinline__ bool attention_phase(Ctx& c, int l) {
   const KParams& p = c.p;
-  int Lc, C;
-  attn_chunks(p.pos + 1, c.nblk, p.nkv, &Lc, &C);
+  if (single_pos(p)) return true;                         // (the QKV projection has done it all)
+  // (the chunk plan is the same for every layer: worked out once, at kernel start; no divisions here)
+  const int Lc = c.sh->attn_lc, C = c.sh->attn_c;
   const int n_tasks = p.nkv * C;
   const int rot = (l * 29) % c.nblk;
-  const int t = (c.cta + c.nblk - rot) % c.nblk;
+  int t = c.cta + c.nblk - rot;
+  if (t >= c.nblk) t -= c.nblk;
   const int task = 5 * l + 1;
   if (p.sync_mode != 0 && t >= n_tasks) return true;      // nothing to do here and nobody to tell
-  if (single_pos(p)) return true;                         // (the QKV projection has done it all)
   if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_ENTER);
   if (!wait_phase(c, 5 * l + 0)) return false;
   if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_JOINED);
@@ -1246,6 +1247,12 @@ __global__ void __launch_bounds__(kThreads, 1) amk_decode_kernel(const __grid_co
   __syncthreads();
   const int cta = sh->slot;
   if (cta < 0) return;
+  if (tid == 32) {
+    int lc, cc;
+    attn_chunks(p.pos + 1, nblk, p.nkv, &lc, &cc);
+    sh->attn_lc = lc;
+    sh->attn_c = cc;
+  }
   if (tid < 10) {
     const int k = tid >> 1, which = tid & 1;
     const int rows = sh->slice_rows[k];
