@@ -79,8 +79,9 @@ enum { AMK_LIN_Q = 0, AMK_LIN_K = 1, AMK_LIN_V = 2, AMK_LIN_O = 3, AMK_LIN_GATE 
 typedef struct amk_config {
   uint32_t struct_size;      /* = sizeof(amk_config)                                                   */
   uint32_t abi_version;      /* = AMK_ABI_VERSION                                                      */
-  uint32_t hidden;           /* H; multiple of 64 (128 for int4), at most 5632                         */
-  uint32_t n_layers;         /* L                                                                      */
+  uint32_t hidden;           /* H; multiple of 64 (128 for int4); at most 5632: a normed input vector is
+                                gathered in one batch of 16 elements per consumer thread               */
+  uint32_t n_layers;         /* L; at most 409 (a task id is kept in 11 bits)                          */
   uint32_t n_q_heads;        /* multiple of n_kv_heads; n_q_heads / n_kv_heads <= 16                   */
   uint32_t n_kv_heads;
   uint32_t head_dim;         /* 64 or 128                                                              */
@@ -99,9 +100,11 @@ typedef struct amk_config {
   uint32_t stage_bytes;      /* bytes per shared-memory ring stage (multiple of 1024)                  */
   uint32_t n_stages;         /* ring depth                                                             */
   uint32_t max_inflight;     /* bulk copies a block keeps in flight (<= n_stages; 0 = default 3)        */
-  uint32_t sync_mode;        /* 0: activations carry sequence numbers AND every task ends with a release-
-                                increment that the next task's readers acquire-spin on (the paper's counter
-                                model); 1: sequence numbers only (no counters, no fences).  Same results.  */
+  uint32_t sync_mode;        /* 0 = automatic = 1.  1: activations carry sequence numbers, nothing else orders
+                                the tasks (no counters, no fences): the mode every published figure uses.
+                                2: as 1, AND every task ends with a release-increment that the next task's
+                                readers acquire-spin on (the paper's counter model, Section 4), kept so
+                                that its cost can be measured.  Same results in both.                    */
   uint32_t n_blocks;         /* persistent blocks; 0 = one per SM of the current device (148 if there is
                                 no device).  The packed layout depends on it.                          */
   uint32_t l2_ahead;         /* ring tiles the producer requests into L2 beyond the ring (weight prefetch
@@ -172,11 +175,13 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* weights, void* p
  * inside one cooperative launch): embedding of `token`, L decoder layers at position `pos`, final norm,
  * LM head, greedy token.
  *   kv_cache_dev   DEVICE, caller-owned, amk_kv_bytes: K then V, each [L][n_kv_heads][max_seq][head_dim]
- *                  bf16.  Entries [0, pos) must be valid; the step writes slot `pos` of every layer (K after
- *                  the rotation, round-to-nearest-even) and reads [0, pos].
- *   logits_dev     DEVICE float[vocab], may be NULL
- *   next_token_dev DEVICE int32[1], may be NULL; lowest index wins an exact tie
- * Asynchronous: returns after the launch.  Synchronous errors: INVALID_ARG, BAD_POS, BAD_TOKEN, CUDA.
+ *                  bf16, 16-byte aligned (rows are fetched with 16-byte bulk copies).  Entries [0, pos) must
+ *                  be valid; the step writes slot `pos` of every layer (K after the rotation,
+ *                  round-to-nearest-even) and reads [0, pos].
+ *   logits_dev     DEVICE float[vocab], 4-byte aligned, may be NULL
+ *   next_token_dev DEVICE int32[1], 4-byte aligned, may be NULL; lowest index wins an exact tie
+ * Asynchronous: returns after the launch.  Synchronous errors: INVALID_ARG (NULL handle or cache, misaligned
+ * pointer), BAD_POS, BAD_TOKEN, CUDA.
  * A device-side failure (expired wait) is reported by amk_last_status after the stream has been
  * synchronised; outputs of that step are then undefined, and the next step is legal.
  */
@@ -221,6 +226,12 @@ amk_status amk_debug_unpack(amk_handle* h, int layer, int which, void* out_dev, 
  * join `phase`, so every waiter runs into the time limit and the step ends with AMK_ERR_TIMEOUT
  * (nothing traps or hangs).  block < 0 clears the hook. */
 amk_status amk_debug_drop_signal(amk_handle* h, int phase, int block);
+
+/* Test hook for the 32-bit sequence numbers: sets the handle's count of steps launched since its activation
+ * area was last cleared.  Every published activation carries step_count * (5 L + 1) + task + 1; shortly before
+ * that would wrap, a step first clears the activation area on its stream and restarts the count (a handle can
+ * decode for ever).  Setting the count close to 2^32 / (5 L + 1) lets a test cross that point. */
+amk_status amk_debug_set_step_count(amk_handle* h, uint32_t steps);
 
 /* Frees host state only.  The caller's buffers are untouched. */
 amk_status amk_destroy(amk_handle* h);
@@ -274,13 +285,16 @@ amk_status amk_plan_check(const amk_config* cfg, const uint64_t* tables, size_t 
  * publishes its best {value, index}, the block that arrives last reduces them -- for callers that change
  * the logits between the decode step and the choice of the token and want neither a workspace nor an
  * allocation: the call allocates no host or device memory at all.
- *   x      DEVICE in, n floats             token  DEVICE out, one int32 (lowest index among equal maxima)
- *   n      1 .. AMK_ARGMAX_STATIC_MAX_N; larger n returns AMK_ERR_UNSUPPORTED, n < 1 or a NULL pointer
- *          AMK_ERR_INVALID_ARG, a failed runtime call AMK_ERR_CUDA
+ *   x      DEVICE in, n floats             token  DEVICE out, one int32 (lowest index among equal maxima;
+ *          NaN elements are never chosen, and a vector of nothing but NaNs gives index 0)
+ *          Both must be 4-byte-aligned memory of the CURRENT device (the scratch used is that device's).
+ *   n      1 .. AMK_ARGMAX_STATIC_MAX_N; larger n returns AMK_ERR_UNSUPPORTED; n < 1, a NULL, misaligned or
+ *          host / other-device pointer AMK_ERR_INVALID_ARG; a failed runtime call AMK_ERR_CUDA
  *   msg    HOST out, msg_bytes bytes, may be NULL: the reason in words when the status is not AMK_OK
  * The scratch (4352 bytes per device: an arrival counter and 512 candidates) belongs to the library.  The
- * counter must be zero at the start of a call: it is zero when the library is loaded and the kernel puts it
- * back to zero before it ends; the candidates need no initial value.  Because all calls on a device share
+ * counter must be zero when the kernel starts: every call clears it on cuda_stream before its launch (so a
+ * launch that never finished leaves nothing behind) and the kernel puts it back to zero before it ends; the
+ * candidates need no initial value.  Because all calls on a device share
  * the one scratch array, two calls that overlap in time (different streams, or different threads without
  * an order between their streams) race and give wrong tokens: keep the calls of a device in one stream or
  * order them with events.  The first call on each device looks up the scratch address (set-up, a

@@ -13,7 +13,7 @@ from typing import Dict, List, Optional, Sequence
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libamk.so")
+LIB_PATH = os.environ.get("AMK_LIB") or os.path.join(_HERE, "libamk.so")      # AMK_LIB: another build of the library
 
 AMK_ABI_VERSION = 1
 AMK_OK, AMK_ERR_INVALID_ARG, AMK_ERR_UNSUPPORTED, AMK_ERR_CUDA, AMK_ERR_OOM = 0, 1, 2, 3, 4
@@ -74,6 +74,7 @@ def _load() -> C.CDLL:
         "amk_debug_trace": (C.c_int, [vp, vp, sz]),
         "amk_debug_unpack": (C.c_int, [vp, C.c_int, C.c_int, vp, vp, vp, vp]),
         "amk_debug_drop_signal": (C.c_int, [vp, C.c_int, C.c_int]),
+        "amk_debug_set_step_count": (C.c_int, [vp, C.c_uint32]),
         "amk_destroy": (C.c_int, [vp]),
         "amk_quantize_int8": (C.c_int, [vp, i64, i64, vp, vp, vp]),
         "amk_quantize_int4": (C.c_int, [vp, i64, i64, vp, vp, vp, vp]),
@@ -90,7 +91,7 @@ def _load() -> C.CDLL:
 lib = _load()
 EXPORTS = ("amk_status_str", "amk_packed_bytes", "amk_workspace_bytes", "amk_kv_bytes", "amk_create",
            "amk_decode_step", "amk_decode_greedy", "amk_last_status", "amk_plan_info", "amk_debug_hidden",
-           "amk_debug_trace", "amk_debug_unpack", "amk_debug_drop_signal", "amk_destroy", "amk_quantize_int8", "amk_quantize_int4",
+           "amk_debug_trace", "amk_debug_unpack", "amk_debug_drop_signal", "amk_debug_set_step_count", "amk_destroy", "amk_quantize_int8", "amk_quantize_int4",
            "amk_argmax_static", "amk_plan_export", "amk_plan_check")
 
 
@@ -195,8 +196,10 @@ def amk_argmax_static(x: torch.Tensor, token: torch.Tensor, n: int = -1) -> None
     ``n`` overrides the element count handed to the library (for argument-checking tests)."""
     assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous()
     assert token.is_cuda and token.dtype == torch.int32 and token.numel() >= 1
+    assert token.device == x.device, "x and token must live on the same device"
     msg = C.create_string_buffer(256)
-    code = lib.amk_argmax_static(x.data_ptr(), x.numel() if n < 0 else n, token.data_ptr(), msg, 256, _stream())
+    with torch.cuda.device(x.device):          # the library uses the scratch array of the current device
+        code = lib.amk_argmax_static(x.data_ptr(), x.numel() if n < 0 else n, token.data_ptr(), msg, 256, _stream())
     if code != AMK_OK:
         raise AmkError(code, msg.value.decode() or "amk_argmax_static")
 
@@ -325,6 +328,9 @@ class Decoder:
 
     def amk_debug_drop_signal(self, phase: int, block: int) -> None:
         _check(lib.amk_debug_drop_signal(self.h, phase, block), "amk_debug_drop_signal")
+
+    def amk_debug_set_step_count(self, steps: int) -> None:
+        _check(lib.amk_debug_set_step_count(self.h, steps), "amk_debug_set_step_count")
 
     def close(self) -> None:
         if getattr(self, "h", None):

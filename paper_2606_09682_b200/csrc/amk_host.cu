@@ -68,7 +68,8 @@ amk_status check_config(const amk_config* c) {
   if (c->l2_ahead > 33u) return AMK_ERR_INVALID_ARG;
   if (!c->hidden || !c->n_layers || !c->n_q_heads || !c->n_kv_heads || !c->mlp || !c->vocab || !c->max_seq)
     return AMK_ERR_INVALID_ARG;
-  if (c->wdtype > AMK_W_INT4 || c->sync_mode > 1) return AMK_ERR_INVALID_ARG;
+  if (c->wdtype > AMK_W_INT4 || c->sync_mode > 2) return AMK_ERR_INVALID_ARG;
+  if (5ull * c->n_layers + 1 > 2047ull) return AMK_ERR_UNSUPPORTED;      // a tile entry keeps its task in 11 bits
   if (c->n_blocks > (uint32_t)kMaxBlocks) return AMK_ERR_INVALID_ARG;
   if (c->head_dim != 64 && c->head_dim != 128) return AMK_ERR_UNSUPPORTED;
   if (c->n_q_heads % c->n_kv_heads) return AMK_ERR_UNSUPPORTED;
@@ -230,7 +231,7 @@ struct amk_handle {
   unsigned char* packed;
   unsigned char* ws;
   KParams base;            // everything but the per-step fields
-  unsigned epoch;          // steps launched: sequence numbers never repeat
+  unsigned epoch;          // steps launched since the activation area was last cleared (see epoch_would_wrap)
   unsigned ctr_epoch;      // steps since the counters were last zeroed
   cudaStream_t last_stream;
   int drop_phase, drop_block;
@@ -526,7 +527,7 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     KParams& p = h->base;
     p.H = H; p.L = L; p.nq = cfg->n_q_heads; p.nkv = cfg->n_kv_heads; p.hd = hd; p.I = I; p.V = cfg->vocab;
     p.S = cfg->max_seq; p.n_rep = n_rep; p.eps = cfg->rms_eps; p.flags = (int)cfg->flags;
-    p.sync_mode = (int)cfg->sync_mode;
+    p.sync_mode = (cfg->sync_mode == 2) ? 0 : 1;      // kernel: 0 = counter joins as well, 1 = sequence numbers only
     for (int k = 0; k < 5; k++) p.shape[k] = h->pl.shape[k];
     p.packed = h->packed;
     p.tiles = (const unsigned long long*)(h->ws + h->wl.tiles);
@@ -576,8 +577,24 @@ fail:
   return status;
 }
 
+// Sequence numbers are 32-bit: step e's task t publishes e * (5 L + 1) + t + 1.  Before that could wrap (after
+// 2^32 / (5 L + 1) steps: tens of millions), the activation area is cleared on the step's stream -- everything in
+// it then carries sequence number 0, which no task ever waits for -- and the step count starts again.
+static bool epoch_would_wrap(const amk_handle* h) {
+  const unsigned long long per = 5ull * h->cfg.n_layers + 1ull;
+  return ((unsigned long long)h->epoch + 2ull) * per + 2ull > 0xffffffffull;
+}
+
 static amk_status launch_step(amk_handle* h, int32_t token, const int* token_ptr, int32_t pos, void* kv, float* logits,
                               int32_t* next_token, cudaStream_t stream) {
+  if (epoch_would_wrap(h)) {
+    // (stream order puts the clear after every earlier step of this handle and before this one)
+    if (cudaMemsetAsync(h->ws + h->wl.x_a, 0, h->wl.hidden - h->wl.x_a, stream) != cudaSuccess) {
+      snprintf(h->errmsg, sizeof(h->errmsg), "clearing the activation area at the sequence-number wrap failed");
+      return AMK_ERR_CUDA;
+    }
+    h->epoch = 0;
+  }
   KParams p = h->base;
   p.token = token;
   p.token_ptr = token_ptr;
@@ -603,9 +620,15 @@ static amk_status launch_step(amk_handle* h, int32_t token, const int* token_ptr
   return AMK_OK;
 }
 
+// The kernel reads cache rows with 16-byte bulk copies and writes logits / tokens as 4-byte words.
+static bool misaligned(const void* kv, const void* a, const void* b) {
+  return ((uintptr_t)kv & 15u) || ((uintptr_t)a & 3u) || ((uintptr_t)b & 3u);
+}
+
 amk_status amk_decode_step(amk_handle* h, int32_t token, int32_t pos, void* kv_cache_dev, float* logits_dev,
                            int32_t* next_token_dev, void* cuda_stream) {
   if (!h || !kv_cache_dev) return AMK_ERR_INVALID_ARG;
+  if (misaligned(kv_cache_dev, logits_dev, next_token_dev)) return AMK_ERR_INVALID_ARG;
   if (pos < 0 || (uint32_t)pos >= h->cfg.max_seq) return AMK_ERR_BAD_POS;
   if (token < 0 || (uint32_t)token >= h->cfg.vocab) return AMK_ERR_BAD_TOKEN;
   return launch_step(h, token, nullptr, pos, kv_cache_dev, logits_dev, next_token_dev, (cudaStream_t)cuda_stream);
@@ -614,6 +637,7 @@ amk_status amk_decode_step(amk_handle* h, int32_t token, int32_t pos, void* kv_c
 amk_status amk_decode_greedy(amk_handle* h, int32_t first_token, int32_t pos0, int32_t n_steps, void* kv_cache_dev,
                              int32_t* tokens_out_dev, float* logits_dev, void* cuda_stream) {
   if (!h || !kv_cache_dev || !tokens_out_dev || n_steps < 1) return AMK_ERR_INVALID_ARG;
+  if (misaligned(kv_cache_dev, logits_dev, tokens_out_dev)) return AMK_ERR_INVALID_ARG;
   if (pos0 < 0 || (uint64_t)pos0 + (uint64_t)n_steps > h->cfg.max_seq) return AMK_ERR_BAD_POS;
   if (first_token < 0 || (uint32_t)first_token >= h->cfg.vocab) return AMK_ERR_BAD_TOKEN;
   for (int i = 0; i < n_steps; i++) {
@@ -720,6 +744,12 @@ amk_status amk_debug_drop_signal(amk_handle* h, int phase, int block) {
   if (phase < 0 || phase >= 5 * (int)h->cfg.n_layers || block >= (int)h->plan.n_blocks) return AMK_ERR_INVALID_ARG;
   h->drop_phase = phase;
   h->drop_block = block;
+  return AMK_OK;
+}
+
+amk_status amk_debug_set_step_count(amk_handle* h, uint32_t steps) {
+  if (!h) return AMK_ERR_INVALID_ARG;
+  h->epoch = steps;
   return AMK_OK;
 }
 

@@ -76,7 +76,8 @@ struct KParams {
   int token;
   const int* token_ptr;                   // if non-null the token is read from device memory
   int pos;
-  unsigned epoch;                         // step number: sequence numbers never repeat
+  unsigned epoch;                         // steps since the activation area was last cleared (the host clears it
+                                          // before the 32-bit sequence numbers could wrap)
   unsigned ctr_epoch;                     // steps since the counters were last zeroed
   // caller buffers
   unsigned short* kcache;

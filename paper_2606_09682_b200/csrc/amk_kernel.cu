@@ -14,7 +14,7 @@
 //     e * n_blocks) so the two can be measured against each other.
 //   * The matrix-vector products run on the tensor cores (warp-level mma, fragments loaded with ldmatrix
 //     straight from the ring): the activation vector occupies two (bf16: high and low halves) or three
-//     (int8 / int4: base-128 digits) of the eight B columns, so nothing is converted per weight and the
+//     (int8 / int4: base-256 digits) of the eight B columns, so nothing is converted per weight and the
 //     result keeps fp32 / exact-integer accuracy.  A scalar loop needs ~2 instructions per weight; the
 //     traced consumer was 3x slower than the HBM stream with it.
 //   * RMSNorm is folded into the consuming GEMV's prologue, RoPE and the KV append into the attention
@@ -37,7 +37,7 @@ constexpr int kBarCons = 1;                          // named barrier of the con
 constexpr int kOutWarps = (kPassRows + 31) / 32;     // warps that hold a pass's output rows
 constexpr int kBatch = 8;                            // 16-byte activation lines a thread gathers at a time
                                                      // (a normed input must fit one batch per thread)
-constexpr float kDigitScale = 1048575.0f;            // int8 / int4 activations: 3 signed base-128 digits
+constexpr float kDigitScale = 4194303.0f;            // int8 / int4 activations: 3 signed base-256 digits, |X| < 2^22
 
 struct Ctx {
   const KParams& p;
@@ -190,45 +190,41 @@ __device__ __forceinline__ float silu_f(float z) { return z / (1.0f + expf(-z));
 // Prologue of a matrix-vector product: bring the input vector (K elements written by `src_task`, or the
 // embedding row) into shared memory in the form the tensor cores take, with RMSNorm folded in.
 //   bf16 weights: X0[K] = bf16(a), X1[K] = bf16(a - X0): two B columns whose sum is a to ~2^-17.
-//   int8 / int4 : a / scale as three signed base-128 digits D2, D1, D0 (three B columns), exact integers.
+//   int8 / int4 : a / scale as three signed base-256 digits D2, D1, D0 (three B columns), exact integers.
 // ------------------------------------------------------------------------------------------------
 
 // two input elements -> their shared-memory form (line `ln` = elements 2 ln, 2 ln + 1)
+// (this runs between the arrival of the input and the first multiply, so every instruction counts: the
+// hardware's paired fp32 -> bf16 conversion, and byte permutes for the digits)
+__device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi) {      // {bf16(lo), bf16(hi)}, round to nearest even
+  unsigned r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
 template <int WD>
 __device__ __forceinline__ void store_line(unsigned char* xs, int n2, int ln, float a, float b, float inv) {
   if (WD == W_BF16) {
     unsigned* X0 = reinterpret_cast<unsigned*>(xs);
     unsigned* X1 = X0 + n2;
-    const unsigned ha = f32_to_bf16_rne(a), hb = f32_to_bf16_rne(b);
-    const unsigned la = f32_to_bf16_rne(a - __uint_as_float(ha << 16));
-    const unsigned lb = f32_to_bf16_rne(b - __uint_as_float(hb << 16));
-    X0[ln] = ha | (hb << 16);
-    X1[ln] = la | (lb << 16);
-    if (inv > 0.f) {                                   // third column: what the first two still miss
-      unsigned* X2 = X1 + n2;
-      const unsigned ra = f32_to_bf16_rne((a - __uint_as_float(ha << 16)) - __uint_as_float(la << 16));
-      const unsigned rb = f32_to_bf16_rne((b - __uint_as_float(hb << 16)) - __uint_as_float(lb << 16));
-      X2[ln] = ra | (rb << 16);
-    }
+    const unsigned h = pack_bf16x2(a, b);
+    const float ra = a - bf16_lo(h), rb = b - bf16_hi(h);            // exact
+    const unsigned l = pack_bf16x2(ra, rb);
+    X0[ln] = h;
+    X1[ln] = l;
+    if (inv > 0.f)                                                   // third column: what the first two still miss
+      (X1 + n2)[ln] = pack_bf16x2(ra - bf16_lo(l), rb - bf16_hi(l));
   } else {
+    // X = d2 * 65536 + d1 * 256 + d0 with every digit in [-128, 127]: the low byte of X is d0's byte, and
+    // (X + 128) >> 8 carries on with the rest
     unsigned short* D2 = reinterpret_cast<unsigned short*>(xs);
     unsigned short* D1 = D2 + n2;
     unsigned short* D0 = D1 + n2;
-    unsigned d2 = 0, d1 = 0, d0 = 0;
-#pragma unroll
-    for (int e = 0; e < 2; e++) {
-      const int X = __float2int_rn((e ? b : a) * inv);
-      const int e0 = ((X + 64) & 127) - 64;
-      const int X1 = (X - e0) >> 7;
-      const int e1 = ((X1 + 64) & 127) - 64;
-      const int e2 = (X1 - e1) >> 7;
-      d0 |= (unsigned)(e0 & 0xff) << (8 * e);
-      d1 |= (unsigned)(e1 & 0xff) << (8 * e);
-      d2 |= (unsigned)(e2 & 0xff) << (8 * e);
-    }
-    D2[ln] = (unsigned short)d2;
-    D1[ln] = (unsigned short)d1;
-    D0[ln] = (unsigned short)d0;
+    const int xa = __float2int_rn(a * inv), xb = __float2int_rn(b * inv);
+    const int ya = (xa + 128) >> 8, yb = (xb + 128) >> 8;
+    const int za = (ya + 128) >> 8, zb = (yb + 128) >> 8;
+    D0[ln] = (unsigned short)__byte_perm((unsigned)xa, (unsigned)xb, 0x0040);
+    D1[ln] = (unsigned short)__byte_perm((unsigned)ya, (unsigned)yb, 0x0040);
+    D2[ln] = (unsigned short)__byte_perm((unsigned)za, (unsigned)zb, 0x0040);
   }
 }
 
@@ -279,12 +275,72 @@ __device__ __forceinline__ bool gather_batch(const KParams& p, uint4 (&raw)[kBat
 
 struct LoadResult {
   float xscale;      // int8 / int4: scale of the digit representation
+  float rnorm;       // bf16 weights, normed input: 1/rms, to be applied to the outputs (1 otherwise)
   bool bad;
 };
 
-// A vector short enough for one batch per thread (every normed input) is held in registers across the
-// reduction; longer vectors are never normed: they are converted as they arrive (bf16) or read twice
-// (integer inputs need their maximum first).
+// bf16 weights: every line is converted as soon as it has arrived.  RMSNorm's 1/rms is one scalar for the whole
+// vector, so W (r * x * g) = r * (W (x * g)): the lines go to shared memory as x * g while the sum of squares is
+// still being collected, and r is applied to the outputs in the epilogue -- no second pass over the input and no
+// block-wide reduction between the arrival of the input and the first multiply.
+__device__ __forceinline__ LoadResult load_input_bf16(const KParams& p, SmemHeader* sh, unsigned char* xs, int cta, int K,
+                                                      const ActPair* src, unsigned seq, int src_task,
+                                                      const unsigned short* embed_row, const unsigned short* normw,
+                                                      int task) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n2 = K >> 1;                               // lines of two elements
+  LoadResult res{1.0f, 1.0f, false};
+  uint4 raw[kBatch];
+  const float inv3 = (6 * K <= p.act_bytes) ? 1.f : 0.f;     // room for a third bf16 column of the input?
+  // norm weights of my lines: requested before the gather, so that their latency (they come from HBM, being
+  // read once per token) is not added to the join's (a normed input is one batch per thread)
+  unsigned gwt[kBatch];
+  if (normw) {
+#pragma unroll
+    for (int i = 0; i < kBatch; i++) {
+      const int ln = tid + i * kConsumerThreads;
+      gwt[i] = (ln < n2) ? __ldg(reinterpret_cast<const unsigned*>(normw) + ln) : 0u;
+    }
+  }
+  float ss = 0.f;
+#pragma unroll 1
+  for (int l0 = tid; l0 < n2; l0 += kBatch * kConsumerThreads) {
+    res.bad |= gather_batch(p, raw, l0, n2, src, seq, src_task, embed_row, cta, task);
+#pragma unroll
+    for (int i = 0; i < kBatch; i++) {
+      const int ln = l0 + i * kConsumerThreads;
+      if (ln < n2) {
+        float a = __uint_as_float(raw[i].x), b = __uint_as_float(raw[i].z);
+        if (normw) {
+          ss = fmaf(a, a, ss);
+          ss = fmaf(b, b, ss);
+          if (embed_row && cta == 0 && (p.flags & AMK_FLAG_DEBUG_HIDDEN))
+            reinterpret_cast<float2*>(p.hidden)[ln] = make_float2(a, b);
+          a *= bf16_lo(gwt[i]);
+          b *= bf16_hi(gwt[i]);
+        }
+        store_line<W_BF16>(xs, n2, ln, a, b, inv3);
+      }
+    }
+  }
+  if (normw) {
+    ss = warp_sum(ss);
+    if (lane == 0) sh->warp_part[0][warp] = ss;
+  }
+  if (tid == 0) stamp(p, cta, task, AMK_TR_JOINED);
+  res.bad = cons_sync_or(res.bad);
+  if (normw) {
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < kConsumerWarps; w++) tot += sh->warp_part[0][w];
+    res.rnorm = 1.0f / sqrtf(tot / (float)K + p.eps);
+  }
+  return res;
+}
+
+// Integer weights: the input becomes three signed digits of a / scale, and the scale needs the maximum of the
+// whole (normed) vector first.  A vector short enough for one batch per thread (every normed input) is held in
+// registers across the block reduction; the down projection's long input comes with its producers' maxima.
 template <int WD>
 __device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* sh, unsigned char* xs, int cta, int K,
                                                  const ActPair* src, unsigned seq, int src_task,
@@ -292,15 +348,14 @@ __device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* s
                                                  int task, const ActPair* amax_src, int nblk) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n2 = K >> 1;                               // lines of two elements
-  LoadResult res{1.0f, false};
+  LoadResult res{1.0f, 1.0f, false};
   uint4 raw[kBatch];
-  const bool reduce = (normw != nullptr) || (WD != W_BF16);
   const bool held = n2 <= kBatch * kConsumerThreads;
   float r = 1.0f, inv = 0.f;
-  // `amax_src`: the producers of this (integer, un-normed) input also published the maximum of their part, so
-  // the vector need not be read twice: the first batch is requested, the maxima are combined meanwhile.
-  const bool have_first = reduce && (held || amax_src != nullptr);
-  if (reduce) {
+  // `amax_src`: the producers of this (un-normed) input also published the maximum of their part, so the vector
+  // need not be read twice: the first batch is requested, the maxima are combined meanwhile.
+  const bool have_first = held || amax_src != nullptr;
+  {
     float ss = 0.f, amax = 0.f;
     if (amax_src) {
       // the blocks' maxima are requested before the gather (they were published with the values), looked at after
@@ -321,8 +376,7 @@ __device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* s
       for (int b = tid + 2 * kConsumerThreads; b < nblk; b += kConsumerThreads)
         amax = fmaxf(amax, fabsf(read_act(p, res.bad, amax_src + b, seq, src_task)));
     }
-    // norm weights of my lines: requested before the gather, so that their latency (they come from HBM, being
-    // read once per token) is not added to the join's (normed inputs are always held: one batch per thread)
+    // norm weights of my lines: requested before the gather (see load_input_bf16)
     unsigned gwt[kBatch];
     if (normw) {
 #pragma unroll
@@ -364,22 +418,19 @@ __device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* s
     for (int w = 0; w < kConsumerWarps; w++) { tot += sh->warp_part[0][w]; mx = fmaxf(mx, sh->warp_part[1][w]); }
     if (normw) r = 1.0f / sqrtf(tot / (float)K + p.eps);
     mx *= r;
-    if (WD != W_BF16) {
-      inv = mx > 0.f ? kDigitScale / mx : 0.f;
-      res.xscale = mx / kDigitScale;
-    }
+    inv = mx > 0.f ? kDigitScale / mx : 0.f;
+    res.xscale = mx / kDigitScale;
   }
-  if (WD == W_BF16) inv = (6 * K <= p.act_bytes) ? 1.f : 0.f;     // room for a third bf16 column of the input?
+  const float rinv = r * inv;
 #pragma unroll 1
   for (int l0 = tid; l0 < n2; l0 += kBatch * kConsumerThreads) {
     if (!(have_first && l0 == tid)) res.bad |= gather_batch(p, raw, l0, n2, src, seq, src_task, embed_row, cta, task);
 #pragma unroll
     for (int i = 0; i < kBatch; i++) {
       const int ln = l0 + i * kConsumerThreads;
-      if (ln < n2) store_line<WD>(xs, n2, ln, __uint_as_float(raw[i].x) * r, __uint_as_float(raw[i].z) * r, inv);
+      if (ln < n2) store_line<WD>(xs, n2, ln, __uint_as_float(raw[i].x), __uint_as_float(raw[i].z), rinv);
     }
   }
-  if (!reduce && tid == 0) stamp(p, cta, task, AMK_TR_JOINED);
   res.bad = cons_sync_or(res.bad);
   return res;
 }
@@ -502,9 +553,9 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int kind
     y0 = facc[0] + facc[1];                            // (columns not in use are zero; the sum over the quad follows)
     y1 = facc[2] + facc[3];
   } else {
-    // columns 2q and 2q+1 of this lane: digit weights 16384 (col 0), 128 (col 1), 1 (col 2), 0 otherwise
-    const float w0 = (q == 0) ? 16384.f : (q == 1 ? 1.f : 0.f);
-    const float w1 = (q == 0) ? 128.f : 0.f;
+    // columns 2q and 2q+1 of this lane: digit weights 65536 (col 0), 256 (col 1), 1 (col 2), 0 otherwise
+    const float w0 = (q == 0) ? 65536.f : (q == 1 ? 1.f : 0.f);
+    const float w1 = (q == 0) ? 256.f : 0.f;
     if (WD == W_INT8) {
       y0 = w0 * (float)iacc[0] + w1 * (float)iacc[1];
       y1 = w0 * (float)iacc[2] + w1 * (float)iacc[3];
@@ -529,9 +580,13 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int kind
 // ------------------------------------------------------------------------------------------------
 // One matrix-vector product with its fused prologue (gather / RMSNorm) and epilogue.
 // ------------------------------------------------------------------------------------------------
-template <int WDL>
-__device__ __forceinline__ bool gemv_op(Ctx& c, int kind, int l) {
+// LMH: the LM head (always bf16, compiled apart from the per-layer code so that a quantised model's layers carry
+// neither its code nor its registers); otherwise `kind_rt` is one of the four per-layer products, of dtype WDL.
+template <int WDL, bool LMH>
+__device__ __forceinline__ bool gemv_op(Ctx& c, int kind_rt, int l) {
   const KParams& p = c.p;
+  const int kind = LMH ? (int)OP_LMHEAD : kind_rt;
+  constexpr int WD = LMH ? (int)W_BF16 : WDL;
   const OpShape d = p.shape[kind];
   const int task = (kind == OP_LMHEAD) ? 5 * p.L : 5 * l + (kind == OP_QKV ? 0 : kind + 1);
   Slice sl;
@@ -593,15 +648,16 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind, int l) {
   };
   if (np > 0) request_operands(0);
 
+  float rnorm = 1.0f;                                    // bf16 weights, normed input: 1/rms, applied to the outputs
   if (!from_embed && !wait_phase(c, src_task)) return false;
   if (np > 0) {
     const unsigned in_seq = from_embed ? 1u : seq_of(p, src_task);
     const unsigned short* erow = from_embed ? embed_row : nullptr;
-    const LoadResult lr = (WDL == W_BF16 || kind == OP_LMHEAD)
-                              ? load_input<W_BF16>(p, c.sh, c.xs, c.cta, K, src, in_seq, src_task, erow, normw, task,
-                                                   nullptr, c.nblk)
-                              : load_input<WDL>(p, c.sh, c.xs, c.cta, K, src, in_seq, src_task, erow, normw, task,
-                                                kind == OP_DOWN ? p.m_amax : nullptr, c.nblk);
+    LoadResult lr;
+    if (WD == W_BF16) lr = load_input_bf16(p, c.sh, c.xs, c.cta, K, src, in_seq, src_task, erow, normw, task);
+    else lr = load_input<WD>(p, c.sh, c.xs, c.cta, K, src, in_seq, src_task, erow, normw, task,
+                             kind == OP_DOWN ? p.m_amax : nullptr, c.nblk);
+    rnorm = lr.rnorm;
     c.xscale = lr.xscale;
     c.bad = lr.bad;
     if (c.bad) return false;
@@ -624,8 +680,7 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind, int l) {
     const bool outp = c.tid < n_out;
     if (ps > 0) request_operands(ps);
 
-    if (WDL == W_BF16 || kind == OP_LMHEAD) consume_pass<W_BF16>(c, g, kind, gw, K, red, task);     // the LM head is always bf16
-    else consume_pass<WDL>(c, g, kind, gw, K, red, task);
+    consume_pass<WD>(c, g, kind, gw, K, red, task);
     if (c.tid == 0 && ps == np - 1) stamp(p, c.cta, task, AMK_TR_REDUCED);
     if (raddr) {
       const unsigned rseq = seq_of(p, rtask);
@@ -635,7 +690,7 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind, int l) {
       }
     }
     const float resid = __uint_as_float(rraw.x);
-    float sc0 = __half2float(sh0), sc1 = __half2float(sh1);
+    float sc0 = __half2float(sh0) * rnorm, sc1 = __half2float(sh1) * rnorm;
     if (d.wdtype != W_BF16) { sc0 *= c.xscale; sc1 *= c.xscale; }
     c.bad = cons_sync_or(c.bad);
     if (c.bad) return false;
@@ -696,7 +751,7 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind, int l) {
       }
     }
   }
-  if (WDL != W_BF16 && kind == OP_GATEUP) {
+  if (WD != W_BF16 && kind == OP_GATEUP) {
     // publish this block's max |m|: the down projection scales its integer input by the maximum over all blocks
     gu_amax = warp_max(gu_amax);
     if (c.lane == 0) c.sh->cand_val[c.warp] = gu_amax;
@@ -711,7 +766,7 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind, int l) {
   }
   if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_COMPUTED);
 
-  if (kind == OP_LMHEAD) {
+  if (LMH) {
     // block argmax, then the block that arrives last reduces all blocks' candidates
     if (c.warp < kOutWarps) {
 #pragma unroll
@@ -1107,6 +1162,15 @@ __device__ __forceinline__ bool attention_phase(Ctx& c, int l) {
   return true;
 }
 
+// The last task of the step: final norm, LM head, greedy token.  Out of line and with its own context: the
+// per-layer loop above it keeps its registers for the code that runs 4 L times.
+__device__ __noinline__ void lm_head_task(const KParams& p, SmemHeader* sh, unsigned char* xs, unsigned char* ring,
+                                          int cta, int nblk, int stage, unsigned parity, int token) {
+  const int tid = threadIdx.x;
+  Ctx c{p, sh, xs, ring, tid, tid >> 5, tid & 31, cta, nblk, stage, parity, token, 1.0f, false};
+  gemv_op<W_BF16, true>(c, (int)OP_LMHEAD, p.L);
+}
+
 // ------------------------------------------------------------------------------------------------
 // Producer: streams this block's weight tiles, in order, into the ring.  The tile list {offset, bytes,
 // task} was laid out by the host, so the producer only waits for a free stage and issues the copy.
@@ -1279,14 +1343,14 @@ __global__ void __launch_bounds__(kThreads, 1) amk_decode_kernel(const __grid_co
   Ctx c{p, sh, xs, ring, tid, warp, lane, cta, nblk, 0, 0u, token, 1.0f, false};
   // the block's queue: tasks 5 l + {0..4} = QKV, attention, O, gate/up, down of layer l, then the LM head
   // (one call site each, so that the per-thread state stays in registers)
-  const int n_tasks = 5 * p.L + 1;
-  for (int task = 0; task < n_tasks; task++) {
+  const int n_layer_tasks = 5 * p.L;
+  bool ok = true;
+  for (int task = 0; task < n_layer_tasks && ok; task++) {
     const int l = task / 5, k = task - 5 * l;
-    bool ok;
     if (k == 1) ok = attention_phase<HD>(c, l);
-    else ok = gemv_op<WDL>(c, task == n_tasks - 1 ? (int)OP_LMHEAD : (k == 0 ? (int)OP_QKV : k - 1), l);
-    if (!ok) break;
+    else ok = gemv_op<WDL, false>(c, k == 0 ? (int)OP_QKV : k - 1, l);
   }
+  if (ok) lm_head_task(p, sh, xs, ring, cta, nblk, c.stage, c.parity, token);
 }
 
 // Calibration: every block (one per SM, same shared-memory footprint as the decode kernel) streams

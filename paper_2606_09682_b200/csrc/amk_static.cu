@@ -20,8 +20,9 @@ constexpr int kCandBase = 32;                                       // word 0: a
 constexpr int kScratchWords = kCandBase + kMaxBlocks;               // 544 words = 4352 bytes
 static_assert(AMK_ARGMAX_STATIC_MAX_N % kPerBlock == 0, "whole blocks");
 
-// Word 0 counts the blocks that have published their candidate.  It must be zero when a call starts: it is
-// zero when the module is loaded, and the block that arrives last puts it back to zero before it leaves.
+// Word 0 counts the blocks that have published their candidate.  It must be zero when the kernel starts: every
+// call clears it on its own stream before the launch (so a call never inherits a count from a launch that did
+// not run to its end), and the block that arrives last puts it back to zero as well.
 // Words kCandBase + b hold block b's candidate {value bits, index}; they are written before they are read in
 // every call and need no initial value.
 static __device__ __align__(256) unsigned long long scratch[kScratchWords];
@@ -83,7 +84,8 @@ __global__ void __launch_bounds__(kThreads) argmax_static_kernel(const float* __
   __syncthreads();   // sv / si are reused
   block_reduce();
   if (threadIdx.x == 0) {
-    *out = bi;
+    // NaN elements compare false and are never chosen; a vector of nothing but NaNs has no candidate: index 0
+    *out = (bi == 0x7fffffff) ? 0 : bi;
     *(unsigned*)s = 0u;   // the next call starts from zero again
   }
 }
@@ -128,7 +130,30 @@ extern "C" amk_status amk_argmax_static(const float* x, int64_t n, int32_t* toke
       g_scratch_of_device[dev] = ptr;
     }
   }
+  // both buffers must be device memory of the current device: the scratch used is this device's
+  for (int k = 0; k < 2; k++) {
+    cudaPointerAttributes at;
+    const void* q = k ? (const void*)token : (const void*)x;
+    const cudaError_t e = cudaPointerGetAttributes(&at, q);
+    if (e != cudaSuccess) (void)cudaGetLastError();
+    if (e != cudaSuccess || (at.type != cudaMemoryTypeDevice && at.type != cudaMemoryTypeManaged) ||
+        (at.type == cudaMemoryTypeDevice && at.device != dev)) {
+      say(msg, msg_bytes, "amk_argmax_static: argument %lld is not device memory of the current device %lld", k, dev);
+      return AMK_ERR_INVALID_ARG;
+    }
+  }
+  if (((uintptr_t)x | (uintptr_t)token) & 3u) {
+    say(msg, msg_bytes, "amk_argmax_static: pointers must be 4-byte aligned", 0, 0);
+    return AMK_ERR_INVALID_ARG;
+  }
   const int blocks = (int)((n + kPerBlock - 1) / kPerBlock);
+  {
+    const cudaError_t e = cudaMemsetAsync(ptr, 0, sizeof(unsigned long long), (cudaStream_t)cuda_stream);
+    if (e != cudaSuccess) {
+      say(msg, msg_bytes, "amk_argmax_static: clearing the arrival counter failed (error %lld)", (long long)e, 0);
+      return AMK_ERR_CUDA;
+    }
+  }
   argmax_static_kernel<<<blocks, kThreads, 0, (cudaStream_t)cuda_stream>>>(x, (int)n, token, ptr);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {

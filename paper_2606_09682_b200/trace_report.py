@@ -101,7 +101,7 @@ def main():
     a = ap.parse_args()
     shape = inp.SHAPES[a.shape]
     tr = collect(shape, a.wdtype, a.pos, a.cycles, sync_mode=a.sync_mode)
-    print(f"{a.shape} {a.wdtype} pos {a.pos}" + (" (counter joins)" if a.sync_mode == 0 else ""))
+    print(f"{a.shape} {a.wdtype} pos {a.pos}" + (" (counter joins)" if a.sync_mode == 2 else ""))
     report(tr, shape, a.pos, a.cycles)
     torch.cuda.synchronize()
 

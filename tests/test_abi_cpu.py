@@ -89,6 +89,23 @@ def test_size_queries_and_argument_checks(amk):
         cfg = amk.make_config(inp.SHAPES["mini"], "bf16")
         setattr(cfg, field, val)
         assert amk.lib.amk_packed_bytes(C.byref(cfg), C.byref(n)) == amk.AMK_ERR_UNSUPPORTED, field
+    # limits of the plan: a task id is kept in 11 bits; sync_mode is 0 (automatic), 1 or 2
+    cfg = amk.make_config(inp.SHAPES["mini"], "bf16")
+    cfg.n_layers = 410
+    assert amk.lib.amk_packed_bytes(C.byref(cfg), C.byref(n)) == amk.AMK_ERR_UNSUPPORTED
+    cfg = amk.make_config(inp.SHAPES["mini"], "bf16", sync_mode=3)
+    assert amk.lib.amk_packed_bytes(C.byref(cfg), C.byref(n)) == amk.AMK_ERR_INVALID_ARG
+    for mode in (0, 1, 2):
+        cfg = amk.make_config(inp.SHAPES["mini"], "bf16", sync_mode=mode)
+        assert amk.lib.amk_packed_bytes(C.byref(cfg), C.byref(n)) == amk.AMK_OK
+    # amk_create refuses buffers that are not 256-byte aligned before it touches the device
+    cfg = amk.make_config(inp.SHAPES["mini"], "bf16")
+    w = amk.amk_weights()
+    h = C.c_void_p()
+    for packed, ws in ((0x10000100 + 16, 0x20000000), (0x10000100 - 0x100, 0x20000000 + 128)):
+        assert amk.lib.amk_create(C.byref(cfg), C.byref(w), packed, 1 << 30, ws, 1 << 30, None,
+                                  C.byref(h)) == amk.AMK_ERR_INVALID_ARG
+        assert not h.value
     # calls on a NULL handle fail cleanly
     assert amk.lib.amk_decode_step(None, 0, 0, None, None, None, None) == amk.AMK_ERR_INVALID_ARG
     assert amk.lib.amk_destroy(None) == amk.AMK_ERR_INVALID_ARG

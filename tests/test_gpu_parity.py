@@ -70,9 +70,9 @@ def test_chunk_boundaries_and_last_position(name, wdtype):
 
 @pytest.mark.parametrize("name,wdtype", [("mini", "bf16"), ("mini_hd128", "int8"), ("mini_wide", "int4")])
 def test_counter_joins(name, wdtype):
-    """sync_mode 0: the paper's synchronisation model on top -- a release-increment of one counter per task and
+    """sync_mode 2: the paper's synchronisation model on top -- a release-increment of one counter per task and
     an acquire-spin on it before the next (Section 4, "Synchronization model") -- gives the same results."""
-    shape, dec, model = _setup(name, wdtype, seed=25, sync_mode=0)
+    shape, dec, model = _setup(name, wdtype, seed=25, sync_mode=2)
     tok = inp.make_token(shape, 8)
     for pos in (0, 1, 40, 100):
         kv_g = inp.make_kv_prefill(shape, 9, pos, device="cuda")

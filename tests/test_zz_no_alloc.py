@@ -73,3 +73,43 @@ def test_static_argmax_rejects_sizes_beyond_its_scratch(amk):
     amk.amk_argmax_static(x, tok)             # still usable afterwards; all equal -> index 0
     torch.cuda.synchronize()
     assert int(tok.item()) == 0
+
+
+def test_static_argmax_nan_and_infinite_inputs(amk):
+    """NaN elements are never chosen; nothing but NaNs gives index 0; -inf everywhere gives the lowest index."""
+    tok = torch.full((3,), -1, dtype=torch.int32, device="cuda")
+    x = torch.full((5000,), float("nan"), device="cuda")
+    amk.amk_argmax_static(x, tok[0:])
+    x2 = x.clone()
+    x2[4097] = -3.0
+    amk.amk_argmax_static(x2, tok[1:])
+    amk.amk_argmax_static(torch.full((5000,), float("-inf"), device="cuda"), tok[2:])
+    torch.cuda.synchronize()
+    assert tok.tolist() == [0, 4097, 0]
+
+
+def test_static_argmax_allocates_nothing_after_its_first_call(amk):
+    """The point of the entry point: once the per-device set-up has run, a call takes no device memory -- neither
+    through torch's allocator nor from the driver."""
+    x = torch.randn(128256, device="cuda")
+    tok = torch.zeros(1, dtype=torch.int32, device="cuda")
+    amk.amk_argmax_static(x, tok)             # first call on the device: set-up
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    alloc0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    for _ in range(20):
+        amk.amk_argmax_static(x, tok)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert (torch.cuda.memory_allocated(), torch.cuda.memory_reserved()) == (alloc0, reserved0)
+    assert free1 == free0, (free0, free1)
+    assert int(tok.item()) == int(torch.argmax(x).item())
+
+
+def test_static_argmax_rejects_host_memory(amk):
+    import ctypes as C
+    host = torch.zeros(16)
+    tok = torch.zeros(1, dtype=torch.int32, device="cuda")
+    msg = C.create_string_buffer(256)
+    code = amk.lib.amk_argmax_static(host.data_ptr(), 16, tok.data_ptr(), msg, 256, None)
+    assert code == amk.AMK_ERR_INVALID_ARG and b"not device memory" in msg.value
