@@ -135,17 +135,18 @@ def job_value(us_per_step_max: float, replicas: int) -> float:
     return us_per_step_max / replicas
 
 
-def build_decoder(workload: str, device, flags: int = 0):
+def build_decoder(workload: str, device, sync_mode: int = 0):
+    """Decoder of a workload plus what the correctness gate needs afterwards: the bf16 weights of layer 0, the
+    norms, the embedding and the LM head (inputs of the shared seeded generator, never outputs of the CUDA path)."""
     from paper_2606_09682_b200 import binding as amk
     name, wd, pos = WORKLOADS[workload]
     shape = inp.SHAPES[name]
     w = inp.make_weights(shape, SEED, device=device)
     wq = amk.quantize_weights(w, wd)
-    dec = amk.Decoder(shape, wq, wd, flags=flags, device=device)
-    keep = None
-    if flags:      # the parity by-product of the CPU-baseline leg needs layer 0's canonical weights
-        keep = {k: (v[0] if isinstance(v, list) else v) for k, v in wq.items() if k not in ("embed", "lm_head")}
-        keep["embed_row_src"] = w["embed"]
+    dec = amk.Decoder(shape, wq, wd, flags=amk.AMK_FLAG_DEBUG_HIDDEN, sync_mode=sync_mode, device=device)
+    keep = {k: w[k][0] for k in inp.KINDS}
+    keep.update(attn_norm=w["attn_norm"][0], mlp_norm=w["mlp_norm"][0], final_norm=w["final_norm"], embed=w["embed"],
+                lm_head=None if shape.tied else w["lm_head"])
     del w, wq
     torch.cuda.empty_cache()
     kv = inp.make_kv_prefill(shape, SEED, pos, device=device)
@@ -201,40 +202,44 @@ def time_e2e(dec, shape, tok, pos, kv, steps, warmup):
     return dt / steps * 1e6, 4, 4 + 4 * shape.vocab
 
 
-class OracleSample:
-    """CPU oracle on a bounded sample of the workload: one decoder layer (layer 0) plus the LM head, with
-    weights of the workload's shape; microseconds per token = L * t_layer + t_head.
-    With `gpu_ctx` the layer runs on the GPU run's own layer-0 weights and token, which also gives a parity
-    figure against the CUDA path's hidden state after layer 0."""
+WDT = {"bf16": 0, "int8": 1, "int4": 2}
 
-    def __init__(self, shape, wd, pos, gpu_ctx=None):
+
+class OracleSample:
+    """The CPU oracle on a bounded sample of a workload: decoder layer 0 and the LM head, with weights of the
+    workload's shape.  Serves two purposes:
+      * timing (`once`): microseconds per token extrapolated as L * t_layer + t_head;
+      * the correctness gate (`gate`): layer 0 applied to the embedding row must give the CUDA path's residual
+        stream after layer 0, and the LM head applied to the CUDA path's final stream must give its logits and an
+        acceptable greedy token.  No latency is reported without a pass (the paper's methodology, Section 5).
+    With `keep` (from build_decoder) the weights are the GPU run's own seeded bf16 weights, quantised here by the
+    oracle's quantiser; without, a one-layer model of the same shape is generated on the CPU."""
+
+    def __init__(self, shape, wd, pos, keep=None, tok=None, kv_gpu=None):
         from oracle import oracle as orc
-        self.orc, self.shape, self.pos = orc, shape, pos
+        self.orc, self.shape, self.pos, self.wd = orc, shape, pos, wd
         s1 = shape.with_(n_layers=1)
-        wdt = {"bf16": orc.W_BF16, "int8": orc.W_INT8, "int4": orc.W_INT4}[wd]
-        self.hidden_gpu = None
-        if gpu_ctx is None:
+        wdt = WDT[wd]
+        if keep is None:
             w = inp.weights_to_numpy(inp.make_weights(s1, SEED, device="cpu"))
-            wq = orc.quantize_weights(w, wdt, 128)
             tok = inp.make_token(shape, SEED)
         else:
-            keep, tok, self.hidden_gpu = gpu_ctx
-            wq = {}
-            for k, v in keep.items():
-                if k == "embed_row_src":
-                    continue
-                t = v.detach().cpu()
-                arr = t.view(torch.int16).numpy().view(np.uint16) if t.dtype in (torch.bfloat16, torch.float16) else t.numpy()
-                wq[k] = arr if k == "final_norm" else [arr]
-            wq["embed"] = inp.bits(keep["embed_row_src"])
-            wq["lm_head"] = None if shape.tied else wq["embed"]      # any [V][H] bf16 matrix serves the head timing
+            w = {k: [inp.bits(keep[k])] for k in inp.KINDS}
+            w.update(attn_norm=[inp.bits(keep["attn_norm"])], mlp_norm=[inp.bits(keep["mlp_norm"])],
+                     final_norm=inp.bits(keep["final_norm"]), embed=inp.bits(keep["embed"]),
+                     lm_head=None if shape.tied else inp.bits(keep["lm_head"]))
+        wq = orc.quantize_weights(w, wdt, 128)
         self.model = orc.Model(s1, wq, wdtype=wdt, group=128)
         self.kv = np.zeros(orc.kv_elems(s1), dtype=np.uint16)
         if pos > 0:
-            self.kv[:] = inp.bits(inp.make_kv_prefill(s1, SEED, pos, device="cpu"))
+            if kv_gpu is None:
+                self.kv[:] = inp.bits(inp.make_kv_prefill(s1, SEED, pos, device="cpu"))
+            else:       # layer 0's slice of the GPU run's pre-filled cache (a seeded input)
+                L, G, S, hd = shape.n_layers, shape.n_kv_heads, shape.max_seq, shape.head_dim
+                self.kv[:] = inp.bits(kv_gpu.view(2, L, G, S, hd)[:, 0].contiguous()).reshape(-1)
+        self.tok = tok
         self.x0 = (wq["embed"][tok].astype(np.uint32) << 16).view(np.float32)
         self.cores = orc.num_threads()
-        self.parity = None
 
     def once(self) -> float:
         """One sample; returns the microseconds-per-token estimate."""
@@ -243,21 +248,83 @@ class OracleSample:
         t1 = time.perf_counter()
         self.model.head_step(out)
         t2 = time.perf_counter()
-        if self.hidden_gpu is not None and self.parity is None:
-            self.parity = float(np.linalg.norm(self.hidden_gpu[1].astype(np.float64) - out) / np.linalg.norm(out))
         return (self.shape.n_layers * (t1 - t0) + (t2 - t1)) * 1e6
 
+    def gate(self, hidden_gpu, logits_gpu, tok_gpu, rows_gpu):
+        """hidden_gpu [L+1][H], logits_gpu [V], the greedy token and layer 0's appended cache rows [2][n_kv][hd] of
+        one step of the CUDA path."""
+        def rel(a, b):
+            a, b = np.asarray(a, np.float64), np.asarray(b, np.float64)
+            return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-30))
+        x1 = self.model.layer_step(0, self.pos, self.x0, self.kv, rows_pref=rows_gpu)
+        logits_o, _ = self.model.head_step(hidden_gpu[self.shape.n_layers])
+        e_h, e_l = rel(hidden_gpu[1], x1), rel(logits_gpu, logits_o)
+        order = np.argsort(-logits_o, kind="stable")
+        gap = float(logits_o[order[0]] - logits_o[order[1]])
+        tok_ok = (tok_gpu == int(order[0])) if gap > 1e-2 else bool(logits_o[tok_gpu] >= logits_o[order[0]] - 1e-2)
+        ok = bool(np.array_equal(hidden_gpu[0], self.x0) and e_h <= 5e-3 and e_l <= 1e-2 and tok_ok)
+        return {"layer0_hidden_rel_l2_vs_oracle": e_h, "logits_rel_l2_vs_oracle_head": e_l,
+                "argmax": "exact" if gap > 1e-2 else "soft", "token_ok": bool(tok_ok), "pass": ok}
 
-def run_one(workload, device, steps, warmup, with_cpu):
-    from paper_2606_09682_b200 import binding as amk
-    shape, wd, pos, dec, kv, tok, keep = build_decoder(workload, device, amk.AMK_FLAG_DEBUG_HIDDEN if with_cpu else 0)
-    per, total_ms = time_device(dec, tok, pos, kv, steps, warmup)
+
+def gate_and_kernel_time(shape, wd, pos, dec, kv, tok, keep, n_kernel=9):
+    """One more step with the read-backs the gate needs, and the kernel-only time of a few steps."""
+    dec.amk_decode_step(tok, pos, kv)
+    st, msg = dec.amk_last_status()
+    if st != 0:
+        raise RuntimeError("decode step failed: " + msg)
+    hidden = dec.amk_debug_hidden().numpy()
+    logits = dec.logits.cpu().numpy()
+    tok_g = int(dec.next_token.item())
+    L, G, S, hd = shape.n_layers, shape.n_kv_heads, shape.max_seq, shape.head_dim
+    rows = inp.bits(kv.view(2, L, G, S, hd)[:, 0, :, pos, :].contiguous())
+    smp = OracleSample(shape, wd, pos, keep, tok, kv)
+    parity = smp.gate(hidden, logits, tok_g, rows)
+    ks = []
+    for _ in range(n_kernel):
+        dec.amk_decode_step(tok, pos, kv)
+        ks.append(dec.amk_last_kernel_ns() / 1e3)
+    return parity, float(np.median(ks)), smp
+
+
+def run_one(workload, device, steps, warmup, peak, sync_mode=0, evict_l2=False):
+    """A side workload: per-call time (CUDA events), kernel-only time, the correctness gate."""
+    shape, wd, pos, dec, kv, tok, keep = build_decoder(workload, device, sync_mode)
+    if evict_l2:
+        per = time_device_evicted(dec, tok, pos, kv, steps, warmup)
+    else:
+        per, _ = time_device(dec, tok, pos, kv, steps, warmup)
+    parity, kernel_us, _ = gate_and_kernel_time(shape, wd, pos, dec, kv, tok, keep)
     b = inp.streamed_bytes(shape, wd, pos)
-    res = {"workload": workload, "us_per_token": float(np.mean(per)), "median_us": float(np.median(per)),
-           "p10_us": float(np.percentile(per, 10)), "p90_us": float(np.percentile(per, 90)),
-           "total_ms": total_ms, "bytes": b["total"], "plan": dec.plan()}
-    res["shape"], res["wd"], res["pos"], res["dec"], res["kv"], res["tok"], res["keep"] = shape, wd, pos, dec, kv, tok, keep
+    us = float(np.mean(per))
+    ach = b["total"] / (us * 1e-6) / 1e9
+    res = {"workload": workload, "us_per_token": us if parity["pass"] else None, "median_us": float(np.median(per)),
+           "kernel_only_us": kernel_us, "achieved_gbs": ach, "frac": ach / peak, "bytes": b["total"], "parity": parity}
+    dec.close()
+    del dec, kv, keep
+    torch.cuda.empty_cache()
     return res
+
+
+def time_device_evicted(dec, tok, pos, kv, steps, warmup, evict_bytes=512 << 20):
+    """As time_device, but a buffer larger than L2 is written between the steps (outside the timed intervals), so
+    that no step finds weights of the previous one in L2."""
+    flush = torch.empty(evict_bytes, dtype=torch.uint8, device=kv.device)
+    for _ in range(warmup):
+        dec.amk_decode_step(tok, pos, kv)
+    a = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    b = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    torch.cuda.synchronize()
+    for i in range(steps):
+        flush.fill_(i & 0xff)
+        a[i].record()
+        dec.amk_decode_step(tok, pos, kv)
+        b[i].record()
+    torch.cuda.synchronize()
+    st, msg = dec.amk_last_status()
+    if st != 0:
+        raise RuntimeError("decode step failed: " + msg)
+    return np.array([a[i].elapsed_time(b[i]) * 1e3 for i in range(steps)])
 
 
 def run_sustained(name, wd, n_steps, device):
@@ -331,7 +398,9 @@ def main():
                 "steps": len(vals), "warmup": n_warm, "ms_per_step": v / 1e3, "higher_is_better": False,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32 (fp64 accumulators)", "data": "synthetic",
                 "config": config,
-                "cpu_baseline": {"value": v, "unit": "us/token", "cores": cores, "kind": "oracle", "sample": sample},
+                "cpu_baseline": {"value": v, "unit": "us/token", "cores": cores,
+                                 "kind": "oracle (extrapolated: L * t_layer + t_head)", "sample": sample,
+                                 "min": float(np.min(vals)), "median": float(np.median(vals))},
                 "e2e": {"value": v, "unit": "us/token", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
         print(json.dumps(line))
         return
@@ -348,21 +417,18 @@ def main():
     amk_build.build()
 
     sampler = ClockSampler(local_rank)
-    r = None
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    with_cpu = (rank == 0 and world == 1)
-    shape, wd, pos, dec, kv, tok, keep = build_decoder(a.workload, device, 1 if with_cpu else 0)
+    shape, wd, pos, dec, kv, tok, keep = build_decoder(a.workload, device)
     for _ in range(a.warmup):
         dec.amk_decode_step(tok, pos, kv)
     st, msg = dec.amk_last_status()
     if st != 0:
         raise SystemExit("decode step failed: " + msg)
-    hidden_gpu = dec.amk_debug_hidden().numpy() if with_cpu else None
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(a.steps + 1)]
     barrier()
     sampler.start()
@@ -378,8 +444,12 @@ def main():
     per = np.array([ev[i].elapsed_time(ev[i + 1]) * 1e3 for i in range(a.steps)])
     total_ms = ev[0].elapsed_time(ev[a.steps])
     total_ms = max_over_ranks(total_ms, device)
-    e2e_us, h2d, d2h = time_e2e(dec, shape, tok, pos, kv, max(5, a.steps // 4), 3)
+    e2e_us, h2d, d2h = time_e2e(dec, shape, tok, pos, kv, a.steps, 3)
     e2e_us = max_over_ranks(e2e_us, device)
+    # the correctness gate and the kernel-only time, on every rank's own replica
+    parity, kernel_us, smp = gate_and_kernel_time(shape, wd, pos, dec, kv, tok, keep)
+    all_pass = max_over_ranks(0.0 if parity["pass"] else 1.0, device) == 0.0
+    kernel_us = max_over_ranks(kernel_us, device)
 
     if rank == 0:
         peak, peak_src = measured_peak()
@@ -387,14 +457,18 @@ def main():
         us = total_ms * 1e3 / a.steps
         achieved = b["total"] / (us * 1e-6) / 1e9
         plan = dec.plan()
-        line = {"metric": METRIC, "value": job_value(us, world), "unit": "us/token", "n_gpus": world, "steps": a.steps,
+        line = {"metric": METRIC, "value": job_value(us, world) if all_pass else None, "unit": "us/token", "n_gpus": world,
+                "steps": a.steps,
                 "warmup": a.warmup, "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak",
                 "vs_baseline": None, "dtype": wd if wd != "bf16" else "bf16 (fp32 accumulate)", "data": "synthetic",
                 "config": config, "clocks": clocks, "gpu_launches": a.steps,
                 "e2e": {"value": job_value(e2e_us, world), "unit": "us/token", "h2d_bytes_per_step": h2d,
-                        "d2h_bytes_per_step": d2h},
+                        "d2h_bytes_per_step": d2h, "steps": a.steps},
                 "latency_us": {"median": float(np.median(per)), "p10": float(np.percentile(per, 10)),
-                               "p90": float(np.percentile(per, 90))},
+                               "p90": float(np.percentile(per, 90)),
+                               "note": "per call: CUDA events around each launch, launch overhead included"},
+                "kernel_only_us": kernel_us,
+                "parity": parity,
                 "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                              "frac": achieved / peak, "traffic": ncu_traffic(a.workload), "peak_source": peak_src,
                              "algorithmic_bytes": b["total"],
@@ -406,33 +480,37 @@ def main():
         if world > 1:
             line["config"]["note"] = ("replicas only: the path does not shard; value = max-over-ranks step time / "
                                       "replicas, i.e. job-level microseconds per decoded token")
-        if with_cpu:
-            smp = OracleSample(shape, wd, pos, (keep, tok, hidden_gpu))
-            cpu_us = float(np.median([smp.once() for _ in range(3)]))
-            parity = smp.parity if pos == 0 else None
-            line["cpu_baseline"] = {"value": cpu_us, "unit": "us/token", "cores": smp.cores, "kind": "oracle",
-                                    "sample": "decoder layer 0 (the GPU run's own weights and token, 3 repeats) + LM head, "
-                                              "us/token = L * t_layer + t_head"}
-            if parity is not None:
-                line["parity"] = {"layer0_hidden_rel_l2_vs_oracle": parity, "pass": bool(parity <= 5e-3)}
-                if parity > 5e-3:
-                    line["value"] = None        # correctness-gated: no latency without a parity pass
+        if world == 1:
+            smp.once()                                                     # warm-up
+            cpu = [smp.once() for _ in range(5)]
+            line["cpu_baseline"] = {"value": float(np.median(cpu)), "min": float(np.min(cpu)), "unit": "us/token",
+                                    "cores": smp.cores, "kind": "oracle (extrapolated: L * t_layer + t_head)",
+                                    "sample": "decoder layer 0 (the GPU run's own seeded weights and token) + LM head, "
+                                              "1 warm-up + 5 repeats, median; us/token = L * t_layer + t_head"}
         dec.close()
-        del dec, kv, keep
+        del dec, kv, keep, smp
         torch.cuda.empty_cache()
         if world == 1 and not a.no_others:
             others = []
-            for wl in OTHER:
+            n_side, w_side = min(a.steps, 50), max(3, min(a.warmup, 10))
+
+            def side(wl, label=None, **kw):
                 try:
-                    r = run_one(wl, device, min(a.steps, 50), max(3, min(a.warmup, 10)), False)
-                    ach = r["bytes"] / (r["us_per_token"] * 1e-6) / 1e9
-                    others.append({"workload": wl, "us_per_token": r["us_per_token"], "median_us": r["median_us"],
-                                   "achieved_gbs": ach, "frac": ach / peak, "bytes": r["bytes"]})
-                    r["dec"].close()
-                    del r
-                    torch.cuda.empty_cache()
+                    r = run_one(wl, device, n_side, w_side, peak, **kw)
+                    if label:
+                        r["workload"] = label
+                    others.append(r)
                 except Exception as e:      # a side run must never take the headline line down
-                    others.append({"workload": wl, "error": str(e)})
+                    others.append({"workload": label or wl, "error": str(e)})
+
+            for wl in OTHER:
+                side(wl)
+            # SmolLM2-135M streams 270 MB, which partly stays in the 126 MB L2 from step to step: the same workload
+            # with L2 evicted between the steps (a latency below bytes / peak would be a measurement artefact)
+            side("smollm2_135m_bf16_pos0", "smollm2_135m_bf16_pos0_l2_evicted", evict_l2=True)
+            # the paper's synchronisation model on top (release-increment / acquire-spin counters at every join)
+            side("tinyllama_1b_bf16_pos0", "tinyllama_1b_bf16_pos0_counter_joins", sync_mode=2)
+            side("llama3_8b_bf16_pos0", "llama3_8b_bf16_pos0_counter_joins", sync_mode=2)
             line["other_configs"] = others
             sustained = []
             for sname, swd, n_steps in SUSTAINED:

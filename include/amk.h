@@ -227,10 +227,18 @@ amk_status amk_debug_unpack(amk_handle* h, int layer, int which, void* out_dev, 
  * (nothing traps or hangs).  block < 0 clears the hook. */
 amk_status amk_debug_drop_signal(amk_handle* h, int phase, int block);
 
+/* Kernel-only time of the handle's last step, apart from the launch (the paper's methodology keeps kernel-only
+ * and whole-decode figures apart, Section 5): every block stamps the global nanosecond timer when its first
+ * thread starts and when its last consumer warp has finished; *ns = latest end - earliest start over all blocks
+ * (resolution of that timer: about a quarter of a microsecond).  HOST out.  Synchronises the step's stream. */
+amk_status amk_last_kernel_ns(amk_handle* h, uint64_t* ns);
+
 /* Test hook for the 32-bit sequence numbers: sets the handle's count of steps launched since its activation
  * area was last cleared.  Every published activation carries step_count * (5 L + 1) + task + 1; shortly before
  * that would wrap, a step first clears the activation area on its stream and restarts the count (a handle can
- * decode for ever).  Setting the count close to 2^32 / (5 L + 1) lets a test cross that point. */
+ * decode for ever).  Setting the count close to 2^32 / (5 L + 1) lets a test cross that point.  The hook also
+ * clears the activation area (on the handle's last stream), since a count set by hand could otherwise meet its
+ * own sequence numbers from earlier steps. */
 amk_status amk_debug_set_step_count(amk_handle* h, uint32_t steps);
 
 /* Frees host state only.  The caller's buffers are untouched. */

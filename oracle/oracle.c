@@ -352,8 +352,42 @@ static void linear(const orc_config* c, const orc_weights* w, int kind, int laye
  * q head h -> kv head floor(h / (n_q/n_kv)); K cached after the rotation; LM head = embedding matrix when
  * tied, and it stays bf16 in the quantised variants (tied or not).
  */
+
+/* Distance between two bf16 values in representable steps (sign-magnitude bit patterns ordered as integers). */
+static int bf16_steps_apart(uint16_t a, uint16_t b) {
+    int ia = (a & 0x8000u) ? -(int)(a & 0x7fffu) : (int)(a & 0x7fffu);
+    int ib = (b & 0x8000u) ? -(int)(b & 0x7fffu) : (int)(b & 0x7fffu);
+    return ia > ib ? ia - ib : ib - ia;
+}
+
+/* The cache entry appended for one fp32 value.  The contract is round-to-nearest-even to bf16.  Two correct
+ * implementations whose fp32 values differ in the last bits (another summation order) may land on either side
+ * of a rounding boundary, i.e. on neighbouring bf16 values: both are valid cache entries.  A caller that
+ * compares another implementation with this one can pass that implementation's entry as `pref`: it is adopted
+ * only if it is this oracle's own rounding or one of its two neighbours, so that everything computed FROM the
+ * cache afterwards is compared like with like; otherwise the oracle keeps its own.  `own` always receives the
+ * oracle's own rounding. */
+static uint16_t cache_entry(float value, const uint16_t* pref, uint16_t* own, int* adopted) {
+    uint16_t r = orc_f32_to_bf16(value);
+    if (own) *own = r;
+    if (pref && *pref != r && bf16_steps_apart(*pref, r) <= 1) { if (adopted) (*adopted)++; return *pref; }
+    return r;
+}
+
+int orc_decode_step_rows(const orc_config* c, const orc_weights* w, int token, int pos,
+                         uint16_t* kv_cache, float* kv_f32, float* logits, int* next_token, float* hidden,
+                         const uint16_t* rows_pref, uint16_t* rows_own, int* n_adopted);
+
 int orc_decode_step(const orc_config* c, const orc_weights* w, int token, int pos,
                     uint16_t* kv_cache, float* kv_f32, float* logits, int* next_token, float* hidden) {
+    return orc_decode_step_rows(c, w, token, pos, kv_cache, kv_f32, logits, next_token, hidden, NULL, NULL, NULL);
+}
+
+/* The same step with the appended cache rows exposed: rows_pref / rows_own are [2][L][n_kv][hd] bf16 (K rows then
+ * V rows of slot `pos`), either may be NULL; see cache_entry.  *n_adopted counts the preferred entries taken. */
+int orc_decode_step_rows(const orc_config* c, const orc_weights* w, int token, int pos,
+                         uint16_t* kv_cache, float* kv_f32, float* logits, int* next_token, float* hidden,
+                         const uint16_t* rows_pref, uint16_t* rows_own, int* n_adopted) {
     const int H = c->hidden, L = c->n_layers, nq = c->n_q_heads, nkv = c->n_kv_heads, hd = c->head_dim;
     const int I = c->mlp, V = c->vocab, S = c->max_seq;
     if (token < 0 || token >= V || pos < 0 || pos >= S || nq % nkv != 0 || (hd & 1)) return -1;
@@ -387,10 +421,13 @@ int orc_decode_step(const orc_config* c, const orc_weights* w, int token, int po
         /* 4: append to the cache (slot pos of this layer) */
         for (int g = 0; g < nkv; g++) {
             size_t base = (((size_t)l * nkv + g) * S + (size_t)pos) * hd;
+            const size_t rbase = ((size_t)l * nkv + g) * hd, rhalf = (size_t)L * nkv * hd;
             for (int d = 0; d < hd; d++) {
                 if (c->round_kv) {
-                    kv_cache[base + d] = orc_f32_to_bf16(k[g * hd + d]);
-                    kv_cache[kv_half + base + d] = orc_f32_to_bf16(v[g * hd + d]);
+                    kv_cache[base + d] = cache_entry(k[g * hd + d], rows_pref ? rows_pref + rbase + d : NULL,
+                                                     rows_own ? rows_own + rbase + d : NULL, n_adopted);
+                    kv_cache[kv_half + base + d] = cache_entry(v[g * hd + d], rows_pref ? rows_pref + rhalf + rbase + d : NULL,
+                                                               rows_own ? rows_own + rhalf + rbase + d : NULL, n_adopted);
                 } else {
                     kv_f32[base + d] = k[g * hd + d];
                     kv_f32[kv_half + base + d] = v[g * hd + d];
@@ -449,8 +486,17 @@ int orc_decode_step(const orc_config* c, const orc_weights* w, int token, int po
 
 /* One decoder layer applied to a given residual stream x_in (fp32 [H]) -> x_out, with the same cache
  * semantics as the full step.  Lets a sampled layer of a large model be checked on its own. */
+int orc_layer_step_rows(const orc_config* c, const orc_weights* w, int layer, int pos, const float* x_in,
+                        uint16_t* kv_cache, float* x_out, const uint16_t* rows_pref, uint16_t* rows_own, int* n_adopted);
+
 int orc_layer_step(const orc_config* c, const orc_weights* w, int layer, int pos, const float* x_in,
                    uint16_t* kv_cache, float* x_out) {
+    return orc_layer_step_rows(c, w, layer, pos, x_in, kv_cache, x_out, NULL, NULL, NULL);
+}
+
+/* rows_pref / rows_own: [2][n_kv][hd] bf16, the K row then the V row this layer appends (see cache_entry). */
+int orc_layer_step_rows(const orc_config* c, const orc_weights* w, int layer, int pos, const float* x_in,
+                        uint16_t* kv_cache, float* x_out, const uint16_t* rows_pref, uint16_t* rows_own, int* n_adopted) {
     const int H = c->hidden, L = c->n_layers, nq = c->n_q_heads, nkv = c->n_kv_heads, hd = c->head_dim;
     const int I = c->mlp, S = c->max_seq;
     if (layer < 0 || layer >= L || pos < 0 || pos >= S || nq % nkv != 0 || (hd & 1)) return -1;
@@ -475,9 +521,12 @@ int orc_layer_step(const orc_config* c, const orc_weights* w, int layer, int pos
     for (int g = 0; g < nkv; g++) orc_rope(k + (size_t)g * hd, hd, pos, (double)c->rope_theta);
     for (int g = 0; g < nkv; g++) {
         size_t base = (((size_t)l * nkv + g) * S + (size_t)pos) * hd;
+        const size_t rbase = (size_t)g * hd, rhalf = (size_t)nkv * hd;
         for (int d = 0; d < hd; d++) {
-            kv_cache[base + d] = orc_f32_to_bf16(k[g * hd + d]);
-            kv_cache[kv_half + base + d] = orc_f32_to_bf16(v[g * hd + d]);
+            kv_cache[base + d] = cache_entry(k[g * hd + d], rows_pref ? rows_pref + rbase + d : NULL,
+                                             rows_own ? rows_own + rbase + d : NULL, n_adopted);
+            kv_cache[kv_half + base + d] = cache_entry(v[g * hd + d], rows_pref ? rows_pref + rhalf + rbase + d : NULL,
+                                                       rows_own ? rows_own + rhalf + rbase + d : NULL, n_adopted);
         }
     }
 #pragma omp parallel for schedule(static)

@@ -72,6 +72,8 @@ def lib() -> C.CDLL:
         L.orc_num_threads.restype = C.c_int
         L.orc_decode_step.restype = C.c_int
         L.orc_layer_step.restype = C.c_int
+        L.orc_decode_step_rows.restype = C.c_int
+        L.orc_layer_step_rows.restype = C.c_int
         L.orc_head_step.restype = C.c_int
     return _lib
 
@@ -334,25 +336,50 @@ class Model:
         return np.zeros(kv_elems(self.shape), dtype=np.uint16)
 
     def decode_step(self, token: int, pos: int, kv: np.ndarray, kv_f32: Optional[np.ndarray] = None,
-                    want_hidden: bool = True):
-        """Returns (logits fp32 [V], next_token, hidden fp32 [L+1][H] or None); updates ``kv`` in place."""
+                    want_hidden: bool = True, rows_pref: Optional[np.ndarray] = None):
+        """Returns (logits fp32 [V], next_token, hidden fp32 [L+1][H] or None); updates ``kv`` in place.
+
+        ``rows_pref`` (uint16 [2][L][n_kv][hd]): another implementation's appended cache rows.  An entry is
+        adopted where it is the oracle's own rounding or a neighbouring bf16 value (both are valid roundings of
+        fp32 values that differ in the last bits); the oracle's own rows and the number of adopted entries are
+        then left in ``self.rows_own`` / ``self.n_adopted``."""
         s = self.shape
         assert kv.dtype == np.uint16 and kv.size == kv_elems(s) and kv.flags["C_CONTIGUOUS"]
         logits = np.empty(s.vocab, dtype=np.float32)
         nxt = C.c_int(-1)
         hidden = np.empty((s.n_layers + 1, s.hidden), dtype=np.float32) if want_hidden else None
-        rc = lib().orc_decode_step(C.byref(self.cfg), C.byref(self.w), C.c_int(token), C.c_int(pos),
-                                   _p(kv), _p(kv_f32), _p(logits), C.byref(nxt), _p(hidden))
+        if rows_pref is None:
+            rc = lib().orc_decode_step(C.byref(self.cfg), C.byref(self.w), C.c_int(token), C.c_int(pos),
+                                       _p(kv), _p(kv_f32), _p(logits), C.byref(nxt), _p(hidden))
+        else:
+            rows_pref = _c(rows_pref, np.uint16)
+            assert rows_pref.size == 2 * s.n_layers * s.n_kv_heads * s.head_dim
+            self.rows_own = np.empty(rows_pref.size, dtype=np.uint16)
+            n = C.c_int(0)
+            rc = lib().orc_decode_step_rows(C.byref(self.cfg), C.byref(self.w), C.c_int(token), C.c_int(pos),
+                                            _p(kv), _p(kv_f32), _p(logits), C.byref(nxt), _p(hidden),
+                                            _p(rows_pref), _p(self.rows_own), C.byref(n))
+            self.n_adopted = int(n.value)
         if rc != 0:
             raise ValueError("oracle: bad argument (token/pos/head shape)")
         return logits, int(nxt.value), hidden
 
-    def layer_step(self, layer: int, pos: int, x_in, kv: np.ndarray) -> np.ndarray:
+    def layer_step(self, layer: int, pos: int, x_in, kv: np.ndarray, rows_pref: Optional[np.ndarray] = None) -> np.ndarray:
+        """One decoder layer on a given residual stream.  ``rows_pref`` (uint16 [2][n_kv][hd]): see decode_step."""
         s = self.shape
         x_in = _c(x_in, np.float32)
         out = np.empty(s.hidden, dtype=np.float32)
-        rc = lib().orc_layer_step(C.byref(self.cfg), C.byref(self.w), C.c_int(layer), C.c_int(pos), _p(x_in),
-                                  _p(kv), _p(out))
+        if rows_pref is None:
+            rc = lib().orc_layer_step(C.byref(self.cfg), C.byref(self.w), C.c_int(layer), C.c_int(pos), _p(x_in),
+                                      _p(kv), _p(out))
+        else:
+            rows_pref = _c(rows_pref, np.uint16)
+            assert rows_pref.size == 2 * s.n_kv_heads * s.head_dim
+            self.rows_own = np.empty(rows_pref.size, dtype=np.uint16)
+            n = C.c_int(0)
+            rc = lib().orc_layer_step_rows(C.byref(self.cfg), C.byref(self.w), C.c_int(layer), C.c_int(pos), _p(x_in),
+                                           _p(kv), _p(out), _p(rows_pref), _p(self.rows_own), C.byref(n))
+            self.n_adopted = int(n.value)
         if rc != 0:
             raise ValueError("oracle: bad argument")
         return out

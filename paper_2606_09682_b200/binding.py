@@ -75,6 +75,7 @@ def _load() -> C.CDLL:
         "amk_debug_unpack": (C.c_int, [vp, C.c_int, C.c_int, vp, vp, vp, vp]),
         "amk_debug_drop_signal": (C.c_int, [vp, C.c_int, C.c_int]),
         "amk_debug_set_step_count": (C.c_int, [vp, C.c_uint32]),
+        "amk_last_kernel_ns": (C.c_int, [vp, C.POINTER(C.c_uint64)]),
         "amk_destroy": (C.c_int, [vp]),
         "amk_quantize_int8": (C.c_int, [vp, i64, i64, vp, vp, vp]),
         "amk_quantize_int4": (C.c_int, [vp, i64, i64, vp, vp, vp, vp]),
@@ -91,7 +92,7 @@ def _load() -> C.CDLL:
 lib = _load()
 EXPORTS = ("amk_status_str", "amk_packed_bytes", "amk_workspace_bytes", "amk_kv_bytes", "amk_create",
            "amk_decode_step", "amk_decode_greedy", "amk_last_status", "amk_plan_info", "amk_debug_hidden",
-           "amk_debug_trace", "amk_debug_unpack", "amk_debug_drop_signal", "amk_debug_set_step_count", "amk_destroy", "amk_quantize_int8", "amk_quantize_int4",
+           "amk_debug_trace", "amk_debug_unpack", "amk_debug_drop_signal", "amk_debug_set_step_count", "amk_last_kernel_ns", "amk_destroy", "amk_quantize_int8", "amk_quantize_int4",
            "amk_argmax_static", "amk_plan_export", "amk_plan_check")
 
 
@@ -239,13 +240,18 @@ class Decoder:
 
     def __init__(self, shape, weights: Dict, wdtype: str = "bf16", flags: int = 0, wait_timeout_us: int = 0,
                  stage_bytes: int = 0, n_stages: int = 0, max_inflight: int = 0, sync_mode: int = 1,
-                 n_blocks: int = 0, l2_ahead: int = 0, device="cuda"):
+                 n_blocks: int = 0, l2_ahead: int = 0, device="cuda", guard_bytes: int = 0):
+        """``guard_bytes`` (a multiple of 256): the packed buffer, the workspace and the logits get that many bytes
+        of a fixed pattern in front and behind, which ``guards_intact()`` checks -- a stand-in for a memory checker."""
         self.shape, self.wdtype = shape, wdtype
         self.device = torch.device(device)
         self.cfg = make_config(shape, wdtype, flags, wait_timeout_us, stage_bytes, n_stages, max_inflight,
                                sync_mode=sync_mode, n_blocks=n_blocks, l2_ahead=l2_ahead)
-        self.packed = torch.empty(amk_packed_bytes(self.cfg), dtype=torch.uint8, device=self.device)
-        self.workspace = torch.empty(amk_workspace_bytes(self.cfg), dtype=torch.uint8, device=self.device)
+        assert guard_bytes % 256 == 0
+        self._guard = guard_bytes
+        self._guarded: List[torch.Tensor] = []
+        self.packed = self._alloc(amk_packed_bytes(self.cfg))
+        self.workspace = self._alloc(amk_workspace_bytes(self.cfg))
         keep: List = []
         w = amk_weights()
         w.embed = weights["embed"].data_ptr()
@@ -264,11 +270,30 @@ class Decoder:
                               self.workspace.data_ptr(), self.workspace.numel(), _stream(), C.byref(h)), "amk_create")
         self.h = h
         torch.cuda.current_stream().synchronize()      # the canonical weights may be freed from here on
-        self.logits = torch.empty(shape.vocab, dtype=torch.float32, device=self.device)
+        self.logits = self._alloc(4 * shape.vocab).view(torch.float32)
         self.next_token = torch.empty(1, dtype=torch.int32, device=self.device)
 
+    def _alloc(self, n_bytes: int) -> torch.Tensor:
+        """uint8 device buffer of n_bytes (256-byte aligned), with guard bands around it if asked for."""
+        g = self._guard
+        if not g:
+            return torch.empty(n_bytes, dtype=torch.uint8, device=self.device)
+        inner = (n_bytes + 255) // 256 * 256
+        whole = torch.full((inner + 2 * g,), 0xA5, dtype=torch.uint8, device=self.device)
+        self._guarded.append((whole, inner))
+        return whole[g:g + n_bytes]
+
+    def guards_intact(self) -> bool:
+        g = self._guard
+        return all(bool((w[:g] == 0xA5).all()) and bool((w[g + inner:] == 0xA5).all()) for w, inner in self._guarded)
+
     def new_cache(self) -> torch.Tensor:
-        return torch.zeros(amk_kv_bytes(self.cfg) // 2, dtype=torch.bfloat16, device=self.device)
+        n = amk_kv_bytes(self.cfg)
+        if not self._guard:
+            return torch.zeros(n // 2, dtype=torch.bfloat16, device=self.device)
+        buf = self._alloc(n)
+        buf.zero_()
+        return buf.view(torch.bfloat16)
 
     def plan(self) -> amk_plan:
         p = amk_plan()
@@ -328,6 +353,12 @@ class Decoder:
 
     def amk_debug_drop_signal(self, phase: int, block: int) -> None:
         _check(lib.amk_debug_drop_signal(self.h, phase, block), "amk_debug_drop_signal")
+
+    def amk_last_kernel_ns(self) -> int:
+        """Kernel-only nanoseconds of the last step (first block start to last block end); synchronises."""
+        ns = C.c_uint64()
+        _check(lib.amk_last_kernel_ns(self.h, C.byref(ns)), "amk_last_kernel_ns")
+        return int(ns.value)
 
     def amk_debug_set_step_count(self, steps: int) -> None:
         _check(lib.amk_debug_set_step_count(self.h, steps), "amk_debug_set_step_count")

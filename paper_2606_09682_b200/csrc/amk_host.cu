@@ -46,7 +46,7 @@ struct Plan {
 
 struct WorkspaceLayout {
   size_t status, phase_ctr, group_ctr, lm_ctr, next_ws, cand_val, cand_idx, x_a, x_b, qkv, o, m, m_amax, part, hidden, rope,
-      trace, slice_tab, bounds, smid_tab, calib, tile_begin, tiles, total;
+      trace, ktime, slice_tab, bounds, smid_tab, calib, tile_begin, tiles, total;
 };
 
 void plan_to_words(const amk_config* cfg, const Plan& pl, const std::vector<unsigned long long>& tiles,
@@ -206,6 +206,7 @@ WorkspaceLayout workspace_layout(const amk_config* c, const Plan& pl) {
   w.hidden = take((L + 1) * H * 4);
   w.rope = take(S * (hd / 2) * sizeof(float2));
   w.trace = take((size_t)pl.n_blocks * (5 * L + 1) * AMK_TRACE_EVENTS * 8);
+  w.ktime = take((size_t)kMaxBlocks * 16);
   w.slice_tab = take(pl.ops.size() * (size_t)pl.n_blocks * 8);
   w.bounds = take(5 * ((size_t)pl.n_blocks + 1) * 4);
   w.smid_tab = take((size_t)kMaxSmid * 4);
@@ -553,6 +554,7 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     p.cand_idx = (int*)(h->ws + h->wl.cand_idx); p.next_ws = (int*)(h->ws + h->wl.next_ws);
     p.status = (DevStatus*)(h->ws + h->wl.status);
     p.trace = (cfg->flags & AMK_FLAG_TRACE) ? (unsigned long long*)(h->ws + h->wl.trace) : nullptr;
+    p.ktime = (unsigned long long*)(h->ws + h->wl.ktime);
     p.stage_bytes = (int)stage_bytes; p.n_stages = (int)n_stages; p.max_inflight = (int)max_inflight;
     p.l2_ahead = cfg->l2_ahead == 0 ? 6 : (cfg->l2_ahead > 32 ? 0 : (int)cfg->l2_ahead);
     p.act_bytes = (int)act;
@@ -749,7 +751,25 @@ amk_status amk_debug_drop_signal(amk_handle* h, int phase, int block) {
 
 amk_status amk_debug_set_step_count(amk_handle* h, uint32_t steps) {
   if (!h) return AMK_ERR_INVALID_ARG;
+  // whatever earlier steps left in the activation area could carry the sequence numbers of the steps to come
+  if (cudaMemsetAsync(h->ws + h->wl.x_a, 0, h->wl.hidden - h->wl.x_a, h->last_stream) != cudaSuccess) return AMK_ERR_CUDA;
   h->epoch = steps;
+  return AMK_OK;
+}
+
+amk_status amk_last_kernel_ns(amk_handle* h, uint64_t* ns) {
+  if (!h || !ns) return AMK_ERR_INVALID_ARG;
+  const int nb = (int)h->plan.n_blocks;
+  std::vector<unsigned long long> t((size_t)nb * 2);
+  cudaError_t e = cudaStreamSynchronize(h->last_stream);
+  if (e == cudaSuccess) e = cudaMemcpy(t.data(), h->ws + h->wl.ktime, t.size() * 8, cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return AMK_ERR_CUDA;
+  unsigned long long first = ~0ull, last = 0ull;
+  for (int b = 0; b < nb; b++) {
+    if (t[2 * b] < first) first = t[2 * b];
+    if (t[2 * b + 1] > last) last = t[2 * b + 1];
+  }
+  *ns = (last >= first && first != 0ull) ? (uint64_t)(last - first) : 0u;
   return AMK_OK;
 }
 

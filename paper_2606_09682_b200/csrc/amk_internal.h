@@ -101,6 +101,7 @@ struct KParams {
   int* next_ws;
   DevStatus* status;
   unsigned long long* trace;              // [n_blocks][5 L + 1][8] or null
+  unsigned long long* ktime;              // [n_blocks][2]: global-timer stamps of each block's first and last instruction
   // plan
   int stage_bytes, n_stages, max_inflight;
   int l2_ahead;                           // ring tiles requested into L2 ahead of the ring (0..32)

@@ -1281,6 +1281,7 @@ __global__ void __launch_bounds__(kThreads, 1) amk_decode_kernel(const __grid_co
   const int nblk = gridDim.x;
 
   if (tid == 0) {
+    p.ktime[2 * blockIdx.x] = globaltimer_ns();
     for (int s = 0; s < p.n_stages; s++) {
       mbar_init(&sh->full[s], 1);
       mbar_init(&sh->empty[s], kConsumerWarps);
@@ -1351,6 +1352,8 @@ __global__ void __launch_bounds__(kThreads, 1) amk_decode_kernel(const __grid_co
     else ok = gemv_op<WDL, false>(c, k == 0 ? (int)OP_QKV : k - 1, l);
   }
   if (ok) lm_head_task(p, sh, xs, ring, cta, nblk, c.stage, c.parity, token);
+  // (every consumer warp stamps; the latest store of the latest block is the kernel's end)
+  if (lane == 0) atomicMax(p.ktime + 2 * blockIdx.x + 1, globaltimer_ns());
 }
 
 // Calibration: every block (one per SM, same shared-memory footprint as the decode kernel) streams

@@ -46,44 +46,68 @@ def check_argmax(logits_oracle, tok_gpu):
     return "soft"
 
 
+ELEM_TOL = 1e-3        # element-wise: |gpu - oracle| <= ELEM_TOL * max|oracle| on the logits and on every hidden row
+KV_NEAR_ZERO = 1e-4    # a cached value more than one bf16 step off must be within this fraction of its row's maximum
+
+
+def max_err(a, b):
+    """Largest element-wise deviation relative to the reference row's largest magnitude."""
+    a, b = np.asarray(a, dtype=np.float64), np.asarray(b, dtype=np.float64)
+    return float(np.abs(a - b).max() / max(np.abs(b).max(), 1e-30))
+
+
+def check_kv_rows(rows_gpu, rows_own):
+    """The appended K / V rows of both sides, as bf16 bit patterns of the same shape [..., hd].  They are roundings
+    of fp32 values that agree to ~1e-6, so they are equal or neighbours -- except where the value itself is
+    rounding noise around zero (there a bf16 step is far smaller than that 1e-6): such entries must be tiny
+    against their row.  Returns (largest distance in bf16 steps, fraction one step apart, number further apart)."""
+    d = bf16_ulp_distance(rows_gpu, rows_own)
+    g_f, o_f = bf16_f32(rows_gpu), bf16_f32(rows_own)
+    row_scale = np.abs(o_f).max(axis=-1, keepdims=True)
+    far = d > 1
+    assert not (far & (np.abs(g_f - o_f) > KV_NEAR_ZERO * row_scale)).any(), (int(d.max()), int(far.sum()))
+    return int(d.max()), float((d == 1).mean()), int(far.sum())
+
+
 def compare_step(shape, dec, model, token, pos, kv_gpu, kv_cpu, check_hidden=True):
-    """One step on both sides; asserts the acceptance bar; returns a dict of measured errors."""
+    """One step on both sides; asserts the acceptance bar; returns a dict of measured errors.
+
+    The CUDA path runs first.  The oracle then takes the step with the CUDA path's appended cache rows as its
+    preference: where such an entry neighbours the oracle's own rounding (both are valid roundings of fp32 values
+    that differ in the last bits) the oracle continues from it, so that everything downstream of the cache is
+    compared like with like and the element-wise bound can be tight."""
+    L, G, S, hd = shape.n_layers, shape.n_kv_heads, shape.max_seq, shape.head_dim
     kv_before = kv_cpu.copy()
     dec.amk_decode_step(token, pos, kv_gpu)
     st, msg = dec.amk_last_status()
     assert st == 0, msg
-    logits_o, tok_o, hidden_o = model.decode_step(token, pos, kv_cpu, want_hidden=check_hidden)
+    kvg = kv_gpu.view(torch.int16).cpu().numpy().view(np.uint16).reshape(2, L, G, S, hd)
+    rows_gpu = np.ascontiguousarray(kvg[:, :, :, pos, :])
+    logits_o, tok_o, hidden_o = model.decode_step(token, pos, kv_cpu, want_hidden=check_hidden, rows_pref=rows_gpu)
     logits_g = dec.logits.cpu().numpy()
     tok_g = int(dec.next_token.item())
     LAST["logits_oracle"], LAST["logits_gpu"], LAST["token_gpu"] = logits_o, logits_g, tok_g
-    out = {"logits": rel_l2(logits_g, logits_o)}
+    out = {"logits": rel_l2(logits_g, logits_o), "logits_max": max_err(logits_g, logits_o)}
     assert np.isfinite(logits_g).all()
     if check_hidden:
         hidden_g = dec.amk_debug_hidden().numpy()
-        errs = [rel_l2(hidden_g[l], hidden_o[l]) for l in range(shape.n_layers + 1)]
+        errs = [rel_l2(hidden_g[l], hidden_o[l]) for l in range(L + 1)]
         out["hidden_max"] = max(errs)
+        out["hidden_elem_max"] = max(max_err(hidden_g[l], hidden_o[l]) for l in range(L + 1))
         assert errs[0] == 0.0, "embedding row must be exact"
         assert max(errs) <= HIDDEN_TOL, errs
+        assert out["hidden_elem_max"] <= ELEM_TOL, out
     assert out["logits"] <= LOGITS_TOL, out
+    assert out["logits_max"] <= ELEM_TOL, out
     out["argmax"] = check_argmax(logits_o, tok_g)
     assert tok_g == int(np.argmax(logits_g)) or logits_g[tok_g] == logits_g.max()
-    # KV cache: exactly slot `pos` of every layer / kv head changed, and it is within 1 bf16 step of the oracle's
-    L, G, S, hd = shape.n_layers, shape.n_kv_heads, shape.max_seq, shape.head_dim
-    kvg = kv_gpu.view(torch.int16).cpu().numpy().view(np.uint16).reshape(2, L, G, S, hd)
-    kvo = kv_cpu.reshape(2, L, G, S, hd)
+    # KV cache: exactly slot `pos` of every layer / kv head changed ...
     kvb = kv_before.reshape(2, L, G, S, hd)
     mask = np.ones(S, dtype=bool)
     mask[pos] = False
     assert np.array_equal(kvg[:, :, :, mask, :], kvb[:, :, :, mask, :]), "a slot other than pos changed"
-    d = bf16_ulp_distance(kvg[:, :, :, pos, :], kvo[:, :, :, pos, :])
-    out["kv_ulp_max"] = int(d.max())
-    out["kv_mismatch_frac"] = float((d > 0).mean())
-    # A cached value may differ by one bf16 step where the two sides' fp32 values straddle a rounding
-    # boundary; beyond that, only by what the hidden-state tolerance allows relative to its row's scale.
-    g_f, o_f = bf16_f32(kvg[:, :, :, pos, :]), bf16_f32(kvo[:, :, :, pos, :])
-    row_scale = np.abs(o_f).max(axis=-1, keepdims=True)
-    bad = (d > 1) & (np.abs(g_f - o_f) > HIDDEN_TOL * row_scale)
-    assert not bad.any(), out
+    # ... and the new rows are the oracle's own roundings or their neighbours
+    out["kv_ulp_max"], out["kv_one_step_frac"], out["kv_far"] = check_kv_rows(rows_gpu, model.rows_own.reshape(rows_gpu.shape))
     # keep both caches identical from here on so later steps compare like with like
     kv_cpu[:] = kv_gpu.view(torch.int16).cpu().numpy().view(np.uint16)
     return out

@@ -82,6 +82,24 @@ def test_counter_joins(name, wdtype):
     dec.close()
 
 
+@pytest.mark.parametrize("n_blocks", [148, 101, 37])
+def test_block_counts(n_blocks):
+    """The split of every product's rows over the blocks (and with it the order of the partial sums) follows the
+    block count; the results stay within the same bar for every split, and each split repeats bit for bit."""
+    shape, dec, model = _setup("mini_wide", "int8", seed=26, n_blocks=n_blocks)
+    tok = inp.make_token(shape, 10)
+    for pos in (0, 50):
+        kv_g = inp.make_kv_prefill(shape, 11, pos, device="cuda")
+        kv_c = inp.bits(kv_g).copy()
+        r = gc.compare_step(shape, dec, model, tok, pos, kv_g, kv_c)
+        first = dec.logits.clone()
+        dec.amk_decode_step(tok, pos, kv_g)
+        torch.cuda.synchronize()
+        assert torch.equal(dec.logits, first)
+        print("blocks", n_blocks, pos, r)
+    dec.close()
+
+
 def test_deterministic_repeat():
     shape, dec, model = _setup("mini_wide", "bf16", seed=23)
     kv = inp.make_kv_prefill(shape, 6, 77, device="cuda")

@@ -110,6 +110,118 @@ def test_argument_errors(amk):
     dec.close()
 
 
+def test_misaligned_buffers_are_refused_on_the_host(amk):
+    """The kernel fetches cache rows with 16-byte bulk copies and writes 4-byte words: a misaligned pointer is an
+    argument error, never a device fault."""
+    shape = inp.SHAPES["mini"]
+    w = inp.make_weights(shape, 45, device="cuda")
+    dec = amk.Decoder(shape, w, "bf16")
+    kv = dec.new_cache()
+    big = torch.zeros(kv.numel() + 64, dtype=torch.bfloat16, device="cuda")
+    odd = torch.zeros(shape.vocab * 4 + 16, dtype=torch.uint8, device="cuda")
+    call = amk.lib.amk_decode_step
+    assert call(dec.h, 1, 0, big.data_ptr() + 2, dec.logits.data_ptr(), dec.next_token.data_ptr(), None) == amk.AMK_ERR_INVALID_ARG
+    assert call(dec.h, 1, 0, big.data_ptr() + 8, dec.logits.data_ptr(), dec.next_token.data_ptr(), None) == amk.AMK_ERR_INVALID_ARG
+    assert call(dec.h, 1, 0, kv.data_ptr(), odd.data_ptr() + 2, dec.next_token.data_ptr(), None) == amk.AMK_ERR_INVALID_ARG
+    assert call(dec.h, 1, 0, kv.data_ptr(), dec.logits.data_ptr(), odd.data_ptr() + 1, None) == amk.AMK_ERR_INVALID_ARG
+    toks = torch.zeros(8, dtype=torch.int32, device="cuda")
+    assert amk.lib.amk_decode_greedy(dec.h, 1, 0, 4, big.data_ptr() + 4, toks.data_ptr(), None, None) == amk.AMK_ERR_INVALID_ARG
+    assert call(dec.h, 1, 0, big.data_ptr() + 16, dec.logits.data_ptr(), dec.next_token.data_ptr(), None) == amk.AMK_OK
+    assert dec.amk_last_status()[0] == amk.AMK_OK
+    dec.close()
+
+
+def test_sequence_numbers_cross_their_wrap(amk):
+    """Every published activation carries steps * (5 L + 1) + task + 1 in 32 bits.  Near 2^32 the library clears
+    the activation area on the stream and restarts the count: steps on both sides of that point, and across it
+    inside one device-resident run, give what a fresh handle gives."""
+    shape = inp.SHAPES["mini_wide"]
+    w = inp.make_weights(shape, 46, device="cuda", std=0.05)
+    ref = amk.Decoder(shape, w, "bf16")
+    dec = amk.Decoder(shape, w, "bf16")
+    per = 5 * shape.n_layers + 1
+    limit = (1 << 32) // per
+    n = 12
+    kv_r, kv_d = ref.new_cache(), dec.new_cache()
+    want = ref.amk_decode_greedy(9, 0, n, kv_r).cpu().tolist()
+    want_logits = ref.logits.clone()
+    dec.amk_debug_set_step_count(limit - 6)                   # the wrap falls inside the 12-step run
+    got = dec.amk_decode_greedy(9, 0, n, kv_d).cpu().tolist()
+    assert dec.amk_last_status()[0] == amk.AMK_OK
+    assert got == want and torch.equal(kv_d, kv_r) and torch.equal(dec.logits, want_logits)
+    # single steps right at the boundary, with stale activations of the highest sequence numbers in the workspace
+    for start in (limit - 3, limit - 2, limit - 1):
+        dec.amk_debug_set_step_count(start)
+        kv1, kv2 = dec.new_cache(), ref.new_cache()
+        tok = 9
+        for pos in range(4):
+            dec.amk_decode_step(tok, pos, kv1)
+            ref.amk_decode_step(tok, pos, kv2)
+            assert dec.amk_last_status()[0] == amk.AMK_OK
+            assert torch.equal(dec.logits, ref.logits) and int(dec.next_token.item()) == int(ref.next_token.item())
+            tok = int(ref.next_token.item())
+        assert torch.equal(kv1, kv2)
+    ref.close()
+    dec.close()
+
+
+@pytest.mark.parametrize("wdtype,pos", [("bf16", 0), ("int8", 70), ("int4", 33)])
+def test_guard_bands_around_every_caller_buffer_stay_intact(amk, wdtype, pos):
+    """Stand-in for a memory checker (none can be run here): the packed buffer, the workspace, the logits and the
+    KV cache sit between bands of a fixed pattern; create, the decode step, the device-resident loop and the
+    debugging read-backs must leave the bands untouched."""
+    shape = inp.SHAPES["mini_ragged" if wdtype != "int4" else "mini_wide"]
+    w = inp.make_weights(shape, 47, device="cuda")
+    wq = amk.quantize_weights(w, wdtype)
+    dec = amk.Decoder(shape, wq, wdtype, flags=amk.AMK_FLAG_DEBUG_HIDDEN | amk.AMK_FLAG_TRACE, guard_bytes=4096)
+    kv = dec.new_cache()
+    kv.view(torch.int16)[:] = inp.make_kv_prefill(shape, 48, pos, device="cuda").view(torch.int16)
+    assert dec.guards_intact()
+    dec.amk_decode_step(3, pos, kv)
+    assert dec.amk_last_status()[0] == amk.AMK_OK
+    dec.amk_decode_greedy(3, pos, min(8, shape.max_seq - pos), kv)
+    assert dec.amk_last_status()[0] == amk.AMK_OK
+    dec.amk_debug_hidden()
+    dec.amk_debug_trace()
+    torch.cuda.synchronize()
+    assert dec.guards_intact()
+    dec.close()
+
+
+@pytest.mark.parametrize("cycles", [False, True])
+def test_trace_stamps_are_ordered_within_every_task(amk, cycles):
+    """amk_debug_trace: within a block every matrix-vector task's stamps follow the order of its stages, tasks
+    follow each other, and the producer issued a task's first tile no later than its last."""
+    shape = inp.SHAPES["mini_wide"]
+    w = inp.make_weights(shape, 49, device="cuda")
+    flags = amk.AMK_FLAG_TRACE | (amk.AMK_FLAG_TRACE_CYCLES if cycles else 0)
+    dec = amk.Decoder(shape, w, "bf16", flags=flags)
+    kv = inp.make_kv_prefill(shape, 50, 40, device="cuda")
+    for pos in (0, 40):
+        dec.amk_decode_step(7, pos, kv)
+        assert dec.amk_last_status()[0] == amk.AMK_OK
+        tr = dec.amk_debug_trace().numpy()                    # [blocks][5 L + 1][events]
+        nb, nt, _ = tr.shape
+        order = [0, 1, 2, 8, 9, 10, 7, 3]                     # enter, joined, loaded, pass begin, first tile, tiles done, reduced, computed
+        p = dec.plan()
+        for b in range(nb):
+            prev_end = 0
+            for t in range(nt):
+                if t % 5 == 1 and t != nt - 1:
+                    continue                                  # attention tasks stamp a different set of stages
+                e = tr[b, t]
+                if e[3] == 0 or e[1] == 0:
+                    continue                                  # a block without rows of this product
+                seq = [int(e[i]) for i in order]
+                assert all(x > 0 for x in seq), (b, t, seq)
+                assert all(x <= y for x, y in zip(seq, seq[1:])), (b, t, seq)
+                assert seq[0] >= prev_end, (b, t)
+                prev_end = seq[-1]
+                if e[5]:
+                    assert e[5] <= e[6], (b, t)
+    dec.close()
+
+
 def test_greedy_loop_equals_single_steps(amk):
     shape = inp.SHAPES["mini_wide"]
     w = inp.make_weights(shape, 44, device="cuda", std=0.05)

@@ -186,6 +186,58 @@ def test_pos0_attention_output_is_cached_v():
     assert np.array_equal(f64(kvv[1, 0, :, 0, :]).ravel(), v)
 
 
+def _bump(bits, steps):
+    """bf16 bit patterns moved `steps` representable values away from zero (finite, non-zero inputs)."""
+    return (np.asarray(bits, dtype=np.uint16) + np.uint16(steps)).astype(np.uint16)
+
+
+def test_preferred_cache_rows_are_adopted_only_next_to_the_own_rounding():
+    """decode_step(rows_pref=...): another implementation's appended rows are taken where they are the oracle's
+    own rounding or a neighbouring bf16 value, and attention then reads them; anything further away is refused.
+    Pinned at position 0, where the attention output is the cached V row, against the dense form."""
+    shape = inp.SHAPES["toy"]
+    wnp = inp.weights_to_numpy(inp.make_weights(shape, seed=14, std=0.25))
+    model = orc.Model(shape, wnp)
+    tok = 42
+    L, G, S, hd = shape.n_layers, shape.n_kv_heads, shape.max_seq, shape.head_dim
+    kv0 = model.new_cache()
+    logits0, nxt0, hidden0 = model.decode_step(tok, 0, kv0)
+    own = kv0.reshape(2, L, G, S, hd)[:, :, :, 0, :].copy()                  # [2][L][G][hd]
+    # 1. preferring the oracle's own rows changes nothing
+    kv1 = model.new_cache()
+    logits1, nxt1, hidden1 = model.decode_step(tok, 0, kv1, rows_pref=own)
+    assert model.n_adopted == 0 and np.array_equal(model.rows_own.reshape(own.shape), own)
+    assert np.array_equal(kv1, kv0) and np.array_equal(logits1, logits0) and np.array_equal(hidden1, hidden0)
+    # 2. layer 0: every third V entry one step away (adopted), every fifth K entry two steps away (refused)
+    pref = own.copy()
+    pref[1, 0].reshape(-1)[::3] = _bump(own[1, 0].reshape(-1)[::3], 1)
+    pref[0, 0].reshape(-1)[::5] = _bump(own[0, 0].reshape(-1)[::5], 2)
+    kv2 = model.new_cache()
+    logits2, nxt2, hidden2 = model.decode_step(tok, 0, kv2, rows_pref=pref)
+    got = kv2.reshape(2, L, G, S, hd)[:, :, :, 0, :]
+    own2 = model.rows_own.reshape(own.shape)
+    assert np.array_equal(own2[:, 0], own[:, 0])                              # layer 0's own roundings are as before
+    assert np.array_equal(got[1, 0], pref[1, 0]) and np.array_equal(got[0, 0], own[0, 0])
+    # (later layers see a changed stream: there the first run's rows are adopted wherever they are neighbours)
+    assert model.n_adopted == int((got != own2).sum()) >= len(own[1, 0].reshape(-1)[::3])
+    # the dense form of layer 0 with the adopted V row
+    W = to_f64(wnp, shape)
+    x0 = W["embed"][tok]
+    v = f64(pref[1, 0]).reshape(G, hd)
+    n_rep = shape.n_q_heads // G
+    o = np.concatenate([v[h // n_rep] for h in range(shape.n_q_heads)])
+    x_attn = x0 + o @ W["wo"][0].T
+    b = x_attn / np.sqrt((x_attn ** 2).mean() + shape.rms_eps)
+    Gt, U = b @ W["wgate"][0].T, b @ W["wup"][0].T
+    x1 = x_attn + ((Gt / (1 + np.exp(-Gt))) * U) @ W["wdown"][0].T
+    assert rel_l2(hidden2[1], x1) < 1e-5
+    assert rel_l2(hidden0[1], x1) > 1e-4                                     # (the bumped entries do matter)
+    # 3. the single-layer form agrees with the full step
+    kv3 = model.new_cache()
+    x = model.layer_step(0, 0, hidden2[0], kv3, rows_pref=pref[:, 0])
+    assert np.array_equal(x, hidden2[1]) and model.n_adopted == len(own[1, 0].reshape(-1)[::3])
+
+
 def test_against_transformers_llama():
     tr = pytest.importorskip("transformers")
     shape = inp.SHAPES["toy"]

@@ -355,6 +355,10 @@ def test_quantisers_vs_numpy_float16_and_error_bounds():
     c_ref = np.clip(np.rint(Wg / s4f[:, :, None]) + z_ref[:, :, None], 0, 15).astype(np.uint8)
     assert np.array_equal(codes.reshape(rows, cols // group, group), c_ref)
     assert z_ref[5, 0] == 0
+    # bit patterns, not only values: a zero point of an all-positive group is -mn / s = -0.0 before the clamp and
+    # is stored as +0 (0x0000); no stored zero point ever carries a sign bit
+    assert z4[5, 0] == 0x0000
+    assert not (z4 & 0x8000).any()
     d4 = orc.dequant(orc.W_INT4, p, s4, z4, group).reshape(rows, cols // group, group)
     # inside the representable range the error is at most half a step (plus the zero point's own rounding)
     assert (np.abs(d4 - Wg) <= s4f[:, :, None] * 1.0 * (1 + 1e-6)).all()
