@@ -22,8 +22,9 @@
  * split-K combine equal to the unsplit result; exact-integer GEMVs; integer pack/unpack round trips and
  * hand-worked quantiser rows; a second, dense, cache-free recomputation of a 2-layer hidden-64 toy; a
  * library cross-check against a random-init transformers LlamaForCausalLM.
- * Parity unpinned: leaving an *untied* LM head in bf16 in the quantised variants is a declared reading
- * of the paper, not something it fixes.
+ * Parity unpinned: whether an *untied* LM head stays bf16 in the quantised variants is not fixed by the
+ * paper; both readings are implemented (quantize_lm_head 0 / 1) and each is pinned against the dense form,
+ * but which of the two the paper's kernels used cannot be pinned from its text.
  */
 #include <math.h>
 #include <stdint.h>
@@ -314,6 +315,9 @@ typedef struct {
     int32_t wdtype;        /* 0 bf16, 1 int8, 2 int4: applies to the seven per-layer linears only */
     int32_t group_size;    /* int4 group length along the input dimension */
     int32_t round_kv;      /* 1: cache entries rounded to bf16 (the contract); 0: test-only, see below */
+    int32_t quantize_lm_head; /* 0: the LM head stays bf16 (the reading taken of the paper); 1: it is quantised like
+                                 the per-layer linears (wdtype, group_size) -- the other reading of "linear GEMV
+                                 weights move to int8 / int4" for an untied head; the embedding gather stays bf16 */
 } orc_config;
 
 /* Canonical weights.  Per-layer arrays are indexed [layer]; linears are indexed by
@@ -327,7 +331,19 @@ typedef struct {
     const void* const* w[7];
     const uint16_t* const* scale[7];
     const uint16_t* const* zero[7];
+    const void* lm_head_q;          /* quantize_lm_head: codes of the LM head (of the embedding matrix when tied) */
+    const uint16_t* lm_head_scale;  /*   fp16 scales: int8 [V]; int4 [V][H/group]                                */
+    const uint16_t* lm_head_zero;   /*   int4: fp16 integer-valued zero points [V][H/group]                      */
 } orc_weights;
+
+/* logits = W_lm . y: the bf16 matrix (the embedding matrix when tied), or its quantised form */
+static void lm_head(const orc_config* c, const orc_weights* w, const float* y, float* logits) {
+    if (c->quantize_lm_head && c->wdtype != 0)
+        orc_gemv(c->wdtype, w->lm_head_q, w->lm_head_scale, c->wdtype == 2 ? w->lm_head_zero : NULL, c->group_size,
+                 c->vocab, c->hidden, y, logits);
+    else
+        orc_gemv(0, c->tied_embeddings ? w->embed : w->lm_head, NULL, NULL, 0, c->vocab, c->hidden, y, logits);
+}
 
 static void linear(const orc_config* c, const orc_weights* w, int kind, int layer, int rows, int cols,
                    const float* x, float* y) {
@@ -475,9 +491,9 @@ int orc_decode_step_rows(const orc_config* c, const orc_weights* w, int token, i
         for (int i = 0; i < H; i++) x[i] = (float)((double)x[i] + (double)t[i]);
         if (hidden) memcpy(hidden + (size_t)(l + 1) * H, x, sizeof(float) * H);
     }
-    /* 9: final norm, LM head (always bf16), greedy token */
+    /* 9: final norm, LM head (bf16 unless quantize_lm_head), greedy token */
     orc_rmsnorm(x, w->final_norm, H, c->rms_eps, a);
-    orc_gemv(0, c->tied_embeddings ? w->embed : w->lm_head, NULL, NULL, 0, V, H, a, logits);
+    lm_head(c, w, a, logits);
     if (next_token) *next_token = orc_argmax(logits, V);
 
     free(x); free(a); free(q); free(k); free(v); free(o); free(t); free(gt); free(up); free(m);
@@ -553,7 +569,7 @@ int orc_head_step(const orc_config* c, const orc_weights* w, const float* x_in, 
     const int H = c->hidden, V = c->vocab;
     float* a = (float*)malloc(sizeof(float) * H);
     orc_rmsnorm(x_in, w->final_norm, H, c->rms_eps, a);
-    orc_gemv(0, c->tied_embeddings ? w->embed : w->lm_head, NULL, NULL, 0, V, H, a, logits);
+    lm_head(c, w, a, logits);
     if (next_token) *next_token = orc_argmax(logits, V);
     free(a);
     return 0;

@@ -37,7 +37,7 @@ class _Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("hidden", "n_layers", "n_q_heads", "n_kv_heads", "head_dim",
                                          "mlp", "vocab", "max_seq", "tied_embeddings")] + [
         ("rms_eps", C.c_float), ("rope_theta", C.c_float),
-        ("wdtype", C.c_int32), ("group_size", C.c_int32), ("round_kv", C.c_int32)]
+        ("wdtype", C.c_int32), ("group_size", C.c_int32), ("round_kv", C.c_int32), ("quantize_lm_head", C.c_int32)]
 
 
 _PP = C.POINTER(C.c_void_p)
@@ -46,7 +46,8 @@ _PP = C.POINTER(C.c_void_p)
 class _Weights(C.Structure):
     _fields_ = [("embed", C.c_void_p), ("lm_head", C.c_void_p), ("final_norm", C.c_void_p),
                 ("attn_norm", _PP), ("mlp_norm", _PP),
-                ("w", _PP * 7), ("scale", _PP * 7), ("zero", _PP * 7)]
+                ("w", _PP * 7), ("scale", _PP * 7), ("zero", _PP * 7),
+                ("lm_head_q", C.c_void_p), ("lm_head_scale", C.c_void_p), ("lm_head_zero", C.c_void_p)]
 
 
 _lib = None
@@ -298,13 +299,17 @@ class Model:
     (int4) ``<kind>_zero`` lists of uint16 arrays.
     """
 
-    def __init__(self, shape, weights: Dict, wdtype: int = W_BF16, group: int = 128, round_kv: bool = True):
+    def __init__(self, shape, weights: Dict, wdtype: int = W_BF16, group: int = 128, round_kv: bool = True,
+                 quantize_lm_head: bool = False):
+        """``quantize_lm_head``: the LM head is read from ``weights["lm_head_q"]`` / ``["lm_head_scale"]`` /
+        ``["lm_head_zero"]`` (see ``quantize_lm_head``), quantised like the layers."""
         self.shape = Shape.of(shape)
         s = self.shape
         self.wdtype, self.group = wdtype, group
         self._keep: List[np.ndarray] = []
+        qlm = bool(quantize_lm_head) and wdtype != W_BF16
         self.cfg = _Config(s.hidden, s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, s.mlp, s.vocab,
-                           s.max_seq, int(s.tied), s.rms_eps, s.rope_theta, wdtype, group, int(round_kv))
+                           s.max_seq, int(s.tied), s.rms_eps, s.rope_theta, wdtype, group, int(round_kv), int(qlm))
         w = _Weights()
         w.embed = self._hold(weights["embed"], np.uint16)
         w.lm_head = None if s.tied else self._hold(weights["lm_head"], np.uint16)
@@ -318,6 +323,11 @@ class Model:
                 w.scale[i] = self._ptr_array(weights[kind + "_scale"], np.uint16)
             if wdtype == W_INT4:
                 w.zero[i] = self._ptr_array(weights[kind + "_zero"], np.uint16)
+        if qlm:
+            w.lm_head_q = self._hold(weights["lm_head_q"], wdt)
+            w.lm_head_scale = self._hold(weights["lm_head_scale"], np.uint16)
+            if wdtype == W_INT4:
+                w.lm_head_zero = self._hold(weights["lm_head_zero"], np.uint16)
         self.w = w
 
     def _hold(self, a, dtype) -> int:
@@ -414,6 +424,18 @@ def quantize_weights(weights: Dict, wdtype: int, group: int = 128) -> Dict:
         out[kind + "_scale"] = ss
         if wdtype == W_INT4:
             out[kind + "_zero"] = zs
+    return out
+
+
+def quantize_lm_head(weights: Dict, wdtype: int, group: int = 128, tied: bool = False) -> Dict:
+    """Adds ``lm_head_q`` / ``lm_head_scale`` (/ ``lm_head_zero``): the oracle's own quantiser applied to the LM head
+    matrix (the embedding matrix when tied).  The bf16 matrices stay in the dict."""
+    out = dict(weights)
+    W = weights["embed"] if (tied or weights.get("lm_head") is None) else weights["lm_head"]
+    if wdtype == W_INT8:
+        out["lm_head_q"], out["lm_head_scale"] = quantize_int8(W)
+    elif wdtype == W_INT4:
+        out["lm_head_q"], out["lm_head_scale"], out["lm_head_zero"] = quantize_int4(W, group)
     return out
 
 

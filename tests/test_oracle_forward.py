@@ -71,7 +71,7 @@ def dense_forward(shape, W, tokens, round_kv=True):
         X = X + ((G / (1.0 + np.exp(-G))) * U) @ W["wdown"][l].T
         hidden.append(X.copy())
     Y = norm(X, W["final_norm"])
-    head = W["embed"] if shape.tied else W["lm_head"]
+    head = W["lm_head_deq"] if W.get("lm_head_deq") is not None else (W["embed"] if shape.tied else W["lm_head"])
     return Y @ head.T, np.stack(hidden, axis=1)
 
 
@@ -93,6 +93,15 @@ def to_f64(wnp, shape, wdtype=orc.W_BF16, group=128):
                 z = wnp[kind + "_zero"][l].view(np.float16).astype(np.float64)
                 mats.append((q - np.repeat(z, group, axis=1)) * np.repeat(s, group, axis=1))
         out[kind] = mats
+    if "lm_head_q" in wnp:                                           # a quantised LM head: its dequantised matrix
+        if wdtype == orc.W_INT8:
+            s = wnp["lm_head_scale"].view(np.float16).astype(np.float64)
+            out["lm_head_deq"] = wnp["lm_head_q"].astype(np.float64) * s[:, None]
+        else:
+            q = orc.unpack_int4(wnp["lm_head_q"]).astype(np.float64)
+            s = wnp["lm_head_scale"].view(np.float16).astype(np.float64)
+            z = wnp["lm_head_zero"].view(np.float16).astype(np.float64)
+            out["lm_head_deq"] = (q - np.repeat(z, group, axis=1)) * np.repeat(s, group, axis=1)
     return out
 
 
@@ -143,6 +152,32 @@ def test_quantised_decode_equals_dense_on_dequantised_matrices(wdtype):
         logits, nxt, hidden = model.decode_step(tok, t, kv)
         assert rel_l2(hidden, hidden_d[t]) < 2e-5
         assert rel_l2(logits, logits_d[t]) < 2e-5
+
+
+@pytest.mark.parametrize("wdtype", [orc.W_INT8, orc.W_INT4])
+@pytest.mark.parametrize("name", ["toy", "toy_ragged"])
+def test_quantised_lm_head_equals_dense_on_its_dequantised_matrix(wdtype, name):
+    """quantize_lm_head = 1: the LM head (the embedding matrix when tied) is quantised like the layers; the
+    embedding gather keeps reading bf16.  The logits must be those of the dense form with the dequantised head, and
+    must differ from the bf16-head logits (so the flag is not a no-op)."""
+    shape = inp.SHAPES[name]
+    group = 32 if name == "toy" else 8                               # toy_ragged: hidden 192, mlp 328 -> groups of 8
+    w = inp.make_weights(shape, seed=15, std=0.25 if name == "toy" else 0.08, norm_jitter=0.1)
+    wq = orc.quantize_weights(inp.weights_to_numpy(w), wdtype, group)
+    wq = orc.quantize_lm_head(wq, wdtype, group, tied=shape.tied)
+    model = orc.Model(shape, wq, wdtype=wdtype, group=group, quantize_lm_head=True)
+    plain = orc.Model(shape, wq, wdtype=wdtype, group=group)
+    toks = greedy_tokens(4, shape.vocab, 7)
+    logits_d, hidden_d = dense_forward(shape, to_f64(wq, shape, wdtype, group), toks)
+    kv, kv2 = model.new_cache(), plain.new_cache()
+    for t, tok in enumerate(toks):
+        logits, nxt, hidden = model.decode_step(tok, t, kv)
+        logits_p, _, hidden_p = plain.decode_step(tok, t, kv2)
+        assert rel_l2(logits, logits_d[t]) < 2e-5
+        assert np.array_equal(hidden, hidden_p)                      # the layers and the embedding row are untouched
+        assert rel_l2(logits, logits_p) > 1e-3
+        lg, nx = model.head_step(hidden[-1])
+        assert np.array_equal(lg, logits) and nx == nxt
 
 
 def test_layer_and_head_steps_compose_to_the_full_step():
