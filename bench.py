@@ -43,11 +43,16 @@ WORKLOADS = {
     "smollm2_135m_bf16_pos0": ("smollm2_135m", "bf16", 0),
     "llama32_1b_bf16_pos0": ("llama32_1b", "bf16", 0),
     "llama32_1b_int8_pos0": ("llama32_1b", "int8", 0),
+    # quantize_lm_head = 1: the LM head streamed as int8 too (the other reading of the paper for an untied head)
+    "tinyllama_1b_int8_qhead_pos0": ("tinyllama_1b", "int8", 0),
+    "llama3_8b_int8_qhead_pos0": ("llama3_8b", "int8", 0),
 }
+QHEAD = {"tinyllama_1b_int8_qhead_pos0", "llama3_8b_int8_qhead_pos0"}
 DEFAULT_WORKLOAD = "llama3_8b_bf16_pos0"      # the largest single-GPU configuration
 OTHER = ["llama3_8b_int8_pos0", "tinyllama_1b_bf16_pos0", "tinyllama_1b_int8_pos0", "tinyllama_1b_int4_pos0",
          "smollm2_135m_bf16_pos0", "tinyllama_1b_bf16_pos1024", "tinyllama_1b_int8_pos512", "llama3_8b_int8_pos4096",
-         "llama3_8b_bf16_pos4096", "llama32_1b_bf16_pos0", "llama32_1b_int8_pos0"]
+         "llama3_8b_bf16_pos4096", "llama32_1b_bf16_pos0", "llama32_1b_int8_pos0", "tinyllama_1b_int8_qhead_pos0",
+         "llama3_8b_int8_qhead_pos0"]
 # device-resident multi-token runs (amk_decode_greedy: the token is fed back on the device): (shape, dtype, steps)
 SUSTAINED = [("smollm2_135m", "bf16", 256), ("tinyllama_1b", "bf16", 256)]
 METRIC = "batch-1 decode us/token; achieved HBM GB/s vs B200 measured peak"
@@ -141,10 +146,15 @@ def build_decoder(workload: str, device, sync_mode: int = 0):
     from paper_2606_09682_b200 import binding as amk
     name, wd, pos = WORKLOADS[workload]
     shape = inp.SHAPES[name]
+    qhead = workload in QHEAD
     w = inp.make_weights(shape, SEED, device=device)
     wq = amk.quantize_weights(w, wd)
-    dec = amk.Decoder(shape, wq, wd, flags=amk.AMK_FLAG_DEBUG_HIDDEN, sync_mode=sync_mode, device=device)
+    if qhead:
+        wq = amk.quantize_lm_head(wq, wd, shape.tied)
+    dec = amk.Decoder(shape, wq, wd, flags=amk.AMK_FLAG_DEBUG_HIDDEN, sync_mode=sync_mode, device=device,
+                      quantize_lm_head=qhead)
     keep = {k: w[k][0] for k in inp.KINDS}
+    keep["qhead"] = qhead
     keep.update(attn_norm=w["attn_norm"][0], mlp_norm=w["mlp_norm"][0], final_norm=w["final_norm"], embed=w["embed"],
                 lm_head=None if shape.tied else w["lm_head"])
     del w, wq
@@ -224,12 +234,15 @@ class OracleSample:
             w = inp.weights_to_numpy(inp.make_weights(s1, SEED, device="cpu"))
             tok = inp.make_token(shape, SEED)
         else:
-            w = {k: [inp.bits(keep[k])] for k in inp.KINDS}
+            w = {k: [inp.bits(keep[k])] for k in inp.KINDS if k in keep}
             w.update(attn_norm=[inp.bits(keep["attn_norm"])], mlp_norm=[inp.bits(keep["mlp_norm"])],
                      final_norm=inp.bits(keep["final_norm"]), embed=inp.bits(keep["embed"]),
                      lm_head=None if shape.tied else inp.bits(keep["lm_head"]))
         wq = orc.quantize_weights(w, wdt, 128)
-        self.model = orc.Model(s1, wq, wdtype=wdt, group=128)
+        self.qhead = bool(keep and keep.get("qhead"))
+        if self.qhead:
+            wq = orc.quantize_lm_head(wq, wdt, 128, tied=shape.tied)
+        self.model = orc.Model(s1, wq, wdtype=wdt, group=128, quantize_lm_head=self.qhead)
         self.kv = np.zeros(orc.kv_elems(s1), dtype=np.uint16)
         if pos > 0:
             if kv_gpu is None:
@@ -295,7 +308,7 @@ def run_one(workload, device, steps, warmup, peak, sync_mode=0, evict_l2=False):
     else:
         per, _ = time_device(dec, tok, pos, kv, steps, warmup)
     parity, kernel_us, _ = gate_and_kernel_time(shape, wd, pos, dec, kv, tok, keep)
-    b = inp.streamed_bytes(shape, wd, pos)
+    b = inp.streamed_bytes(shape, wd, pos, quantize_lm_head=workload in QHEAD)
     us = float(np.mean(per))
     ach = b["total"] / (us * 1e-6) / 1e9
     res = {"workload": workload, "us_per_token": us if parity["pass"] else None, "median_us": float(np.median(per)),
@@ -368,7 +381,7 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     name, wd, pos = WORKLOADS[a.workload]
     shape = inp.SHAPES[name]
-    config = {"workload": f"{name} shape, {wd} weights, batch 1, decode position {pos}, "
+    config = {"workload": f"{name} shape, {wd} weights{' (LM head quantised too)' if a.workload in QHEAD else ''}, batch 1, decode position {pos}, "
                           f"{'pre-filled N(0,1) bf16 KV cache' if pos else 'empty KV cache'}, random-init N(0,0.02) weights",
               "l2": "inputs larger than L2: every step streams the whole weight set from HBM",
               "replicas": world}
@@ -453,7 +466,7 @@ def main():
 
     if rank == 0:
         peak, peak_src = measured_peak()
-        b = inp.streamed_bytes(shape, wd, pos)
+        b = inp.streamed_bytes(shape, wd, pos, quantize_lm_head=a.workload in QHEAD)
         us = total_ms * 1e3 / a.steps
         achieved = b["total"] / (us * 1e-6) / 1e9
         plan = dec.plan()

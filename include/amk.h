@@ -27,7 +27,7 @@
 extern "C" {
 #endif
 
-#define AMK_ABI_VERSION 1u
+#define AMK_ABI_VERSION 2u
 
 typedef enum {
   AMK_OK = 0,
@@ -93,7 +93,10 @@ typedef struct amk_config {
   float rope_theta;          /* rotary base; pairs (i, i + head_dim/2), no scaling                     */
   uint32_t wdtype;           /* amk_wdtype of the seven per-layer linears                              */
   uint32_t group_size;       /* int4: 128 (the only supported value); ignored otherwise                */
-  uint32_t quantize_lm_head; /* must be 0: embedding and LM head stay bf16, as in the paper            */
+  uint32_t quantize_lm_head; /* 0: the LM head stays bf16 (tied or not), as the paper says of the tied
+                                embedding matrix.  1 (int8 / int4 models only): the LM head GEMV streams a
+                                copy quantised like the layers (amk_weights.lm_head_q ...); the embedding
+                                gather still reads the bf16 matrix                                     */
   uint32_t wait_timeout_us;  /* bound on every device-side wait; 0 = 200000                            */
   uint32_t flags;            /* AMK_FLAG_*                                                             */
   /* tuning knobs, 0 = automatic */
@@ -129,6 +132,11 @@ typedef struct amk_weights {
   const void* const* linear[AMK_LIN_COUNT]; /* [L] each: q, k, v, o, gate, up, down                   */
   const void* const* scale[AMK_LIN_COUNT];  /* [L] each; NULL arrays for bf16                         */
   const void* const* zero[AMK_LIN_COUNT];   /* [L] each; int4 only                                    */
+  /* quantize_lm_head = 1 only: the LM head matrix (the embedding matrix when tied) quantised like a layer
+   * linear of [V][H]: codes, fp16 scales (int8 [V]; int4 [V][H/128]) and, for int4, fp16 zero points */
+  const void* lm_head_q;
+  const void* lm_head_scale;
+  const void* lm_head_zero;
 } amk_weights;
 
 typedef struct amk_handle amk_handle;

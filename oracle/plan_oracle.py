@@ -8,7 +8,8 @@ model is decided by brute force -- an explicit graph of (task, block) events for
 reachability -- instead of the checker's rule about all-to-all joins.
 
 is_safe(words, model) -> (bool, reason).  `model` is a dict with hidden, n_layers, n_q_heads, n_kv_heads,
-head_dim, mlp, vocab, wdtype (0 bf16, 1 int8, 2 int4), stage_bytes, n_blocks.
+head_dim, mlp, vocab, wdtype (0 bf16, 1 int8, 2 int4), stage_bytes, n_blocks, and optionally lm_wdtype (the LM
+head's dtype when it is quantised like the layers; 0 otherwise).
 """
 from collections import deque
 
@@ -174,7 +175,8 @@ def is_safe(words, model):
 
     H, I, V, wd = model["hidden"], model["mlp"], model["vocab"], model["wdtype"]
     qd, kvd = model["n_q_heads"] * model["head_dim"], model["n_kv_heads"] * model["head_dim"]
-    shape = [(H, qd + 2 * kvd, 1, wd), (qd, H, 1, wd), (H, 2 * I, 2, wd), (I, H, 1, wd), (H, V, 1, 0)]
+    # (the LM head is bf16 unless the model says it is quantised like the layers)
+    shape = [(H, qd + 2 * kvd, 1, wd), (qd, H, 1, wd), (H, 2 * I, 2, wd), (I, H, 1, wd), (H, V, 1, model.get("lm_wdtype", 0))]
     # every row of every GEMV: exactly one producer
     for k in range(5):
         units = shape[k][1] // shape[k][2]

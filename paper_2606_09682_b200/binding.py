@@ -15,7 +15,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("AMK_LIB") or os.path.join(_HERE, "libamk.so")      # AMK_LIB: another build of the library
 
-AMK_ABI_VERSION = 1
+AMK_ABI_VERSION = 2
 AMK_OK, AMK_ERR_INVALID_ARG, AMK_ERR_UNSUPPORTED, AMK_ERR_CUDA, AMK_ERR_OOM = 0, 1, 2, 3, 4
 AMK_ERR_TIMEOUT, AMK_ERR_ABORTED, AMK_ERR_BAD_POS, AMK_ERR_BAD_TOKEN = 5, 6, 7, 8
 AMK_W_BF16, AMK_W_INT8, AMK_W_INT4 = 0, 1, 2
@@ -44,7 +44,8 @@ _PP = C.POINTER(C.c_void_p)
 class amk_weights(C.Structure):
     _fields_ = [("embed", C.c_void_p), ("lm_head", C.c_void_p), ("final_norm", C.c_void_p),
                 ("attn_norm", _PP), ("mlp_norm", _PP),
-                ("linear", _PP * 7), ("scale", _PP * 7), ("zero", _PP * 7)]
+                ("linear", _PP * 7), ("scale", _PP * 7), ("zero", _PP * 7),
+                ("lm_head_q", C.c_void_p), ("lm_head_scale", C.c_void_p), ("lm_head_zero", C.c_void_p)]
 
 
 class amk_plan(C.Structure):
@@ -109,7 +110,7 @@ def _check(code: int, what: str):
 
 def make_config(shape, wdtype: str = "bf16", flags: int = 0, wait_timeout_us: int = 0, stage_bytes: int = 0,
                 n_stages: int = 0, max_inflight: int = 0, group_size: int = 128, sync_mode: int = 1,
-                n_blocks: int = 0, l2_ahead: int = 0) -> amk_config:
+                n_blocks: int = 0, l2_ahead: int = 0, quantize_lm_head: bool = False) -> amk_config:
     """``shape``: any object with hidden, n_layers, n_q_heads, n_kv_heads, head_dim, mlp, vocab, max_seq,
     tied, rms_eps, rope_theta attributes."""
     c = amk_config()
@@ -123,6 +124,7 @@ def make_config(shape, wdtype: str = "bf16", flags: int = 0, wait_timeout_us: in
     c.wait_timeout_us, c.flags = wait_timeout_us, flags
     c.stage_bytes, c.n_stages, c.max_inflight = stage_bytes, n_stages, max_inflight
     c.sync_mode, c.n_blocks, c.l2_ahead = sync_mode, n_blocks, l2_ahead
+    c.quantize_lm_head = int(bool(quantize_lm_head))
     return c
 
 
@@ -226,6 +228,18 @@ def quantize_weights(weights: Dict, wdtype: str) -> Dict:
     return out
 
 
+def quantize_lm_head(weights: Dict, wdtype: str, tied: bool) -> Dict:
+    """Adds ``lm_head_q`` / ``lm_head_scale`` (/ ``lm_head_zero``): the library's quantiser applied to the LM head
+    matrix (the embedding matrix when tied), for a decoder created with ``quantize_lm_head=True``."""
+    out = dict(weights)
+    w = weights["embed"] if (tied or weights.get("lm_head") is None) else weights["lm_head"]
+    if wdtype == "int8":
+        out["lm_head_q"], out["lm_head_scale"] = amk_quantize_int8(w)
+    elif wdtype == "int4":
+        out["lm_head_q"], out["lm_head_scale"], out["lm_head_zero"] = amk_quantize_int4(w)
+    return out
+
+
 def _ptr_array(tensors: Sequence[torch.Tensor], keep: List):
     arr = (C.c_void_p * len(tensors))()
     for i, t in enumerate(tensors):
@@ -240,13 +254,16 @@ class Decoder:
 
     def __init__(self, shape, weights: Dict, wdtype: str = "bf16", flags: int = 0, wait_timeout_us: int = 0,
                  stage_bytes: int = 0, n_stages: int = 0, max_inflight: int = 0, sync_mode: int = 1,
-                 n_blocks: int = 0, l2_ahead: int = 0, device="cuda", guard_bytes: int = 0):
+                 n_blocks: int = 0, l2_ahead: int = 0, device="cuda", guard_bytes: int = 0,
+                 quantize_lm_head: bool = False):
         """``guard_bytes`` (a multiple of 256): the packed buffer, the workspace and the logits get that many bytes
         of a fixed pattern in front and behind, which ``guards_intact()`` checks -- a stand-in for a memory checker."""
         self.shape, self.wdtype = shape, wdtype
         self.device = torch.device(device)
         self.cfg = make_config(shape, wdtype, flags, wait_timeout_us, stage_bytes, n_stages, max_inflight,
-                               sync_mode=sync_mode, n_blocks=n_blocks, l2_ahead=l2_ahead)
+                               sync_mode=sync_mode, n_blocks=n_blocks, l2_ahead=l2_ahead,
+                               quantize_lm_head=quantize_lm_head)
+        self.quantize_lm_head = bool(quantize_lm_head)
         assert guard_bytes % 256 == 0
         self._guard = guard_bytes
         self._guarded: List[torch.Tensor] = []
@@ -256,6 +273,10 @@ class Decoder:
         w = amk_weights()
         w.embed = weights["embed"].data_ptr()
         w.lm_head = None if shape.tied else weights["lm_head"].data_ptr()
+        if quantize_lm_head:
+            w.lm_head_q = weights["lm_head_q"].data_ptr()
+            w.lm_head_scale = weights["lm_head_scale"].data_ptr()
+            w.lm_head_zero = weights["lm_head_zero"].data_ptr() if wdtype == "int4" else None
         w.final_norm = weights["final_norm"].data_ptr()
         w.attn_norm = _ptr_array(weights["attn_norm"], keep)
         w.mlp_norm = _ptr_array(weights["mlp_norm"], keep)
@@ -334,7 +355,7 @@ class Decoder:
         qd, kvd = s.n_q_heads * s.head_dim, s.n_kv_heads * s.head_dim
         dims = [(qd, s.hidden), (kvd, s.hidden), (kvd, s.hidden), (s.hidden, qd), (s.mlp, s.hidden),
                 (s.mlp, s.hidden), (s.hidden, s.mlp), (s.vocab, s.hidden)][which]
-        wd = "bf16" if which == AMK_LIN_LM_HEAD else self.wdtype
+        wd = "bf16" if (which == AMK_LIN_LM_HEAD and not self.quantize_lm_head) else self.wdtype
         rows, cols = dims
         scale = zero = None
         if wd == "bf16":

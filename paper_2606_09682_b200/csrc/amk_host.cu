@@ -38,7 +38,7 @@ struct Plan {
   OpShape shape[5];
   std::vector<PlanOp> ops;
   std::vector<int> bounds[5];        // per op kind: unit boundaries of the slots (n_blocks + 1)
-  size_t scale_base = 0, scale_layer_stride = 0, scale_kind_off[4] = {0, 0, 0, 0};
+  size_t scale_base = 0, scale_layer_stride = 0, scale_kind_off[4] = {0, 0, 0, 0}, lm_scale_off = 0;
   size_t embed_off = 0, attn_norm_off = 0, mlp_norm_off = 0, final_norm_off = 0, packed_total = 0;
   size_t weight_stream_bytes = 0;    // op regions + scale regions (what a token streams)
   size_t n_tiles = 0;                // total ring tiles over all blocks
@@ -74,7 +74,8 @@ amk_status check_config(const amk_config* c) {
   if (c->head_dim != 64 && c->head_dim != 128) return AMK_ERR_UNSUPPORTED;
   if (c->n_q_heads % c->n_kv_heads) return AMK_ERR_UNSUPPORTED;
   if (c->n_q_heads / c->n_kv_heads > (uint32_t)kMaxRep) return AMK_ERR_UNSUPPORTED;
-  if (c->quantize_lm_head) return AMK_ERR_UNSUPPORTED;
+  if (c->quantize_lm_head > 1) return AMK_ERR_INVALID_ARG;
+  if (c->quantize_lm_head && c->wdtype == AMK_W_BF16) return AMK_ERR_UNSUPPORTED;   // nothing to quantise it like
   const uint32_t kdiv = (c->wdtype == AMK_W_INT4) ? 128 : 64;
   const uint32_t qdim = c->n_q_heads * c->head_dim;
   if (c->hidden % kdiv || c->mlp % kdiv || qdim % kdiv) return AMK_ERR_UNSUPPORTED;
@@ -102,7 +103,7 @@ Plan make_plan(const amk_config* c, int n_blocks, const double* weights, bool wi
   pl.shape[OP_O] = OpShape{qd, H, 1, wd};
   pl.shape[OP_GATEUP] = OpShape{H, 2 * I, 2, wd};
   pl.shape[OP_DOWN] = OpShape{I, H, 1, wd};
-  pl.shape[OP_LMHEAD] = OpShape{H, V, 1, W_BF16};
+  pl.shape[OP_LMHEAD] = OpShape{H, V, 1, c->quantize_lm_head ? wd : (int)W_BF16};
   for (int k = 0; k < 5; k++) {
     pl.bounds[k].resize(n_blocks + 1);
     make_bounds(pl.shape[k].rows / pl.shape[k].unit_rows, n_blocks, weights, pl.bounds[k].data());
@@ -138,6 +139,11 @@ Plan make_plan(const amk_config* c, int n_blocks, const double* weights, bool wi
     for (auto& op : pl.ops)
       if (op.kind != OP_LMHEAD) op.scale_off = pl.scale_base + (size_t)op.layer * k + pl.scale_kind_off[op.kind];
     off = align_up(off + (size_t)L * k);
+    if (c->quantize_lm_head) {
+      pl.lm_scale_off = off;
+      pl.ops.back().scale_off = off;
+      off = align_up(off + (size_t)V * 2);
+    }
   }
   pl.weight_stream_bytes = off;
   pl.embed_off = off;      off = align_up(off + (size_t)V * H * 2);
@@ -303,7 +309,9 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
   if (!wts || !packed_dev || !workspace_dev) return AMK_ERR_INVALID_ARG;
   if (((uintptr_t)packed_dev | (uintptr_t)workspace_dev) & (kAlign - 1)) return AMK_ERR_INVALID_ARG;
   if (!wts->embed || !wts->final_norm || !wts->attn_norm || !wts->mlp_norm) return AMK_ERR_INVALID_ARG;
-  if (!cfg->tied_embeddings && !wts->lm_head) return AMK_ERR_INVALID_ARG;
+  if (!cfg->tied_embeddings && !wts->lm_head && !cfg->quantize_lm_head) return AMK_ERR_INVALID_ARG;
+  if (cfg->quantize_lm_head && (!wts->lm_head_q || !wts->lm_head_scale || (cfg->wdtype == AMK_W_INT4 && !wts->lm_head_zero)))
+    return AMK_ERR_INVALID_ARG;
   for (int k = 0; k < AMK_LIN_COUNT; k++) {
     if (!wts->linear[k]) return AMK_ERR_INVALID_ARG;
     if (cfg->wdtype != AMK_W_BF16 && !wts->scale[k]) return AMK_ERR_INVALID_ARG;
@@ -419,7 +427,7 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     size_t kmax = (size_t)(H > I ? H : I);
     if ((size_t)qd > kmax) kmax = qd;
     size_t act = kmax * (cfg->wdtype == AMK_W_BF16 ? 4 : 3);   // bf16 high + low halves, or three int8 digits
-    if ((size_t)H * 4 > act) act = (size_t)H * 4;               // the LM head is always bf16
+    if (!cfg->quantize_lm_head && (size_t)H * 4 > act) act = (size_t)H * 4;   // a bf16 LM head in an integer model
     // attention scratch: q vectors, per-warp partial outputs, the new K / V rows, the scores of the longest chunk
     int lc_max = 0, c_max = 0;
     attn_chunks((int)cfg->max_seq, (int)n_blocks, (int)cfg->n_kv_heads, &lc_max, &c_max);
@@ -507,7 +515,15 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
         case OP_O: okp = lin(0, AMK_LIN_O); break;
         case OP_GATEUP: s.mode = 2; okp = lin(0, AMK_LIN_GATE) & lin(1, AMK_LIN_UP); break;
         case OP_DOWN: okp = lin(0, AMK_LIN_DOWN); break;
-        default: s.w[0] = cfg->tied_embeddings ? wts->embed : wts->lm_head; break;
+        default:
+          if (cfg->quantize_lm_head) {
+            s.w[0] = wts->lm_head_q;
+            s.scale[0] = wts->lm_head_scale;
+            s.zero[0] = wts->lm_head_zero;
+          } else {
+            s.w[0] = cfg->tied_embeddings ? wts->embed : wts->lm_head;
+          }
+          break;
       }
       if (!okp) { status = AMK_ERR_INVALID_ARG; goto fail; }
       AMK_CUDA(launch_pack(d, s, h->packed, n_blocks, (int)stage_bytes, false, stream));
@@ -540,6 +556,7 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     p.scale_base = h->pl.scale_base;
     p.scale_layer_stride = (unsigned)h->pl.scale_layer_stride;
     for (int k = 0; k < 4; k++) p.scale_kind_off[k] = (unsigned)h->pl.scale_kind_off[k];
+    p.lm_scale_off = h->pl.lm_scale_off;
     p.embed = (const unsigned short*)(h->packed + h->pl.embed_off);
     p.attn_norm = (const unsigned short*)(h->packed + h->pl.attn_norm_off);
     p.mlp_norm = (const unsigned short*)(h->packed + h->pl.mlp_norm_off);
@@ -997,7 +1014,8 @@ extern "C" amk_status amk_plan_check(const amk_config* cfg, const uint64_t* t, s
   // ---- op table: the model's GEMVs in step order, regions inside the weight area and disjoint -------------
   const int H = cfg->hidden, I = cfg->mlp, V = cfg->vocab, wd = (int)cfg->wdtype;
   const int qd = cfg->n_q_heads * cfg->head_dim, kvd = cfg->n_kv_heads * cfg->head_dim;
-  const OpShape want[5] = {{H, qd + 2 * kvd, 1, wd}, {qd, H, 1, wd}, {H, 2 * I, 2, wd}, {I, H, 1, wd}, {H, V, 1, W_BF16}};
+  const OpShape want[5] = {{H, qd + 2 * kvd, 1, wd}, {qd, H, 1, wd}, {H, 2 * I, 2, wd}, {I, H, 1, wd},
+                           {H, V, 1, cfg->quantize_lm_head ? wd : (int)W_BF16}};
   long long prev_end = 0;
   for (long long i = 0; i < n_ops; i++) {
     const uint64_t* o = ops + (size_t)i * kOpWords;

@@ -67,6 +67,7 @@ struct KParams {
   unsigned long long scale_base;          // int8: fp16 row scales, op-major in virtual row order
   unsigned scale_layer_stride;            // bytes per layer
   unsigned scale_kind_off[4];             // byte offset of each op kind inside a layer's scales
+  unsigned long long lm_scale_off;        // int8 LM head (quantize_lm_head): its fp16 row scales
   const unsigned short* embed;            // bf16 [V][H], canonical copy
   const unsigned short* attn_norm;        // bf16 [L][H]
   const unsigned short* mlp_norm;         // bf16 [L][H]

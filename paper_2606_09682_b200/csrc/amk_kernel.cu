@@ -580,13 +580,14 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int kind
 // ------------------------------------------------------------------------------------------------
 // One matrix-vector product with its fused prologue (gather / RMSNorm) and epilogue.
 // ------------------------------------------------------------------------------------------------
-// LMH: the LM head (always bf16, compiled apart from the per-layer code so that a quantised model's layers carry
-// neither its code nor its registers); otherwise `kind_rt` is one of the four per-layer products, of dtype WDL.
+// LMH: the LM head (bf16 unless the configuration quantises it; compiled apart from the per-layer code so that a
+// quantised model's layers carry neither its code nor its registers); otherwise `kind_rt` is one of the four
+// per-layer products.  WDL is the dtype of the product's weights.
 template <int WDL, bool LMH>
 __device__ __forceinline__ bool gemv_op(Ctx& c, int kind_rt, int l) {
   const KParams& p = c.p;
   const int kind = LMH ? (int)OP_LMHEAD : kind_rt;
-  constexpr int WD = LMH ? (int)W_BF16 : WDL;
+  constexpr int WD = WDL;
   const OpShape d = p.shape[kind];
   const int task = (kind == OP_LMHEAD) ? 5 * p.L : 5 * l + (kind == OP_QKV ? 0 : kind + 1);
   Slice sl;
@@ -636,7 +637,7 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind_rt, int l) {
       if (raddr) rraw = ld_pair(raddr);
       if (d.wdtype == W_INT8) {
         const __half* scales = reinterpret_cast<const __half*>(
-            p.packed + p.scale_base + (size_t)l * p.scale_layer_stride + p.scale_kind_off[kind]);
+            p.packed + (LMH ? p.lm_scale_off : p.scale_base + (size_t)l * p.scale_layer_stride + p.scale_kind_off[kind]));
         if (kind == OP_GATEUP) {
           sh0 = __ldg(scales + vrow0 + 2 * c.tid);
           sh1 = __ldg(scales + vrow0 + 2 * c.tid + 1);
@@ -1164,11 +1165,12 @@ __device__ __forceinline__ bool attention_phase(Ctx& c, int l) {
 
 // The last task of the step: final norm, LM head, greedy token.  Out of line and with its own context: the
 // per-layer loop above it keeps its registers for the code that runs 4 L times.
+template <int WD>
 __device__ __noinline__ void lm_head_task(const KParams& p, SmemHeader* sh, unsigned char* xs, unsigned char* ring,
                                           int cta, int nblk, int stage, unsigned parity, int token) {
   const int tid = threadIdx.x;
   Ctx c{p, sh, xs, ring, tid, tid >> 5, tid & 31, cta, nblk, stage, parity, token, 1.0f, false};
-  gemv_op<W_BF16, true>(c, (int)OP_LMHEAD, p.L);
+  gemv_op<WD, true>(c, (int)OP_LMHEAD, p.L);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1351,7 +1353,11 @@ __global__ void __launch_bounds__(kThreads, 1) amk_decode_kernel(const __grid_co
     if (k == 1) ok = attention_phase<HD>(c, l);
     else ok = gemv_op<WDL, false>(c, k == 0 ? (int)OP_QKV : k - 1, l);
   }
-  if (ok) lm_head_task(p, sh, xs, ring, cta, nblk, c.stage, c.parity, token);
+  if (ok) {
+    // the LM head is bf16 unless the configuration quantises it like the layers
+    if (WDL == W_BF16 || p.shape[OP_LMHEAD].wdtype == W_BF16) lm_head_task<W_BF16>(p, sh, xs, ring, cta, nblk, c.stage, c.parity, token);
+    else lm_head_task<WDL>(p, sh, xs, ring, cta, nblk, c.stage, c.parity, token);
+  }
   // (every consumer warp stamps; the latest store of the latest block is the kernel's end)
   if (lane == 0) atomicMax(p.ktime + 2 * blockIdx.x + 1, globaltimer_ns());
 }

@@ -147,8 +147,10 @@ def weights_to_numpy(w: Dict) -> Dict:
     return out
 
 
-def streamed_bytes(shape: ModelShape, wdtype: str = "bf16", pos: int = 0, group: int = 128) -> Dict[str, float]:
-    """Algorithmic bytes one decode step must move: weights + scales + KV read/write + activations."""
+def streamed_bytes(shape: ModelShape, wdtype: str = "bf16", pos: int = 0, group: int = 128,
+                   quantize_lm_head: bool = False) -> Dict[str, float]:
+    """Algorithmic bytes one decode step must move: weights + scales + KV read/write + activations.
+    ``quantize_lm_head``: the LM head is streamed at the layers' width (with its scales) instead of as bf16."""
     H, L, I, V = shape.hidden, shape.n_layers, shape.mlp, shape.vocab
     nq, nkv, hd = shape.n_q_heads, shape.n_kv_heads, shape.head_dim
     lin = sum(r * c for r, c in (shape.linear_dims(k) for k in KINDS))
@@ -161,8 +163,13 @@ def streamed_bytes(shape: ModelShape, wdtype: str = "bf16", pos: int = 0, group:
         wl, sc = 0.5 * lin, 4.0 * lin / group
     else:
         raise ValueError(wdtype)
-    weights = L * wl + 2.0 * V * H + 2.0 * (2 * L + 1) * H + 2.0 * H      # linears + LM head + norms + one embedding row
-    scales = L * sc
+    head, head_sc = 2.0 * V * H, 0.0
+    if quantize_lm_head and wdtype == "int8":
+        head, head_sc = 1.0 * V * H, 2.0 * V
+    elif quantize_lm_head and wdtype == "int4":
+        head, head_sc = 0.5 * V * H, 4.0 * V * H / group
+    weights = L * wl + head + 2.0 * (2 * L + 1) * H + 2.0 * H            # linears + LM head + norms + one embedding row
+    scales = L * sc + head_sc
     kv = 2.0 * L * nkv * hd * 2 * pos + 2.0 * L * nkv * hd * 2
     act = 4.0 * (L * (4 * H + (nq + 2 * nkv) * hd + nq * hd + 2 * I) + 2 * H) + 4.0 * V
     return {"weights": weights, "scales": scales, "kv": kv, "act": act, "total": weights + scales + kv + act}

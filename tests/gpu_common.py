@@ -30,10 +30,13 @@ def bf16_ulp_distance(a_bits, b_bits):
     return np.abs(key(a_bits) - key(b_bits))
 
 
-def oracle_model(shape, weights_gpu, wdtype):
+def oracle_model(shape, weights_gpu, wdtype, quantize_lm_head=False):
+    """The oracle's model of the same seeded bf16 weights, quantised by the oracle's own quantiser."""
     wnp = inp.weights_to_numpy(weights_gpu)
     wq = orc.quantize_weights(wnp, WD[wdtype], 128)
-    return orc.Model(shape, wq, wdtype=WD[wdtype], group=128), wq
+    if quantize_lm_head:
+        wq = orc.quantize_lm_head(wq, WD[wdtype], 128, tied=shape.tied)
+    return orc.Model(shape, wq, wdtype=WD[wdtype], group=128, quantize_lm_head=quantize_lm_head), wq
 
 
 def check_argmax(logits_oracle, tok_gpu):

@@ -85,10 +85,14 @@ def test_size_queries_and_argument_checks(amk):
     cfg = amk.make_config(inp.SHAPES["mini"], "bf16")
     cfg.abi_version = 99
     assert amk.lib.amk_kv_bytes(C.byref(cfg), C.byref(n)) == amk.AMK_ERR_INVALID_ARG
-    for field, val in (("head_dim", 48), ("n_q_heads", 3), ("quantize_lm_head", 1)):
+    for field, val in (("head_dim", 48), ("n_q_heads", 3), ("quantize_lm_head", 1)):     # (a bf16 model has nothing to quantise its head like)
         cfg = amk.make_config(inp.SHAPES["mini"], "bf16")
         setattr(cfg, field, val)
         assert amk.lib.amk_packed_bytes(C.byref(cfg), C.byref(n)) == amk.AMK_ERR_UNSUPPORTED, field
+    cfg = amk.make_config(inp.SHAPES["mini"], "int8", quantize_lm_head=True)
+    assert amk.lib.amk_packed_bytes(C.byref(cfg), C.byref(n)) == amk.AMK_OK
+    cfg.quantize_lm_head = 2
+    assert amk.lib.amk_packed_bytes(C.byref(cfg), C.byref(n)) == amk.AMK_ERR_INVALID_ARG
     # limits of the plan: a task id is kept in 11 bits; sync_mode is 0 (automatic), 1 or 2
     cfg = amk.make_config(inp.SHAPES["mini"], "bf16")
     cfg.n_layers = 410

@@ -25,11 +25,13 @@ def amk():
     return binding
 
 
-def _build(amk, name, wdtype, seed, **kw):
+def _build(amk, name, wdtype, seed, quantize_lm_head=False, **kw):
     shape = inp.SHAPES[name]
     w = inp.make_weights(shape, seed, device="cuda")
     wq = amk.quantize_weights(w, wdtype)
-    dec = amk.Decoder(shape, wq, wdtype, flags=amk.AMK_FLAG_DEBUG_HIDDEN, **kw)
+    if quantize_lm_head:
+        wq = amk.quantize_lm_head(wq, wdtype, shape.tied)
+    dec = amk.Decoder(shape, wq, wdtype, flags=amk.AMK_FLAG_DEBUG_HIDDEN, quantize_lm_head=quantize_lm_head, **kw)
     return shape, w, wq, dec
 
 
@@ -107,6 +109,17 @@ def test_tinyllama_shape(amk, wdtype, pos):
     kv_c = inp.bits(kv_g).copy()
     r = gc.compare_step(shape, dec, model, inp.make_token(shape, 0xA3C2), pos, kv_g, kv_c)
     print("tinyllama", wdtype, pos, r)
+    dec.close()
+
+
+@pytest.mark.parametrize("wdtype,pos", [("int8", 0), ("int4", 200)])
+def test_tinyllama_shape_quantised_lm_head(amk, wdtype, pos):
+    shape, w, _, dec = _build(amk, "tinyllama_1b", wdtype, 0xA3C2, quantize_lm_head=True)
+    model, _ = gc.oracle_model(shape, w, wdtype, quantize_lm_head=True)
+    kv_g = inp.make_kv_prefill(shape, 0xA3C2, pos, device="cuda")
+    kv_c = inp.bits(kv_g).copy()
+    r = gc.compare_step(shape, dec, model, inp.make_token(shape, 0xA3C2), pos, kv_g, kv_c)
+    print("tinyllama quantised head", wdtype, pos, r)
     dec.close()
 
 

@@ -11,13 +11,15 @@ pytestmark = pytest.mark.gpu
 import gpu_common as gc  # noqa: E402
 
 
-def _setup(name, wdtype, seed, std=0.05, norm_jitter=0.1, **kw):
+def _setup(name, wdtype, seed, std=0.05, norm_jitter=0.1, quantize_lm_head=False, **kw):
     from paper_2606_09682_b200 import binding as amk
     shape = inp.SHAPES[name]
     w = inp.make_weights(shape, seed, device="cuda", std=std, norm_jitter=norm_jitter)
     wq = amk.quantize_weights(w, wdtype)
-    dec = amk.Decoder(shape, wq, wdtype, flags=amk.AMK_FLAG_DEBUG_HIDDEN, **kw)
-    model, _ = gc.oracle_model(shape, w, wdtype)
+    if quantize_lm_head:
+        wq = amk.quantize_lm_head(wq, wdtype, shape.tied)
+    dec = amk.Decoder(shape, wq, wdtype, flags=amk.AMK_FLAG_DEBUG_HIDDEN, quantize_lm_head=quantize_lm_head, **kw)
+    model, _ = gc.oracle_model(shape, w, wdtype, quantize_lm_head)
     return shape, dec, model
 
 
@@ -37,6 +39,21 @@ def test_multi_step_decode_matches_oracle(name, wdtype):
         r = gc.compare_step(shape, dec, model, tok, pos, kv_g, kv_c)
         worst = {k: max(worst[k], r[k]) for k in worst}
     print(name, wdtype, worst)
+    dec.close()
+
+
+@pytest.mark.parametrize("name,wdtype", [("mini", "int8"), ("mini_ragged", "int8"), ("mini_wide", "int4"),
+                                         ("mini_hd128", "int4")])
+def test_quantised_lm_head(name, wdtype):
+    """quantize_lm_head = 1: the LM head GEMV streams codes quantised like the layers (a quantised copy of the
+    embedding matrix for the tied mini_ragged shape), against the oracle with the same reading switched on."""
+    shape, dec, model = _setup(name, wdtype, seed=27, quantize_lm_head=True)
+    kv_g, kv_c = dec.new_cache(), model.new_cache()
+    rng = np.random.default_rng(4)
+    for pos in range(4):
+        tok = int(rng.integers(0, shape.vocab))
+        r = gc.compare_step(shape, dec, model, tok, pos, kv_g, kv_c)
+        print(name, wdtype, "quantised head", pos, r)
     dec.close()
 
 

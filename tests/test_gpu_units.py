@@ -67,6 +67,28 @@ def test_packed_layout_unpacks_bit_exact(amk, name, wdtype):
     dec.close()
 
 
+@pytest.mark.parametrize("name,wdtype", [("mini_ragged", "int8"), ("mini_wide", "int4")])
+def test_quantised_lm_head_unpacks_bit_exact(amk, name, wdtype):
+    """With quantize_lm_head the packed LM head holds the codes, scales and zero points it was given -- which are
+    the oracle quantiser's, bit for bit, of the LM head matrix (of the embedding matrix for the tied shape)."""
+    shape = inp.SHAPES[name]
+    w = inp.make_weights(shape, 52, device="cuda")
+    wq = amk.quantize_lm_head(amk.quantize_weights(w, wdtype), wdtype, shape.tied)
+    dec = amk.Decoder(shape, wq, wdtype, quantize_lm_head=True)
+    out, sc, zr = dec.amk_debug_unpack(0, amk.AMK_LIN_LM_HEAD)
+    assert torch.equal(out.view(torch.uint8), wq["lm_head_q"].view(torch.uint8))
+    assert torch.equal(sc.view(torch.int16), wq["lm_head_scale"].view(torch.int16))
+    head = inp.bits(w["embed"] if shape.tied else w["lm_head"])
+    if wdtype == "int8":
+        qo, so = orc.quantize_int8(head)
+    else:
+        qo, so, zo = orc.quantize_int4(head, 128)
+        assert torch.equal(zr.view(torch.int16), wq["lm_head_zero"].view(torch.int16))
+        assert np.array_equal(inp.bits(zr), zo)
+    assert np.array_equal(out.cpu().numpy().view(qo.dtype), qo) and np.array_equal(inp.bits(sc), so)
+    dec.close()
+
+
 def test_bounded_wait_reports_timeout_and_recovers(amk):
     """A signal that never comes: every waiter gives up after the time limit, the status says which join,
     and the following step is correct again.  Nothing traps or hangs."""

@@ -14,6 +14,7 @@ from paper_2606_09682_b200 import inputs as inp
 WD = {"bf16": 0, "int8": 1, "int4": 2}
 CASES = [("mini", "bf16", 148), ("mini_ragged", "int8", 132), ("mini_hd128", "int4", 7), ("mini_wide", "int4", 148),
          ("tinyllama_1b", "int8", 148), ("smollm2_135m", "bf16", 148), ("llama3_8b", "bf16", 148)]
+QHEAD_CASES = [("mini_ragged", "int8", 132), ("mini_wide", "int4", 148), ("tinyllama_1b", "int8", 148)]
 
 
 def _plan(name, wdtype, n_blocks, **kw):
@@ -22,7 +23,8 @@ def _plan(name, wdtype, n_blocks, **kw):
     words = amk.amk_plan_export(cfg)
     model = dict(hidden=shape.hidden, n_layers=shape.n_layers, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
                  head_dim=shape.head_dim, mlp=shape.mlp, vocab=shape.vocab, wdtype=WD[wdtype],
-                 stage_bytes=int(words[4]), n_blocks=n_blocks)
+                 stage_bytes=int(words[4]), n_blocks=n_blocks,
+                 lm_wdtype=WD[wdtype] if kw.get("quantize_lm_head") else 0)
     return cfg, words, model
 
 
@@ -43,6 +45,19 @@ def test_real_plans_are_accepted_by_checker_and_oracle(name, wdtype, n_blocks):
     assert st == amk.AMK_OK, why
     ok, why = plan_oracle.is_safe(words, model)
     assert ok, why
+
+
+@pytest.mark.parametrize("name,wdtype,n_blocks", QHEAD_CASES)
+def test_plans_with_a_quantised_lm_head(name, wdtype, n_blocks):
+    cfg, words, model = _plan(name, wdtype, n_blocks, quantize_lm_head=True)
+    st, why = amk.amk_plan_check(cfg, words)
+    assert st == amk.AMK_OK, why
+    ok, why = plan_oracle.is_safe(words, model)
+    assert ok, why
+    # the same tables are not those of the bf16-head model, for either judge
+    cfg0, words0, model0 = _plan(name, wdtype, n_blocks)
+    assert amk.amk_plan_check(cfg0, words)[0] != amk.AMK_OK
+    assert not plan_oracle.is_safe(words, model0)[0]
 
 
 def test_other_stage_sizes_are_accepted():
