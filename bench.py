@@ -33,6 +33,7 @@ WORKLOADS = {
     # name: (shape, weight dtype, position)
     "llama3_8b_bf16_pos0": ("llama3_8b", "bf16", 0),
     "llama3_8b_int8_pos0": ("llama3_8b", "int8", 0),
+    "llama3_8b_int4_pos0": ("llama3_8b", "int4", 0),
     "llama3_8b_bf16_pos4096": ("llama3_8b", "bf16", 4096),
     "llama3_8b_int8_pos4096": ("llama3_8b", "int8", 4096),
     "tinyllama_1b_int8_pos512": ("tinyllama_1b", "int8", 512),
@@ -43,6 +44,10 @@ WORKLOADS = {
     "smollm2_135m_bf16_pos0": ("smollm2_135m", "bf16", 0),
     "llama32_1b_bf16_pos0": ("llama32_1b", "bf16", 0),
     "llama32_1b_int8_pos0": ("llama32_1b", "int8", 0),
+    # the paper's 4-layer "small" model (622.9 MB bf16; its Table 10 quotes int8 at 1.12x over bf16 on an RTX 5090)
+    "paper_small_bf16_pos0": ("paper_small", "bf16", 0),
+    "paper_small_int8_pos0": ("paper_small", "int8", 0),
+    "paper_small_int4_pos0": ("paper_small", "int4", 0),
     # quantize_lm_head = 1: the LM head streamed as int8 too (the other reading of the paper for an untied head)
     "tinyllama_1b_int8_qhead_pos0": ("tinyllama_1b", "int8", 0),
     "llama3_8b_int8_qhead_pos0": ("llama3_8b", "int8", 0),
@@ -52,7 +57,8 @@ DEFAULT_WORKLOAD = "llama3_8b_bf16_pos0"      # the largest single-GPU configura
 OTHER = ["llama3_8b_int8_pos0", "tinyllama_1b_bf16_pos0", "tinyllama_1b_int8_pos0", "tinyllama_1b_int4_pos0",
          "smollm2_135m_bf16_pos0", "tinyllama_1b_bf16_pos1024", "tinyllama_1b_int8_pos512", "llama3_8b_int8_pos4096",
          "llama3_8b_bf16_pos4096", "llama32_1b_bf16_pos0", "llama32_1b_int8_pos0", "tinyllama_1b_int8_qhead_pos0",
-         "llama3_8b_int8_qhead_pos0"]
+         "llama3_8b_int8_qhead_pos0", "paper_small_bf16_pos0", "paper_small_int8_pos0", "paper_small_int4_pos0",
+         "llama3_8b_int4_pos0"]
 # device-resident multi-token runs (amk_decode_greedy: the token is fed back on the device): (shape, dtype, steps)
 SUSTAINED = [("smollm2_135m", "bf16", 256), ("tinyllama_1b", "bf16", 256)]
 METRIC = "batch-1 decode us/token; achieved HBM GB/s vs B200 measured peak"

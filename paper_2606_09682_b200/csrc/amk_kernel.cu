@@ -439,8 +439,6 @@ __device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* s
 // One pass on the tensor cores: this warp walks every ring tile of the pass, multiplies its row group
 // (<= 16 rows, one m16 tile) by the input columns over its column blocks, and publishes per-row sums.
 // ------------------------------------------------------------------------------------------------
-#define AMK_LO(x, z) ((((x) & 0x0F0F0F0Fu) + (z)) ^ 0x80808080u)
-#define AMK_HI(x, z) (((((x) >> 4) & 0x0F0F0F0Fu) + (z)) ^ 0x80808080u)
 
 template <int WD>
 __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int kind, int gw, int K, float* red,
@@ -479,20 +477,35 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int kind
       mma_s8(iacc, fa[0][0], fa[0][1], fa[0][2], fa[0][3], fx0.x, fx0.y);
       mma_s8(iacc2, fa[1][0], fa[1][1], fa[1][2], fa[1][3], fx0.z, fx0.w);
     } else {
+      // sum over k of s (q_k - z) x_k = s (sum q_k x_k - z sum x_k): the codes go to the tensor cores as they are
+      // (unsigned bytes 0..15: one AND per four codes, a shift more for the high nibbles), and the zero point meets
+      // the sum of the input's digits over the group, which every lane takes from its own B fragments (its quad
+      // position's 32 columns of its digit column, then the quad) and hands to the lanes whose accumulator
+      // columns those are.
       const float s0 = __half2float(__ushort_as_half((unsigned short)(fsz0 & 0xffffu)));
       const float s1 = __half2float(__ushort_as_half((unsigned short)(fsz1 & 0xffffu)));
-      // code - zero as a signed byte: (code + 128 - zero) ^ 0x80; no carries between bytes
-      const unsigned z0 = (unsigned)(128 - (int)__half2float(__ushort_as_half((unsigned short)(fsz0 >> 16)))) * 0x01010101u;
-      const unsigned z1 = (unsigned)(128 - (int)__half2float(__ushort_as_half((unsigned short)(fsz1 >> 16)))) * 0x01010101u;
-      int g4[4] = {0, 0, 0, 0}, h4[4] = {0, 0, 0, 0};
-      mma_s8(g4, AMK_LO(fa[0][0], z0), AMK_LO(fa[0][1], z1), AMK_LO(fa[0][2], z0), AMK_LO(fa[0][3], z1), fx0.x, fx0.y);
-      mma_s8(h4, AMK_HI(fa[0][0], z0), AMK_HI(fa[0][1], z1), AMK_HI(fa[0][2], z0), AMK_HI(fa[0][3], z1), fx0.z, fx0.w);
-      mma_s8(g4, AMK_LO(fa[1][0], z0), AMK_LO(fa[1][1], z1), AMK_LO(fa[1][2], z0), AMK_LO(fa[1][3], z1), fx1.x, fx1.y);
-      mma_s8(h4, AMK_HI(fa[1][0], z0), AMK_HI(fa[1][1], z1), AMK_HI(fa[1][2], z0), AMK_HI(fa[1][3], z1), fx1.z, fx1.w);
-      facc[0] = fmaf(s0, (float)(g4[0] + h4[0]), facc[0]);
-      facc[1] = fmaf(s0, (float)(g4[1] + h4[1]), facc[1]);
-      facc[2] = fmaf(s1, (float)(g4[2] + h4[2]), facc[2]);
-      facc[3] = fmaf(s1, (float)(g4[3] + h4[3]), facc[3]);
+      const int z0 = (int)(fsz0 >> 16), z1 = (int)(fsz1 >> 16);      // (the packer stores the zero point as an integer)
+      constexpr unsigned M = 0x0F0F0F0Fu;
+      int g4[4] = {0, 0, 0, 0};
+      mma_u8s8(g4, fa[0][0] & M, fa[0][1] & M, fa[0][2] & M, fa[0][3] & M, fx0.x, fx0.y);
+      mma_u8s8(g4, (fa[0][0] >> 4) & M, (fa[0][1] >> 4) & M, (fa[0][2] >> 4) & M, (fa[0][3] >> 4) & M, fx0.z, fx0.w);
+      mma_u8s8(g4, fa[1][0] & M, fa[1][1] & M, fa[1][2] & M, fa[1][3] & M, fx1.x, fx1.y);
+      mma_u8s8(g4, (fa[1][0] >> 4) & M, (fa[1][1] >> 4) & M, (fa[1][2] >> 4) & M, (fa[1][3] >> 4) & M, fx1.z, fx1.w);
+      int sx = __dp4a((int)fx0.x, 0x01010101, 0);
+      sx = __dp4a((int)fx0.y, 0x01010101, sx);
+      sx = __dp4a((int)fx0.z, 0x01010101, sx);
+      sx = __dp4a((int)fx0.w, 0x01010101, sx);
+      sx = __dp4a((int)fx1.x, 0x01010101, sx);
+      sx = __dp4a((int)fx1.y, 0x01010101, sx);
+      sx = __dp4a((int)fx1.z, 0x01010101, sx);
+      sx = __dp4a((int)fx1.w, 0x01010101, sx);
+      sx += __shfl_xor_sync(0xffffffffu, sx, 1);
+      sx += __shfl_xor_sync(0xffffffffu, sx, 2);
+      const int sx0 = __shfl_sync(0xffffffffu, sx, 8 * q), sx1 = __shfl_sync(0xffffffffu, sx, 8 * q + 4);
+      facc[0] = fmaf(s0, (float)(g4[0] - z0 * sx0), facc[0]);
+      facc[1] = fmaf(s0, (float)(g4[1] - z0 * sx1), facc[1]);
+      facc[2] = fmaf(s1, (float)(g4[2] - z1 * sx0), facc[2]);
+      facc[3] = fmaf(s1, (float)(g4[3] - z1 * sx1), facc[3]);
     }
   };
   int next_b = wk;                                   // my next column block
@@ -574,8 +587,6 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int kind
     if (gq + 8 < urows) dst[gq + 8] = y1;
   }
 }
-#undef AMK_LO
-#undef AMK_HI
 
 // ------------------------------------------------------------------------------------------------
 // One matrix-vector product with its fused prologue (gather / RMSNorm) and epilogue.

@@ -119,14 +119,18 @@ __global__ void pack_kernel(const PackOp d, const PackSrc s, unsigned char* pack
       }
       if (!inverse) *chunk = make_uint4(v[0], v[1], v[2], v[3]);
       if (c == 0) {
-        // fp16 {scale, zero} of this row's group (= this block) after the unit's code bytes
+        // {fp16 scale, zero point as a 16-bit integer} of this row's group (= this block) after the unit's code
+        // bytes (the canonical zero point is an fp16 holding an integer 0..15: the kernel wants the integer)
         unsigned* sz = reinterpret_cast<unsigned*>(unit + (size_t)urows * 64 + (size_t)gi * 4);
         if (!inverse) {
-          if (src.scale && src.zero) *sz = (unsigned)src.scale[b] | ((unsigned)src.zero[b] << 16);
+          if (src.scale && src.zero) {
+            const unsigned zi = (unsigned)(int)__half2float(__ushort_as_half(src.zero[b])) & 0xffffu;
+            *sz = (unsigned)src.scale[b] | (zi << 16);
+          }
         } else {
           const unsigned t = *sz;
           if (src.scale) src.scale[b] = (unsigned short)(t & 0xffffu);
-          if (src.zero) src.zero[b] = (unsigned short)(t >> 16);
+          if (src.zero) src.zero[b] = __half_as_ushort(__float2half_rn((float)(t >> 16)));
         }
       }
     }

@@ -110,6 +110,15 @@ __device__ __forceinline__ void mma_s8(int (&c)[4], unsigned a0, unsigned a1, un
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// D (16x8, int32) += A (16x32 unsigned bytes, row) * B (32x8 int8, col)
+__device__ __forceinline__ void mma_u8s8(int (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, unsigned b0,
+                                         unsigned b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
 // ---- activation elements {value, sequence number}: 8-byte single-copy-atomic accesses at GPU scope -----
 // They carry an L2 evict_last policy: the few hundred KB of activations are touched once per layer while
 // hundreds of MB of weights stream through L2 in between; an 8-byte store to a line that has been evicted

@@ -67,6 +67,10 @@ SHAPES: Dict[str, ModelShape] = {
     # with an untied LM head
     "llama32_1b": ModelShape("llama32_1b", 2048, 16, 32, 8, 64, 8192, 128256, 2048, False,
                              rope_theta=500000.0),
+    # the paper's 4-layer hidden-2048 "small" model (Section 5, Tables 7-8: 622.9 MB of bf16 weights).  The paper gives
+    # its layer count, hidden size and weight bytes only; taken here as four layers of the b1 dimensions with a tied
+    # embedding of 33280 rows, the vocabulary at which the bf16 bytes come to the paper's 622.9 MB (an assumption)
+    "paper_small": ModelShape("paper_small", 2048, 4, 32, 8, 64, 8192, 33280, 2048, True, rope_theta=500000.0),
 }
 
 

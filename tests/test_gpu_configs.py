@@ -123,6 +123,18 @@ def test_tinyllama_shape_quantised_lm_head(amk, wdtype, pos):
     dec.close()
 
 
+@pytest.mark.parametrize("wdtype,pos", [("bf16", 0), ("int8", 77), ("int4", 0)])
+def test_paper_small_shape(amk, wdtype, pos):
+    """The paper's 4-layer hidden-2048 "small" model (vocabulary assumed: see the shape record): the whole step."""
+    shape, w, _, dec = _build(amk, "paper_small", wdtype, 0xA3C6)
+    model, _ = gc.oracle_model(shape, w, wdtype)
+    kv_g = inp.make_kv_prefill(shape, 0xA3C6, pos, device="cuda")
+    kv_c = inp.bits(kv_g).copy()
+    r = gc.compare_step(shape, dec, model, inp.make_token(shape, 0xA3C6), pos, kv_g, kv_c)
+    print("paper_small", wdtype, pos, r)
+    dec.close()
+
+
 @pytest.mark.parametrize("wdtype,pos", [("bf16", 0), ("int8", 0), ("int4", 300)])
 def test_llama32_1b_shape(amk, wdtype, pos):
     """The paper's 16-layer "b1" shape (Llama-3.2-1B dimensions, untied head): the whole step against the oracle."""

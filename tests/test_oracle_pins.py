@@ -395,6 +395,8 @@ def test_parameter_counts_and_byte_ratios_match_paper():
     assert abs(smol.n_params() * 4 / 1e6 - v) <= tol
     v, tol = g["llama32_1b_bf16_MB"]
     assert abs(SHAPES["llama32_1b"].n_params() * 2 / 1e6 - v) <= tol
+    v, tol = g["paper_small_bf16_MB"]
+    assert abs(SHAPES["paper_small"].n_params() * 2 / 1e6 - v) <= tol
 
     def wbytes(dt):
         b = streamed_bytes(smol, dt, 0)
