@@ -184,7 +184,8 @@ __device__ __forceinline__ float read_act(const KParams& p, bool& bad, const Act
   return __uint_as_float(v.x);
 }
 
-__device__ __forceinline__ float silu_f(float z) { return z / (1.0f + expf(-z)); }
+// (on the gate/up -> down critical path: the hardware's exp2 and reciprocal, ~1e-6 relative)
+__device__ __forceinline__ float silu_f(float z) { return __fdividef(z, 1.0f + __expf(-z)); }
 
 // ------------------------------------------------------------------------------------------------
 // Prologue of a matrix-vector product: bring the input vector (K elements written by `src_task`, or the
@@ -333,7 +334,7 @@ __device__ __forceinline__ LoadResult load_input_bf16(const KParams& p, SmemHead
     float tot = 0.f;
 #pragma unroll
     for (int w = 0; w < kConsumerWarps; w++) tot += sh->warp_part[0][w];
-    res.rnorm = 1.0f / sqrtf(tot / (float)K + p.eps);
+    res.rnorm = rsqrtf(__fdividef(tot, (float)K) + p.eps);       // (2 ulp: the same factor on every output)
   }
   return res;
 }
@@ -416,10 +417,10 @@ __device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* s
     float tot = 0.f, mx = 0.f;
 #pragma unroll
     for (int w = 0; w < kConsumerWarps; w++) { tot += sh->warp_part[0][w]; mx = fmaxf(mx, sh->warp_part[1][w]); }
-    if (normw) r = 1.0f / sqrtf(tot / (float)K + p.eps);
+    if (normw) r = rsqrtf(__fdividef(tot, (float)K) + p.eps);   // (2 ulp: the same factor on every element)
     mx *= r;
-    inv = mx > 0.f ? kDigitScale / mx : 0.f;
-    res.xscale = mx / kDigitScale;
+    inv = mx > 0.f ? __fdividef(kDigitScale, mx) : 0.f;
+    res.xscale = mx * (1.0f / kDigitScale);
   }
   const float rinv = r * inv;
 #pragma unroll 1
