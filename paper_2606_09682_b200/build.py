@@ -9,8 +9,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libamk.so")
-SOURCES = ["amk_host.cu", "amk_kernel.cu", "amk_pack.cu", "amk_static.cu"]
-HEADERS = ["amk_layout.h", "amk_internal.h", "amk_ptx.cuh", os.path.join(ROOT, "include", "amk.h")]
+SOURCES = ["amk_host.cu", "amk_kernel.cu", "amk_kernel_trace.cu", "amk_pack.cu", "amk_static.cu"]
+HEADERS = ["amk_layout.h", "amk_internal.h", "amk_ptx.cuh", "amk_kernel_impl.cuh", os.path.join(ROOT, "include", "amk.h")]
 
 
 def _stale() -> bool:
@@ -25,7 +25,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
+    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17", "--threads", "4",
            "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
            "-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES]
     if verbose:

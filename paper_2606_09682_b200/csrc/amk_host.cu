@@ -431,8 +431,11 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     // attention scratch: q vectors, per-warp partial outputs, the new K / V rows, the scores of the longest chunk
     int lc_max = 0, c_max = 0;
     attn_chunks((int)cfg->max_seq, (int)n_blocks, (int)cfg->n_kv_heads, &lc_max, &c_max);
-    const size_t attn_need = ((size_t)n_rep * hd + (size_t)kConsumerWarps * 4 * (hd + 2)) * 4 + (size_t)hd * 4 +
-                             (size_t)n_rep * lc_max * 4;
+    // (AttnScratch in the kernel: q fp32, q as tensor-core fragments, per-warp partial outputs for the heads padded to
+    //  sets of four, the new rows, the scores)
+    const size_t n_sets = ((size_t)n_rep + 3) / 4;
+    const size_t attn_need = (size_t)n_rep * hd * 4 + n_sets * (hd / 16) * 256 +
+                             (size_t)kConsumerWarps * 4 * n_sets * (hd + 2) * 4 + (size_t)hd * 4 + (size_t)n_rep * lc_max * 4;
     if (attn_need > act) act = attn_need;
     act = (act + 127) & ~(size_t)127;
     const uint32_t stage_bytes = h->pl.stage_bytes;
@@ -452,7 +455,8 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     if (max_inflight > n_stages) max_inflight = n_stages;
     const size_t smem_bytes = hdr + act + (size_t)n_stages * stage_bytes;
     int per_sm = 0;
-    AMK_CUDA(decode_kernel_attrs((int)cfg->wdtype, hd, smem_bytes, &per_sm));
+    if (cfg->flags & AMK_FLAG_TRACE) AMK_CUDA(decode_kernel_attrs_traced((int)cfg->wdtype, hd, smem_bytes, &per_sm));
+    else AMK_CUDA(decode_kernel_attrs((int)cfg->wdtype, hd, smem_bytes, &per_sm));
     if (per_sm < 1) {
       snprintf(h->errmsg, sizeof(h->errmsg), "decode kernel does not fit one block per SM");
       status = AMK_ERR_UNSUPPORTED;
@@ -629,7 +633,8 @@ static amk_status launch_step(amk_handle* h, int32_t token, const int* token_ptr
   p.drop_block = h->drop_block;
   h->drop_phase = h->drop_block = -1;
   h->last_stream = stream;
-  cudaError_t e = launch_decode(p, (int)h->plan.n_blocks, h->plan.smem_bytes, stream);
+  cudaError_t e = (h->cfg.flags & AMK_FLAG_TRACE) ? launch_decode_traced(p, (int)h->plan.n_blocks, h->plan.smem_bytes, stream)
+                                                  : launch_decode(p, (int)h->plan.n_blocks, h->plan.smem_bytes, stream);
   if (e != cudaSuccess) {
     --h->epoch;
     --h->ctr_epoch;

@@ -112,8 +112,11 @@ struct KParams {
 };
 
 // Launchers implemented in the .cu files.
+// (two builds of the decode kernel: without and with the trace stamps compiled in)
 cudaError_t launch_decode(const KParams& p, int n_blocks, size_t smem_bytes, cudaStream_t stream);
 cudaError_t decode_kernel_attrs(int wdtype, int hd, size_t smem_bytes, int* max_blocks_per_sm);
+cudaError_t launch_decode_traced(const KParams& p, int n_blocks, size_t smem_bytes, cudaStream_t stream);
+cudaError_t decode_kernel_attrs_traced(int wdtype, int hd, size_t smem_bytes, int* max_blocks_per_sm);
 
 // One op to pack: its shape, rotation and region, plus where the canonical rows come from.
 struct PackOp {
