@@ -44,8 +44,8 @@ namespace {
 
 constexpr int kBarCons = 1;                          // named barrier of the consumer warps
 constexpr int kOutWarps = (kPassRows + 31) / 32;     // warps that hold a pass's output rows
-constexpr int kBatch = 8;                            // 16-byte activation lines a thread gathers at a time
-                                                     // (a normed input must fit one batch per thread)
+constexpr int kBatch = 4;                            // 32-byte items (four activation elements) a thread gathers at a
+                                                     // time (a normed input must fit one batch per thread)
 constexpr float kDigitScale = 4194303.0f;            // int8 / int4 activations: 3 signed base-256 digits, |X| < 2^22
 
 struct Ctx {
@@ -223,53 +223,78 @@ __device__ __forceinline__ float silu_f(float z) { return __fdividef(z, 1.0f + _
 //   int8 / int4 : a / scale as three signed base-256 digits D2, D1, D0 (three B columns), exact integers.
 // ------------------------------------------------------------------------------------------------
 
-// two input elements -> their shared-memory form (line `ln` = elements 2 ln, 2 ln + 1)
-// (this runs between the arrival of the input and the first multiply, so every instruction counts: the
-// hardware's paired fp32 -> bf16 conversion, and byte permutes for the digits)
+// Four input elements (item `it` = elements 4 it .. 4 it + 3) -> their shared-memory form.
+// (This runs between the arrival of the input and the first multiply, so every instruction counts: the
+// hardware's paired fp32 -> bf16 conversion, byte permutes for the digits, 8-byte stores.)
 __device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi) {      // {bf16(lo), bf16(hi)}, round to nearest even
   unsigned r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
 }
 template <int WD>
-__device__ __forceinline__ void store_line(unsigned char* xs, int n2, int ln, float a, float b, float inv) {
+__device__ __forceinline__ void store_item(unsigned char* xs, int n4, int it, const float (&a)[4], float inv) {
   if (WD == W_BF16) {
-    unsigned* X0 = reinterpret_cast<unsigned*>(xs);
-    unsigned* X1 = X0 + n2;
-    const unsigned h = pack_bf16x2(a, b);
-    const float ra = a - bf16_lo(h), rb = b - bf16_hi(h);            // exact
-    const unsigned l = pack_bf16x2(ra, rb);
-    X0[ln] = h;
-    X1[ln] = l;
+    uint2* X0 = reinterpret_cast<uint2*>(xs);                        // columns of K bf16 = n4 items of 8 bytes
+    const unsigned h0 = pack_bf16x2(a[0], a[1]), h1 = pack_bf16x2(a[2], a[3]);
+    const float r0 = a[0] - bf16_lo(h0), r1 = a[1] - bf16_hi(h0), r2 = a[2] - bf16_lo(h1), r3 = a[3] - bf16_hi(h1);   // exact
+    const unsigned l0 = pack_bf16x2(r0, r1), l1 = pack_bf16x2(r2, r3);
+    X0[it] = make_uint2(h0, h1);
+    X0[n4 + it] = make_uint2(l0, l1);
     if (inv > 0.f)                                                   // third column: what the first two still miss
-      (X1 + n2)[ln] = pack_bf16x2(ra - bf16_lo(l), rb - bf16_hi(l));
+      X0[2 * n4 + it] = make_uint2(pack_bf16x2(r0 - bf16_lo(l0), r1 - bf16_hi(l0)),
+                                   pack_bf16x2(r2 - bf16_lo(l1), r3 - bf16_hi(l1)));
   } else {
     // X = d2 * 65536 + d1 * 256 + d0 with every digit in [-128, 127]: the low byte of X is d0's byte, and
     // (X + 128) >> 8 carries on with the rest
-    unsigned short* D2 = reinterpret_cast<unsigned short*>(xs);
-    unsigned short* D1 = D2 + n2;
-    unsigned short* D0 = D1 + n2;
-    const int xa = __float2int_rn(a * inv), xb = __float2int_rn(b * inv);
-    const int ya = (xa + 128) >> 8, yb = (xb + 128) >> 8;
-    const int za = (ya + 128) >> 8, zb = (yb + 128) >> 8;
-    D0[ln] = (unsigned short)__byte_perm((unsigned)xa, (unsigned)xb, 0x0040);
-    D1[ln] = (unsigned short)__byte_perm((unsigned)ya, (unsigned)yb, 0x0040);
-    D2[ln] = (unsigned short)__byte_perm((unsigned)za, (unsigned)zb, 0x0040);
+    unsigned* D2 = reinterpret_cast<unsigned*>(xs);                  // columns of K bytes = n4 items of 4 bytes
+    int x[4], y[4], z[4];
+#pragma unroll
+    for (int e = 0; e < 4; e++) {
+      x[e] = __float2int_rn(a[e] * inv);
+      y[e] = (x[e] + 128) >> 8;
+      z[e] = (y[e] + 128) >> 8;
+    }
+    D2[2 * n4 + it] = __byte_perm(__byte_perm((unsigned)x[0], (unsigned)x[1], 0x0040), __byte_perm((unsigned)x[2], (unsigned)x[3], 0x0040), 0x5410);
+    D2[n4 + it] = __byte_perm(__byte_perm((unsigned)y[0], (unsigned)y[1], 0x0040), __byte_perm((unsigned)y[2], (unsigned)y[3], 0x0040), 0x5410);
+    D2[it] = __byte_perm(__byte_perm((unsigned)z[0], (unsigned)z[1], 0x0040), __byte_perm((unsigned)z[2], (unsigned)z[3], 0x0040), 0x5410);
   }
 }
 
-// Gather one batch of lines (line0, line0 + T, ...): request them all, and if any has not arrived yet request
+// An item of four consecutive activation elements, {value, sequence number} each, fetched with one 32-byte
+// request (four 64-bit accesses, each single-copy atomic like the store that wrote it).
+struct Item {
+  unsigned long long e[4];
+  __device__ __forceinline__ float val(int j) const { return __uint_as_float((unsigned)e[j]); }
+  __device__ __forceinline__ bool carries(unsigned seq) const {
+    return (unsigned)(e[0] >> 32) == seq && (unsigned)(e[1] >> 32) == seq && (unsigned)(e[2] >> 32) == seq &&
+           (unsigned)(e[3] >> 32) == seq;
+  }
+};
+__device__ __forceinline__ Item ld_item(const ActPair* p4) {
+  Item t;
+  asm volatile("ld.relaxed.gpu.global.L2::cache_hint.v4.u64 {%0,%1,%2,%3}, [%4], %5;"
+               : "=l"(t.e[0]), "=l"(t.e[1]), "=l"(t.e[2]), "=l"(t.e[3])
+               : "l"(p4), "l"(policy_evict_last())
+               : "memory");
+  return t;
+}
+
+// Gather one batch of items (item0, item0 + T, ...): request them all, and if any has not arrived yet request
 // the whole batch again until all carry `seq` (bounded).  Returns true on failure.
-__device__ __forceinline__ bool gather_batch(const KParams& p, uint4 (&raw)[kBatch], int line0, int n2,
+__device__ __forceinline__ bool gather_batch(const KParams& p, Item (&raw)[kBatch], int item0, int n4,
                                              const ActPair* src, unsigned seq, int src_task,
                                              const unsigned short* embed_row, int cta, int task) {
   if (embed_row) {
 #pragma unroll
     for (int i = 0; i < kBatch; i++) {
-      const int ln = line0 + i * kConsumerThreads;
-      if (ln < n2) {
-        const unsigned w = __ldg(reinterpret_cast<const unsigned*>(embed_row) + ln);
-        raw[i] = make_uint4(w << 16, seq, w & 0xffff0000u, seq);
+      const int it = item0 + i * kConsumerThreads;
+      if (it < n4) {
+        const uint2 w = __ldg(reinterpret_cast<const uint2*>(embed_row) + it);
+        const unsigned long long sq = (unsigned long long)seq << 32;
+        raw[i].e[0] = sq | (w.x << 16);
+        raw[i].e[1] = sq | (w.x & 0xffff0000u);
+        raw[i].e[2] = sq | (w.y << 16);
+        raw[i].e[3] = sq | (w.y & 0xffff0000u);
       }
     }
     return false;
@@ -279,17 +304,17 @@ __device__ __forceinline__ bool gather_batch(const KParams& p, uint4 (&raw)[kBat
     bool all = true;
 #pragma unroll
     for (int i = 0; i < kBatch; i++) {
-      const int ln = line0 + i * kConsumerThreads;
-      if (ln < n2) raw[i] = ld_pair2(src + 2 * ln);
+      const int it = item0 + i * kConsumerThreads;
+      if (it < n4) raw[i] = ld_item(src + 4 * it);
     }
 #pragma unroll
     for (int i = 0; i < kBatch; i++) {
-      const int ln = line0 + i * kConsumerThreads;
-      if (ln < n2) all = all && (raw[i].y == seq) && (raw[i].w == seq);
+      const int it = item0 + i * kConsumerThreads;
+      if (it < n4) all = all && raw[i].carries(seq);
     }
     if (all) {
 #if AMK_TRACE_BUILD
-      if (p.trace && line0 == 0)     // (not a time) how many requests thread 0 needed for its first batch
+      if (p.trace && item0 == 0)     // (not a time) how many requests thread 0 needed for its first batch
         p.trace[((size_t)cta * (5 * p.L + 1) + task) * AMK_TRACE_EVENTS + AMK_TR_POLLS] = spins + 1u;
 #endif
       return false;
@@ -311,8 +336,8 @@ struct LoadResult {
   bool bad;
 };
 
-// bf16 weights: every line is converted as soon as it has arrived.  RMSNorm's 1/rms is one scalar for the whole
-// vector, so W (r * x * g) = r * (W (x * g)): the lines go to shared memory as x * g while the sum of squares is
+// bf16 weights: every item is converted as soon as it has arrived.  RMSNorm's 1/rms is one scalar for the whole
+// vector, so W (r * x * g) = r * (W (x * g)): the items go to shared memory as x * g while the sum of squares is
 // still being collected, and r is applied to the outputs in the epilogue -- no second pass over the input and no
 // block-wide reduction between the arrival of the input and the first multiply.
 __device__ __forceinline__ LoadResult load_input_bf16(const KParams& p, SmemHeader* sh, unsigned char* xs, int cta, int K,
@@ -320,38 +345,42 @@ __device__ __forceinline__ LoadResult load_input_bf16(const KParams& p, SmemHead
                                                       const unsigned short* embed_row, const unsigned short* normw,
                                                       int task) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int n2 = K >> 1;                               // lines of two elements
+  const int n4 = K >> 2;                               // items of four elements
   LoadResult res{1.0f, 1.0f, false};
-  uint4 raw[kBatch];
+  Item raw[kBatch];
   const float inv3 = (6 * K <= p.act_bytes) ? 1.f : 0.f;     // room for a third bf16 column of the input?
-  // norm weights of my lines: requested before the gather, so that their latency (they come from HBM, being
+  // norm weights of my items: requested before the gather, so that their latency (they come from HBM, being
   // read once per token) is not added to the join's (a normed input is one batch per thread)
-  unsigned gwt[kBatch];
+  uint2 gwt[kBatch];
   if (normw) {
 #pragma unroll
     for (int i = 0; i < kBatch; i++) {
-      const int ln = tid + i * kConsumerThreads;
-      gwt[i] = (ln < n2) ? __ldg(reinterpret_cast<const unsigned*>(normw) + ln) : 0u;
+      const int it = tid + i * kConsumerThreads;
+      gwt[i] = (it < n4) ? __ldg(reinterpret_cast<const uint2*>(normw) + it) : make_uint2(0u, 0u);
     }
   }
   float ss = 0.f;
 #pragma unroll 1
-  for (int l0 = tid; l0 < n2; l0 += kBatch * kConsumerThreads) {
-    res.bad |= gather_batch(p, raw, l0, n2, src, seq, src_task, embed_row, cta, task);
+  for (int i0 = tid; i0 < n4; i0 += kBatch * kConsumerThreads) {
+    res.bad |= gather_batch(p, raw, i0, n4, src, seq, src_task, embed_row, cta, task);
 #pragma unroll
     for (int i = 0; i < kBatch; i++) {
-      const int ln = l0 + i * kConsumerThreads;
-      if (ln < n2) {
-        float a = __uint_as_float(raw[i].x), b = __uint_as_float(raw[i].z);
+      const int it = i0 + i * kConsumerThreads;
+      if (it < n4) {
+        float a[4] = {raw[i].val(0), raw[i].val(1), raw[i].val(2), raw[i].val(3)};
         if (normw) {
-          ss = fmaf(a, a, ss);
-          ss = fmaf(b, b, ss);
+          ss = fmaf(a[0], a[0], ss);
+          ss = fmaf(a[1], a[1], ss);
+          ss = fmaf(a[2], a[2], ss);
+          ss = fmaf(a[3], a[3], ss);
           if (embed_row && cta == 0 && (p.flags & AMK_FLAG_DEBUG_HIDDEN))
-            reinterpret_cast<float2*>(p.hidden)[ln] = make_float2(a, b);
-          a *= bf16_lo(gwt[i]);
-          b *= bf16_hi(gwt[i]);
+            reinterpret_cast<float4*>(p.hidden)[it] = make_float4(a[0], a[1], a[2], a[3]);
+          a[0] *= bf16_lo(gwt[i].x);
+          a[1] *= bf16_hi(gwt[i].x);
+          a[2] *= bf16_lo(gwt[i].y);
+          a[3] *= bf16_hi(gwt[i].y);
         }
-        store_line<W_BF16>(xs, n2, ln, a, b, inv3);
+        store_item<W_BF16>(xs, n4, it, a, inv3);
       }
     }
   }
@@ -379,10 +408,10 @@ __device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* s
                                                  const unsigned short* embed_row, const unsigned short* normw,
                                                  int task, const ActPair* amax_src, int nblk) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int n2 = K >> 1;                               // lines of two elements
+  const int n4 = K >> 2;                               // items of four elements
   LoadResult res{1.0f, 1.0f, false};
-  uint4 raw[kBatch];
-  const bool held = n2 <= kBatch * kConsumerThreads;
+  Item raw[kBatch];
+  const bool held = n4 <= kBatch * kConsumerThreads;
   float r = 1.0f, inv = 0.f;
   // `amax_src`: the producers of this (un-normed) input also published the maximum of their part, so the vector
   // need not be read twice: the first batch is requested, the maxima are combined meanwhile.
@@ -391,52 +420,49 @@ __device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* s
     float ss = 0.f, amax = 0.f;
     if (amax_src) {
       // the blocks' maxima are requested before the gather (they were published with the values), looked at after
-      uint2 ar[2] = {make_uint2(0u, seq), make_uint2(0u, seq)};
-#pragma unroll
-      for (int j = 0; j < 2; j++)
-        if (tid + j * kConsumerThreads < nblk) ar[j] = ld_pair(amax_src + tid + j * kConsumerThreads);
-      res.bad |= gather_batch(p, raw, tid, n2, src, seq, src_task, embed_row, cta, task);
-#pragma unroll
-      for (int j = 0; j < 2; j++) {
-        const int b = tid + j * kConsumerThreads;
-        if (b < nblk && ar[j].y != seq) {
-          ar[j] = poll_pair_slow(p, amax_src + b, seq, src_task);
-          if (ar[j].y != seq) res.bad = true;
-        }
-        amax = fmaxf(amax, fabsf(__uint_as_float(ar[j].x)));
+      uint2 ar = make_uint2(0u, seq);
+      if (tid < nblk) ar = ld_pair(amax_src + tid);
+      res.bad |= gather_batch(p, raw, tid, n4, src, seq, src_task, embed_row, cta, task);
+      if (tid < nblk && ar.y != seq) {
+        ar = poll_pair_slow(p, amax_src + tid, seq, src_task);
+        if (ar.y != seq) res.bad = true;
       }
-      for (int b = tid + 2 * kConsumerThreads; b < nblk; b += kConsumerThreads)
+      amax = fabsf(__uint_as_float(ar.x));
+      for (int b = tid + kConsumerThreads; b < nblk; b += kConsumerThreads)
         amax = fmaxf(amax, fabsf(read_act(p, res.bad, amax_src + b, seq, src_task)));
     }
-    // norm weights of my lines: requested before the gather (see load_input_bf16)
-    unsigned gwt[kBatch];
+    // norm weights of my items: requested before the gather (see load_input_bf16)
+    uint2 gwt[kBatch];
     if (normw) {
 #pragma unroll
       for (int i = 0; i < kBatch; i++) {
-        const int ln = tid + i * kConsumerThreads;
-        gwt[i] = (ln < n2) ? __ldg(reinterpret_cast<const unsigned*>(normw) + ln) : 0u;
+        const int it = tid + i * kConsumerThreads;
+        gwt[i] = (it < n4) ? __ldg(reinterpret_cast<const uint2*>(normw) + it) : make_uint2(0u, 0u);
       }
     }
 #pragma unroll 1
-    for (int l0 = tid; l0 < n2 && !amax_src; l0 += kBatch * kConsumerThreads) {
-      res.bad |= gather_batch(p, raw, l0, n2, src, seq, src_task, embed_row, cta, task);
+    for (int i0 = tid; i0 < n4 && !amax_src; i0 += kBatch * kConsumerThreads) {
+      res.bad |= gather_batch(p, raw, i0, n4, src, seq, src_task, embed_row, cta, task);
 #pragma unroll
       for (int i = 0; i < kBatch; i++) {
-        const int ln = l0 + i * kConsumerThreads;
-        if (ln < n2) {
-          float a = __uint_as_float(raw[i].x), b = __uint_as_float(raw[i].z);
+        const int it = i0 + i * kConsumerThreads;
+        if (it < n4) {
+          float a[4] = {raw[i].val(0), raw[i].val(1), raw[i].val(2), raw[i].val(3)};
           if (normw) {                                 // (normed inputs are always held)
-            ss = fmaf(a, a, ss);
-            ss = fmaf(b, b, ss);
+            ss = fmaf(a[0], a[0], ss);
+            ss = fmaf(a[1], a[1], ss);
+            ss = fmaf(a[2], a[2], ss);
+            ss = fmaf(a[3], a[3], ss);
             if (embed_row && cta == 0 && (p.flags & AMK_FLAG_DEBUG_HIDDEN))
-              reinterpret_cast<float2*>(p.hidden)[ln] = make_float2(a, b);
-            const unsigned gw = gwt[i];
-            a *= bf16_lo(gw);                          // norm weight now, 1/rms after the sum
-            b *= bf16_hi(gw);
-            raw[i].x = __float_as_uint(a);
-            raw[i].z = __float_as_uint(b);
+              reinterpret_cast<float4*>(p.hidden)[it] = make_float4(a[0], a[1], a[2], a[3]);
+            a[0] *= bf16_lo(gwt[i].x);                 // norm weight now, 1/rms after the sum
+            a[1] *= bf16_hi(gwt[i].x);
+            a[2] *= bf16_lo(gwt[i].y);
+            a[3] *= bf16_hi(gwt[i].y);
+#pragma unroll
+            for (int e = 0; e < 4; e++) raw[i].e[e] = (raw[i].e[e] & 0xffffffff00000000ull) | __float_as_uint(a[e]);
           }
-          amax = fmaxf(amax, fmaxf(fabsf(a), fabsf(b)));
+          amax = fmaxf(amax, fmaxf(fmaxf(fabsf(a[0]), fabsf(a[1])), fmaxf(fabsf(a[2]), fabsf(a[3]))));
         }
       }
     }
@@ -455,12 +481,15 @@ __device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* s
   }
   const float rinv = r * inv;
 #pragma unroll 1
-  for (int l0 = tid; l0 < n2; l0 += kBatch * kConsumerThreads) {
-    if (!(have_first && l0 == tid)) res.bad |= gather_batch(p, raw, l0, n2, src, seq, src_task, embed_row, cta, task);
+  for (int i0 = tid; i0 < n4; i0 += kBatch * kConsumerThreads) {
+    if (!(have_first && i0 == tid)) res.bad |= gather_batch(p, raw, i0, n4, src, seq, src_task, embed_row, cta, task);
 #pragma unroll
     for (int i = 0; i < kBatch; i++) {
-      const int ln = l0 + i * kConsumerThreads;
-      if (ln < n2) store_line<WD>(xs, n2, ln, __uint_as_float(raw[i].x), __uint_as_float(raw[i].z), rinv);
+      const int it = i0 + i * kConsumerThreads;
+      if (it < n4) {
+        const float a[4] = {raw[i].val(0), raw[i].val(1), raw[i].val(2), raw[i].val(3)};
+        store_item<WD>(xs, n4, it, a, rinv);
+      }
     }
   }
   res.bad = cons_sync_or(res.bad);

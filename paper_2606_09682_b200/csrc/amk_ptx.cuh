@@ -147,15 +147,4 @@ __device__ __forceinline__ uint2 ld_pair(const void* p) {
                : "memory");
   return make_uint2((unsigned)w, (unsigned)(w >> 32));
 }
-// two consecutive elements with one 16-byte request: two 64-bit accesses, each single-copy atomic like the
-// 64-bit store that wrote it (a vector access is a set of per-element accesses), split in registers
-__device__ __forceinline__ uint4 ld_pair2(const void* p) {
-  unsigned long long a, b;
-  asm volatile("ld.relaxed.gpu.global.L2::cache_hint.v2.u64 {%0,%1}, [%2], %3;"
-               : "=l"(a), "=l"(b)
-               : "l"(p), "l"(policy_evict_last())
-               : "memory");
-  return make_uint4((unsigned)a, (unsigned)(a >> 32), (unsigned)b, (unsigned)(b >> 32));
-}
-
 }  // namespace amk
