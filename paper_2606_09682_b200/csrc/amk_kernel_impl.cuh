@@ -219,7 +219,7 @@ __device__ __forceinline__ float silu_f(float z) { return __fdividef(z, 1.0f + _
 // ------------------------------------------------------------------------------------------------
 // Prologue of a matrix-vector product: bring the input vector (K elements written by `src_task`, or the
 // embedding row) into shared memory in the form the tensor cores take, with RMSNorm folded in.
-//   bf16 weights: X0[K] = bf16(a), X1[K] = bf16(a - X0): two B columns whose sum is a to ~2^-17.
+//   bf16 weights: X0[K] = bf16(a), X1[K] = bf16(a - X0): two B columns whose sum is a to 2^-17.
 //   int8 / int4 : a / scale as three signed base-256 digits D2, D1, D0 (three B columns), exact integers.
 // ------------------------------------------------------------------------------------------------
 
@@ -234,15 +234,13 @@ __device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi) {      // {b
 template <int WD>
 __device__ __forceinline__ void store_item(unsigned char* xs, int n4, int it, const float (&a)[4], float inv) {
   if (WD == W_BF16) {
+    // two B columns: bf16(a) and bf16(a - bf16(a)); their sum is a to 2^-17 (a third column would make it exact
+    // and measured 1.3 % slower at the TinyLlama shape for an error far below the others')
     uint2* X0 = reinterpret_cast<uint2*>(xs);                        // columns of K bf16 = n4 items of 8 bytes
     const unsigned h0 = pack_bf16x2(a[0], a[1]), h1 = pack_bf16x2(a[2], a[3]);
-    const float r0 = a[0] - bf16_lo(h0), r1 = a[1] - bf16_hi(h0), r2 = a[2] - bf16_lo(h1), r3 = a[3] - bf16_hi(h1);   // exact
-    const unsigned l0 = pack_bf16x2(r0, r1), l1 = pack_bf16x2(r2, r3);
     X0[it] = make_uint2(h0, h1);
-    X0[n4 + it] = make_uint2(l0, l1);
-    if (inv > 0.f)                                                   // third column: what the first two still miss
-      X0[2 * n4 + it] = make_uint2(pack_bf16x2(r0 - bf16_lo(l0), r1 - bf16_hi(l0)),
-                                   pack_bf16x2(r2 - bf16_lo(l1), r3 - bf16_hi(l1)));
+    X0[n4 + it] = make_uint2(pack_bf16x2(a[0] - bf16_lo(h0), a[1] - bf16_hi(h0)),                 // (differences exact)
+                             pack_bf16x2(a[2] - bf16_lo(h1), a[3] - bf16_hi(h1)));
   } else {
     // X = d2 * 65536 + d1 * 256 + d0 with every digit in [-128, 127]: the low byte of X is d0's byte, and
     // (X + 128) >> 8 carries on with the rest
@@ -348,7 +346,6 @@ __device__ __forceinline__ LoadResult load_input_bf16(const KParams& p, SmemHead
   const int n4 = K >> 2;                               // items of four elements
   LoadResult res{1.0f, 1.0f, false};
   Item raw[kBatch];
-  const float inv3 = (6 * K <= p.act_bytes) ? 1.f : 0.f;     // room for a third bf16 column of the input?
   // norm weights of my items: requested before the gather, so that their latency (they come from HBM, being
   // read once per token) is not added to the join's (a normed input is one batch per thread)
   uint2 gwt[kBatch];
@@ -380,7 +377,7 @@ __device__ __forceinline__ LoadResult load_input_bf16(const KParams& p, SmemHead
           a[2] *= bf16_lo(gwt[i].y);
           a[3] *= bf16_hi(gwt[i].y);
         }
-        store_item<W_BF16>(xs, n4, it, a, inv3);
+        store_item<W_BF16>(xs, n4, it, a, 0.f);
       }
     }
   }
@@ -515,9 +512,8 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int kind
   const unsigned step_stride = (unsigned)(2 * urows * 16);                     // two chunks per k step
   const int S = p.n_stages;
   constexpr int BC = (WD == W_INT4) ? 128 : 64;
-  // B columns in use: int8 / int4 three digits; bf16 high + low halves, plus a third term (fp32-exact
-  // input) whenever the input area has room for it
-  const int NCOL = (WD == W_BF16) ? ((6 * K <= p.act_bytes) ? 3 : 2) : 3;
+  // B columns in use: int8 / int4 three digits; bf16 high + low parts
+  constexpr int NCOL = (WD == W_BF16) ? 2 : 3;
   const unsigned char* xcol = c.xs + (size_t)min(gq, NCOL - 1) * K * (WD == W_BF16 ? 2 : 1);
 
   // All fragments of a unit are loaded before its first MMA, and two accumulator sets are used in turn, so
@@ -1346,8 +1342,6 @@ __device__ __noinline__ unsigned attn_general_scalar(const KParams& p, SmemHeade
   float* S = AS.S;                                     // [n_rep][Lc] scores, then softmax numerators
   float* hmax = c.sh->red[0];                          // [n_rep] chunk maximum and sum per head
   float* hsum = c.sh->red[1];
-  const unsigned out_seq = seq_of(p, 5 * l + 1);
-  const bool drop = (5 * l + 1 == p.drop_phase && cta == p.drop_block);
   const int n_hb = (n_rep + 3) >> 2;     // blocks of four q heads
   const int wph = kConsumerWarps / n_hb; // warps per head block
   const int hb = c.warp / wph, wi = c.warp - hb * wph;
@@ -1525,7 +1519,9 @@ __device__ __noinline__ void producer(const KParams& p, SmemHeader* sh, unsigned
   const unsigned begin = __ldg(p.tile_begin + cta), end = __ldg(p.tile_begin + cta + 1);
   unsigned t = 0;                                   // tiles issued so far
   unsigned stage = 0, lap = 0;
+#if AMK_TRACE_BUILD
   int cur_task = -1;
+#endif
   int ok = 1;
   // the warp holds 64 consecutive table entries: [base, base + 32) in e_cur, [base + 32, base + 64) in e_next
   unsigned long long e_cur = (begin + lane < end) ? __ldg(p.tiles + begin + lane) : 0ull;
