@@ -455,8 +455,9 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     if (max_inflight > n_stages) max_inflight = n_stages;
     const size_t smem_bytes = hdr + act + (size_t)n_stages * stage_bytes;
     int per_sm = 0;
-    if (cfg->flags & AMK_FLAG_TRACE) AMK_CUDA(decode_kernel_attrs_traced((int)cfg->wdtype, hd, smem_bytes, &per_sm));
-    else AMK_CUDA(decode_kernel_attrs((int)cfg->wdtype, hd, smem_bytes, &per_sm));
+    // (both builds of the kernel: the diagnostic one serves tracing, counter joins and the dropped-signal hook)
+    AMK_CUDA(decode_kernel_attrs_traced((int)cfg->wdtype, hd, smem_bytes, &per_sm));
+    AMK_CUDA(decode_kernel_attrs((int)cfg->wdtype, hd, smem_bytes, &per_sm));
     if (per_sm < 1) {
       snprintf(h->errmsg, sizeof(h->errmsg), "decode kernel does not fit one block per SM");
       status = AMK_ERR_UNSUPPORTED;
@@ -604,7 +605,7 @@ fail:
 // 2^32 / (5 L + 1) steps: tens of millions), the activation area is cleared on the step's stream -- everything in
 // it then carries sequence number 0, which no task ever waits for -- and the step count starts again.
 static bool epoch_would_wrap(const amk_handle* h) {
-  const unsigned long long per = 5ull * h->cfg.n_layers + 1ull;
+  const unsigned long long per = 5ull * h->cfg.n_layers + 2ull;
   return ((unsigned long long)h->epoch + 2ull) * per + 2ull > 0xffffffffull;
 }
 
@@ -633,8 +634,9 @@ static amk_status launch_step(amk_handle* h, int32_t token, const int* token_ptr
   p.drop_block = h->drop_block;
   h->drop_phase = h->drop_block = -1;
   h->last_stream = stream;
-  cudaError_t e = (h->cfg.flags & AMK_FLAG_TRACE) ? launch_decode_traced(p, (int)h->plan.n_blocks, h->plan.smem_bytes, stream)
-                                                  : launch_decode(p, (int)h->plan.n_blocks, h->plan.smem_bytes, stream);
+  const bool diagnostic = (h->cfg.flags & AMK_FLAG_TRACE) || p.sync_mode == 0 || p.drop_block >= 0;
+  cudaError_t e = diagnostic ? launch_decode_traced(p, (int)h->plan.n_blocks, h->plan.smem_bytes, stream)
+                             : launch_decode(p, (int)h->plan.n_blocks, h->plan.smem_bytes, stream);
   if (e != cudaSuccess) {
     --h->epoch;
     --h->ctr_epoch;

@@ -124,16 +124,31 @@ __device__ __forceinline__ bool wait_mbar(const KParams& p, uint64_t* bar, unsig
 
 // A step at position 0 with data-carried dependencies has no attention task: the QKV projection's epilogue
 // publishes the attention output and appends the cache rows itself (see gemv_op).
-__device__ __forceinline__ bool single_pos(const KParams& p) { return p.pos == 0 && p.sync_mode != 0; }
+// Test hook of the bounded waits (diagnostic build): this block withholds what it would publish for `task`.
+__device__ __forceinline__ bool dropped(const KParams& p, int task, int cta) {
+#if AMK_TRACE_BUILD
+  return task == p.drop_phase && cta == p.drop_block;
+#else
+  return false;
+#endif
+}
 
-// Sequence number carried by everything task `task` publishes in this step (never 0).
+#if AMK_TRACE_BUILD
+__device__ __forceinline__ bool counter_joins(const KParams& p) { return p.sync_mode == 0; }
+#else
+__device__ __forceinline__ bool counter_joins(const KParams&) { return false; }     // (the diagnostic build has them)
+#endif
+__device__ __forceinline__ bool single_pos(const KParams& p) { return p.pos == 0 && !counter_joins(p); }
+
+// Sequence number carried by everything task `task` publishes in this step (never 0).  Task -1 is the embedding
+// row, which every block publishes its share of at kernel start like any other activation.
 __device__ __forceinline__ unsigned seq_of(const KParams& p, int task) {
-  return p.epoch * (unsigned)(5 * p.L + 1) + (unsigned)task + 1u;
+  return p.epoch * (unsigned)(5 * p.L + 2) + (unsigned)(task + 2);
 }
 
 // Counter layer (sync_mode 0): all consumer threads wait until every block has signalled `phase`.
 __device__ __forceinline__ bool wait_phase(Ctx& c, int phase) {
-  if (c.p.sync_mode != 0) return true;
+  if (!counter_joins(c.p)) return true;
   if (c.tid == 0) {
     if (!poll_counter(c.p, c.p.phase_ctr + phase, c.p.ctr_epoch * (unsigned)c.nblk, phase)) c.bad = true;
   }
@@ -142,8 +157,8 @@ __device__ __forceinline__ bool wait_phase(Ctx& c, int phase) {
 }
 // Called after a consumer barrier that follows the task's last store: release-increment the counter.
 __device__ __forceinline__ void signal_phase(Ctx& c, int phase) {
-  if (c.p.sync_mode != 0) return;
-  if (c.tid == 0 && !(phase == c.p.drop_phase && c.cta == c.p.drop_block))
+  if (!counter_joins(c.p)) return;
+  if (c.tid == 0 && !dropped(c.p, phase, c.cta))
     red_release_gpu_add(c.p.phase_ctr + phase, 1u);
 }
 
@@ -280,23 +295,7 @@ __device__ __forceinline__ Item ld_item(const ActPair* p4) {
 // Gather one batch of items (item0, item0 + T, ...): request them all, and if any has not arrived yet request
 // the whole batch again until all carry `seq` (bounded).  Returns true on failure.
 __device__ __forceinline__ bool gather_batch(const KParams& p, Item (&raw)[kBatch], int item0, int n4,
-                                             const ActPair* src, unsigned seq, int src_task,
-                                             const unsigned short* embed_row, int cta, int task) {
-  if (embed_row) {
-#pragma unroll
-    for (int i = 0; i < kBatch; i++) {
-      const int it = item0 + i * kConsumerThreads;
-      if (it < n4) {
-        const uint2 w = __ldg(reinterpret_cast<const uint2*>(embed_row) + it);
-        const unsigned long long sq = (unsigned long long)seq << 32;
-        raw[i].e[0] = sq | (w.x << 16);
-        raw[i].e[1] = sq | (w.x & 0xffff0000u);
-        raw[i].e[2] = sq | (w.y << 16);
-        raw[i].e[3] = sq | (w.y & 0xffff0000u);
-      }
-    }
-    return false;
-  }
+                                             const ActPair* src, unsigned seq, int src_task, int cta, int task) {
   unsigned long long t0 = 0;
   for (unsigned spins = 0;; spins++) {
     bool all = true;
@@ -340,8 +339,7 @@ struct LoadResult {
 // block-wide reduction between the arrival of the input and the first multiply.
 __device__ __forceinline__ LoadResult load_input_bf16(const KParams& p, SmemHeader* sh, unsigned char* xs, int cta, int K,
                                                       const ActPair* src, unsigned seq, int src_task,
-                                                      const unsigned short* embed_row, const unsigned short* normw,
-                                                      int task) {
+                                                      const unsigned short* normw, int task) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n4 = K >> 2;                               // items of four elements
   LoadResult res{1.0f, 1.0f, false};
@@ -359,7 +357,7 @@ __device__ __forceinline__ LoadResult load_input_bf16(const KParams& p, SmemHead
   float ss = 0.f;
 #pragma unroll 1
   for (int i0 = tid; i0 < n4; i0 += kBatch * kConsumerThreads) {
-    res.bad |= gather_batch(p, raw, i0, n4, src, seq, src_task, embed_row, cta, task);
+    res.bad |= gather_batch(p, raw, i0, n4, src, seq, src_task, cta, task);
 #pragma unroll
     for (int i = 0; i < kBatch; i++) {
       const int it = i0 + i * kConsumerThreads;
@@ -370,8 +368,6 @@ __device__ __forceinline__ LoadResult load_input_bf16(const KParams& p, SmemHead
           ss = fmaf(a[1], a[1], ss);
           ss = fmaf(a[2], a[2], ss);
           ss = fmaf(a[3], a[3], ss);
-          if (embed_row && cta == 0 && (p.flags & AMK_FLAG_DEBUG_HIDDEN))
-            reinterpret_cast<float4*>(p.hidden)[it] = make_float4(a[0], a[1], a[2], a[3]);
           a[0] *= bf16_lo(gwt[i].x);
           a[1] *= bf16_hi(gwt[i].x);
           a[2] *= bf16_lo(gwt[i].y);
@@ -402,8 +398,8 @@ __device__ __forceinline__ LoadResult load_input_bf16(const KParams& p, SmemHead
 template <int WD>
 __device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* sh, unsigned char* xs, int cta, int K,
                                                  const ActPair* src, unsigned seq, int src_task,
-                                                 const unsigned short* embed_row, const unsigned short* normw,
-                                                 int task, const ActPair* amax_src, int nblk) {
+                                                 const unsigned short* normw, int task, const ActPair* amax_src,
+                                                 int nblk) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n4 = K >> 2;                               // items of four elements
   LoadResult res{1.0f, 1.0f, false};
@@ -419,7 +415,7 @@ __device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* s
       // the blocks' maxima are requested before the gather (they were published with the values), looked at after
       uint2 ar = make_uint2(0u, seq);
       if (tid < nblk) ar = ld_pair(amax_src + tid);
-      res.bad |= gather_batch(p, raw, tid, n4, src, seq, src_task, embed_row, cta, task);
+      res.bad |= gather_batch(p, raw, tid, n4, src, seq, src_task, cta, task);
       if (tid < nblk && ar.y != seq) {
         ar = poll_pair_slow(p, amax_src + tid, seq, src_task);
         if (ar.y != seq) res.bad = true;
@@ -439,7 +435,7 @@ __device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* s
     }
 #pragma unroll 1
     for (int i0 = tid; i0 < n4 && !amax_src; i0 += kBatch * kConsumerThreads) {
-      res.bad |= gather_batch(p, raw, i0, n4, src, seq, src_task, embed_row, cta, task);
+      res.bad |= gather_batch(p, raw, i0, n4, src, seq, src_task, cta, task);
 #pragma unroll
       for (int i = 0; i < kBatch; i++) {
         const int it = i0 + i * kConsumerThreads;
@@ -450,8 +446,6 @@ __device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* s
             ss = fmaf(a[1], a[1], ss);
             ss = fmaf(a[2], a[2], ss);
             ss = fmaf(a[3], a[3], ss);
-            if (embed_row && cta == 0 && (p.flags & AMK_FLAG_DEBUG_HIDDEN))
-              reinterpret_cast<float4*>(p.hidden)[it] = make_float4(a[0], a[1], a[2], a[3]);
             a[0] *= bf16_lo(gwt[i].x);                 // norm weight now, 1/rms after the sum
             a[1] *= bf16_hi(gwt[i].x);
             a[2] *= bf16_lo(gwt[i].y);
@@ -479,7 +473,7 @@ __device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* s
   const float rinv = r * inv;
 #pragma unroll 1
   for (int i0 = tid; i0 < n4; i0 += kBatch * kConsumerThreads) {
-    if (!(have_first && i0 == tid)) res.bad |= gather_batch(p, raw, i0, n4, src, seq, src_task, embed_row, cta, task);
+    if (!(have_first && i0 == tid)) res.bad |= gather_batch(p, raw, i0, n4, src, seq, src_task, cta, task);
 #pragma unroll
     for (int i = 0; i < kBatch; i++) {
       const int it = i0 + i * kConsumerThreads;
@@ -662,8 +656,6 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind_rt, int l) {
   sl.row0 = c.sh->slice_row0[kind];
   sl.rows = c.sh->slice_rows[kind];
   const int K = d.K;
-  const bool first_layer = (l == 0);
-  const unsigned short* embed_row = p.embed + (size_t)c.token * p.H;
   const unsigned my_seq = seq_of(p, task);
   if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_ENTER);
 
@@ -671,10 +663,9 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind_rt, int l) {
   const ActPair* src = nullptr;
   const unsigned short* normw = nullptr;
   int src_task = -1;
-  bool from_embed = false;
   switch (kind) {
-    case OP_QKV:
-      src = p.x_a; src_task = 5 * (l - 1) + 4; normw = p.attn_norm + (size_t)l * p.H; from_embed = first_layer;
+    case OP_QKV:       // (layer 0: task -1, the embedding row)
+      src = p.x_a; src_task = 5 * (l - 1) + 4; normw = p.attn_norm + (size_t)l * p.H;
       break;
     case OP_O: src = p.o; src_task = 5 * l + 1; break;
     case OP_GATEUP: src = p.x_b; src_task = 5 * l + 2; normw = p.mlp_norm + (size_t)l * p.H; break;
@@ -696,8 +687,8 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind_rt, int l) {
     if (c.tid < ((kind == OP_GATEUP) ? (R >> 1) : R)) {
       const int vrow = vrow0 + c.tid;
       if (kind == OP_O) {
-        if (first_layer) rraw.x = (unsigned)__ldg(embed_row + vrow) << 16;
-        else { raddr = p.x_a + vrow; rtask = 5 * (l - 1) + 4; }
+        raddr = p.x_a + vrow;
+        rtask = 5 * (l - 1) + 4;
       } else if (kind == OP_DOWN) {
         raddr = p.x_b + vrow;
         rtask = 5 * l + 2;
@@ -718,13 +709,12 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind_rt, int l) {
   if (np > 0) request_operands(0);
 
   float rnorm = 1.0f;                                    // bf16 weights, normed input: 1/rms, applied to the outputs
-  if (!from_embed && !wait_phase(c, src_task)) return false;
+  if (src_task >= 0 && !wait_phase(c, src_task)) return false;
   if (np > 0) {
-    const unsigned in_seq = from_embed ? 1u : seq_of(p, src_task);
-    const unsigned short* erow = from_embed ? embed_row : nullptr;
+    const unsigned in_seq = seq_of(p, src_task);
     LoadResult lr;
-    if (WD == W_BF16) lr = load_input_bf16(p, c.sh, c.xs, c.cta, K, src, in_seq, src_task, erow, normw, task);
-    else lr = load_input<WD>(p, c.sh, c.xs, c.cta, K, src, in_seq, src_task, erow, normw, task,
+    if (WD == W_BF16) lr = load_input_bf16(p, c.sh, c.xs, c.cta, K, src, in_seq, src_task, normw, task);
+    else lr = load_input<WD>(p, c.sh, c.xs, c.cta, K, src, in_seq, src_task, normw, task,
                              kind == OP_DOWN ? p.m_amax : nullptr, c.nblk);
     rnorm = lr.rnorm;
     c.xscale = lr.xscale;
@@ -736,7 +726,7 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind_rt, int l) {
   // ---- passes -------------------------------------------------------------------------------------------
   float best_val = -CUDART_INF_F;
   int best_idx = 0x7fffffff;
-  const bool drop = (task == p.drop_phase && c.cta == p.drop_block);
+  const bool drop = dropped(p, task, c.cta);
   float gu_amax = 0.f;                                // gate/up of an integer-weight model: max |output| of this block
   for (int ps = 0; ps < np; ps++) {
     const int R = pass_rows(sl.rows, ps);
@@ -890,7 +880,7 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind_rt, int l) {
     return true;
   }
 
-  if (p.sync_mode == 0) {
+  if (counter_joins(p)) {
     c.bad = cons_sync_or(c.bad);
     if (c.bad) return false;
     signal_phase(c, task);
@@ -973,7 +963,7 @@ __device__ __forceinline__ bool attn_task(const KParams& p, SmemHeader* sh, unsi
   const float qscale = 1.4426950408889634f * rsqrtf((float)HD);
   const size_t kvrow = ((size_t)l * p.nkv + g) * p.S;
   const unsigned in_seq = seq_of(p, 5 * l), out_seq = seq_of(p, 5 * l + 1);
-  const bool drop = (5 * l + 1 == p.drop_phase && c.cta == p.drop_block);
+  const bool drop = dropped(p, 5 * l + 1, c.cta);
 
   // ---- gather q (all heads of the group) and, in the chunk that owns the new position, k and v ----------
   // items: [0, n_rep*half) = q pairs (head h, dims e and e + half); then k pairs; then v pairs.
@@ -1048,7 +1038,7 @@ __device__ __forceinline__ unsigned finish_chunk(const KParams& p, SmemHeader* s
                                                  unsigned ring_pos, F partial) {
   const int tid = threadIdx.x, n_rep = p.n_rep;
   const unsigned out_seq = seq_of(p, 5 * l + 1);
-  const bool drop = (5 * l + 1 == p.drop_phase && cta == p.drop_block);
+  const bool drop = dropped(p, 5 * l + 1, cta);
   for (int i = tid; i < n_rep * HD; i += kConsumerThreads) {
     const int h = i / HD, dd = i - h * HD;
     const float A = partial(h, dd);
@@ -1481,7 +1471,7 @@ __device__ __forceinline__ bool attention_phase(Ctx& c, int l) {
   int t = c.cta + c.nblk - rot;
   if (t >= c.nblk) t -= c.nblk;
   const int task = 5 * l + 1;
-  if (p.sync_mode != 0 && t >= n_tasks) return true;      // nothing to do here and nobody to tell
+  if (!counter_joins(p) && t >= n_tasks) return true;     // nothing to do here and nobody to tell
   if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_ENTER);
   if (!wait_phase(c, 5 * l + 0)) return false;
   if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_JOINED);
@@ -1681,6 +1671,15 @@ __global__ void __launch_bounds__(kThreads, 1) AMK_KERNEL(const __grid_constant_
 
   int token = p.token_ptr ? __ldcg(p.token_ptr) : p.token;
   token = min(max(token, 0), p.V - 1);
+  // Task -1: the embedding row enters the residual stream like every other activation -- every block publishes its
+  // share of the row as {value, sequence number} elements, and layer 0 reads it the way layer l reads layer l - 1.
+  {
+    for (int e = cta * kConsumerThreads + tid; e < p.H; e += nblk * kConsumerThreads) {
+      const float v = __uint_as_float((unsigned)__ldg(p.embed + (size_t)token * p.H + e) << 16);
+      st_pair(p.x_a + e, v, seq_of(p, -1));
+      if (p.flags & AMK_FLAG_DEBUG_HIDDEN) p.hidden[e] = v;
+    }
+  }
   Ctx c{p, sh, xs, ring, tid, warp, lane, cta, nblk, 0, 0u, token, 1.0f, false};
   // the block's queue: tasks 5 l + {0..4} = QKV, attention, O, gate/up, down of layer l, then the LM head
   // (one call site each, so that the per-thread state stays in registers)
