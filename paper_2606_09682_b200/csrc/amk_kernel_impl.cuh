@@ -46,7 +46,12 @@ constexpr int kBarCons = 1;                          // named barrier of the con
 constexpr int kOutWarps = (kPassRows + 31) / 32;     // warps that hold a pass's output rows
 constexpr int kBatch = 4;                            // 32-byte items (four activation elements) a thread gathers at a
                                                      // time (a normed input must fit one batch per thread)
-constexpr float kDigitScale = 4194303.0f;            // int8 / int4 activations: 3 signed base-256 digits, |X| < 2^22
+// int8 / int4 activations: X = round(a / scale) as three signed base-256 digits, |X| <= kDigitScale.  Adding
+// kDigitBias = 2^23 + 0x408080 in the same fused multiply-add rounds to the integer and leaves, in the low three
+// bytes of the float's bit pattern, d0 + 128, d1 + 128 and d2 + 64 (needs -4227200 <= X < 4161408; the margin
+// covers the few ulp of the approximate reciprocal behind the scale).
+constexpr float kDigitScale = 4161000.0f;
+constexpr float kDigitBias = 12615808.0f;
 
 struct Ctx {
   const KParams& p;
@@ -247,7 +252,7 @@ __device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi) {      // {b
   return r;
 }
 template <int WD>
-__device__ __forceinline__ void store_item(unsigned char* xs, int n4, int it, const float (&a)[4], float inv) {
+__device__ __forceinline__ void store_item(unsigned char* xs, int n4, int it, const float (&a)[4], float inv = 0.f) {
   if (WD == W_BF16) {
     // two B columns: bf16(a) and bf16(a - bf16(a)); their sum is a to 2^-17 (a third column would make it exact
     // and measured 1.3 % slower at the TinyLlama shape for an error far below the others')
@@ -257,19 +262,40 @@ __device__ __forceinline__ void store_item(unsigned char* xs, int n4, int it, co
     X0[n4 + it] = make_uint2(pack_bf16x2(a[0] - bf16_lo(h0), a[1] - bf16_hi(h0)),                 // (differences exact)
                              pack_bf16x2(a[2] - bf16_lo(h1), a[3] - bf16_hi(h1)));
   } else {
-    // X = d2 * 65536 + d1 * 256 + d0 with every digit in [-128, 127]: the low byte of X is d0's byte, and
-    // (X + 128) >> 8 carries on with the rest
+    // X = d2 * 65536 + d1 * 256 + d0 with every digit in [-128, 127] (see kDigitBias)
     unsigned* D2 = reinterpret_cast<unsigned*>(xs);                  // columns of K bytes = n4 items of 4 bytes
-    int x[4], y[4], z[4];
-#pragma unroll
-    for (int e = 0; e < 4; e++) {
-      x[e] = __float2int_rn(a[e] * inv);
-      y[e] = (x[e] + 128) >> 8;
-      z[e] = (y[e] + 128) >> 8;
+    float gmax = 0.f;
+    if (WD == W_INT4) {
+      // int4: a scale of its own for every group of 128 elements, which is exactly a warp's 32 items (items are
+      // dealt out warp by warp and K is a multiple of 128): one warp-wide maximum, no pass over the whole vector
+      gmax = warp_max_nonneg(fmaxf(fmaxf(fabsf(a[0]), fabsf(a[1])), fmaxf(fabsf(a[2]), fabsf(a[3]))));
+      inv = gmax > 0.f ? __fdividef(kDigitScale, gmax) : 0.f;
     }
-    D2[2 * n4 + it] = __byte_perm(__byte_perm((unsigned)x[0], (unsigned)x[1], 0x0040), __byte_perm((unsigned)x[2], (unsigned)x[3], 0x0040), 0x5410);
-    D2[n4 + it] = __byte_perm(__byte_perm((unsigned)y[0], (unsigned)y[1], 0x0040), __byte_perm((unsigned)y[2], (unsigned)y[3], 0x0040), 0x5410);
-    D2[it] = __byte_perm(__byte_perm((unsigned)z[0], (unsigned)z[1], 0x0040), __byte_perm((unsigned)z[2], (unsigned)z[3], 0x0040), 0x5410);
+    unsigned t[4];
+#pragma unroll
+    for (int e = 0; e < 4; e++) t[e] = __float_as_uint(fmaf(a[e], inv, kDigitBias));
+    const unsigned p01 = __byte_perm(t[0], t[1], 0x5140), p23 = __byte_perm(t[2], t[3], 0x5140);   // {b0, b0', b1, b1'}
+    const unsigned w0 = __byte_perm(p01, p23, 0x5410) ^ 0x80808080u;
+    const unsigned w1 = __byte_perm(p01, p23, 0x7632) ^ 0x80808080u;
+    const unsigned w2 = (__byte_perm(__byte_perm(t[0], t[1], 0x0062), __byte_perm(t[2], t[3], 0x0062), 0x5410) + 0x40404040u) ^ 0x80808080u;
+    D2[2 * n4 + it] = w0;
+    D2[n4 + it] = w1;
+    D2[it] = w2;
+    if (WD == W_INT4) {
+      // The zero point of a weight group meets the sum of the input's integers X over the group (see consume_pass):
+      // one warp-wide integer sum (below 2^29), split into signed base-256 digits like the elements themselves so
+      // that each meets the accumulator column of its weight.  The group's entry of the table behind the digit
+      // columns, laid out by accumulator column pair: {A2, A1, scale, -} {A0, 0, scale, -}.
+      const int sx = (int)(__reduce_add_sync(0xffffffffu, (t[0] + t[1]) + (t[2] + t[3])) - 128u * 0x4B408080u);
+      const int s0 = (sx << 24) >> 24, r1 = (sx - s0) >> 8;
+      const int s1 = (r1 << 24) >> 24, s2 = (r1 - s1) >> 8;
+      const int lane = threadIdx.x & 31;
+      if (lane < 2) {
+        const int sc = __float_as_int(gmax * (1.0f / kDigitScale));
+        reinterpret_cast<int4*>(xs + 12 * (size_t)n4)[2 * (it >> 5) + lane] =
+            lane == 0 ? make_int4(s2, s1, sc, 0) : make_int4(s0, 0, sc, 0);
+      }
+    }
   }
 }
 
@@ -333,13 +359,15 @@ struct LoadResult {
   bool bad;
 };
 
-// bf16 weights: every item is converted as soon as it has arrived.  RMSNorm's 1/rms is one scalar for the whole
-// vector, so W (r * x * g) = r * (W (x * g)): the items go to shared memory as x * g while the sum of squares is
-// still being collected, and r is applied to the outputs in the epilogue -- no second pass over the input and no
-// block-wide reduction between the arrival of the input and the first multiply.
-__device__ __forceinline__ LoadResult load_input_bf16(const KParams& p, SmemHeader* sh, unsigned char* xs, int cta, int K,
-                                                      const ActPair* src, unsigned seq, int src_task,
-                                                      const unsigned short* normw, int task) {
+// bf16 and int4 weights: every item is converted as soon as it has arrived.  RMSNorm's 1/rms is one scalar for the
+// whole vector, so W (r * x * g) = r * (W (x * g)): the items go to shared memory as x * g while the sum of squares
+// is still being collected, and r is applied to the outputs in the epilogue -- no second pass over the input and no
+// block-wide reduction between the arrival of the input and the first multiply.  (int4: the digits' scale is per
+// group of 128 elements, like the weights' own, and meets them in the same multiply.)
+template <int WD>
+__device__ __forceinline__ LoadResult load_input_1pass(const KParams& p, SmemHeader* sh, unsigned char* xs, int cta, int K,
+                                                       const ActPair* src, unsigned seq, int src_task,
+                                                       const unsigned short* normw, int task) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n4 = K >> 2;                               // items of four elements
   LoadResult res{1.0f, 1.0f, false};
@@ -373,7 +401,7 @@ __device__ __forceinline__ LoadResult load_input_bf16(const KParams& p, SmemHead
           a[2] *= bf16_lo(gwt[i].y);
           a[3] *= bf16_hi(gwt[i].y);
         }
-        store_item<W_BF16>(xs, n4, it, a, 0.f);
+        store_item<WD>(xs, n4, it, a);
       }
     }
   }
@@ -392,8 +420,8 @@ __device__ __forceinline__ LoadResult load_input_bf16(const KParams& p, SmemHead
   return res;
 }
 
-// Integer weights: the input becomes three signed digits of a / scale, and the scale needs the maximum of the
-// whole (normed) vector first.  A vector short enough for one batch per thread (every normed input) is held in
+// int8 weights (one integer accumulation over the whole row): the input becomes three signed digits of a / scale
+// with one scale, which needs the maximum of the whole (normed) vector first.  A vector short enough for one batch per thread (every normed input) is held in
 // registers across the block reduction; the down projection's long input comes with its producers' maxima.
 template <int WD>
 __device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* sh, unsigned char* xs, int cta, int K,
@@ -517,7 +545,8 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int kind
   constexpr int NA = (WD == W_BF16) ? 4 : 2;         // ldmatrix.x4 loads per unit
   unsigned fa[NA][4];                                // pending unit: weight fragments,
   uint4 fx0 = make_uint4(0u, 0u, 0u, 0u), fx1 = fx0; // input fragments,
-  unsigned fsz0 = 0u, fsz1 = 0u;                     // int4: {scale, zero} of my two rows
+  unsigned fsz0 = 0u, fsz1 = 0u;                     // int4: {scale, zero} of my two rows,
+  int4 fsx = make_int4(0, 0, 0, 0);                  //       the input group's digit sums for my two columns, its scale
   auto flush = [&]() {
     if (WD == W_BF16) {
       mma_bf16(facc, fa[0], fx0.x, fx0.y);
@@ -528,31 +557,26 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int kind
       mma_s8(iacc, fa[0][0], fa[0][1], fa[0][2], fa[0][3], fx0.x, fx0.y);
       mma_s8(iacc2, fa[1][0], fa[1][1], fa[1][2], fa[1][3], fx0.z, fx0.w);
     } else {
-      // sum over k of s (q_k - z) x_k = s (sum q_k x_k - z sum x_k): the codes go to the tensor cores as they are
-      // (unsigned bytes 0..15: one AND per four codes, a shift more for the high nibbles), and the zero point meets
-      // the sum of the input's digits over the group, which every lane takes from its own B fragments (its quad
-      // position's 32 columns of its digit column, then the quad) and hands to the lanes whose accumulator
-      // columns those are.
-      const float s0 = __half2float(__ushort_as_half((unsigned short)(fsz0 & 0xffffu)));
-      const float s1 = __half2float(__ushort_as_half((unsigned short)(fsz1 & 0xffffu)));
+      // sum over k of s (q_k - z) x_k = s (sum q_k x_k - z sum x_k): the codes go to the tensor cores as unsigned
+      // bytes, and the zero point meets the sum of the input's digits over the group, which the input's loader
+      // left in a table (store_item).
+      const float xsc = __int_as_float(fsx.z);
+      const float s0 = __half2float(__ushort_as_half((unsigned short)(fsz0 & 0xffffu))) * xsc;
+      const float s1 = __half2float(__ushort_as_half((unsigned short)(fsz1 & 0xffffu))) * xsc;
       const int z0 = (int)(fsz0 >> 16), z1 = (int)(fsz1 >> 16);      // (the packer stores the zero point as an integer)
-      constexpr unsigned M = 0x0F0F0F0Fu;
-      int g4[4] = {0, 0, 0, 0};
+      // The low nibbles go in as they are (one AND per four codes); the high nibbles stay where they are, as 16 x
+      // code (unsigned bytes 0..240), in a chain of their own whose exact sum is divided by 16 at the end.
+      constexpr unsigned M = 0x0F0F0F0Fu, MH = 0xF0F0F0F0u;
+      int g4[4] = {0, 0, 0, 0}, h4[4] = {0, 0, 0, 0};
       mma_u8s8(g4, fa[0][0] & M, fa[0][1] & M, fa[0][2] & M, fa[0][3] & M, fx0.x, fx0.y);
-      mma_u8s8(g4, (fa[0][0] >> 4) & M, (fa[0][1] >> 4) & M, (fa[0][2] >> 4) & M, (fa[0][3] >> 4) & M, fx0.z, fx0.w);
+      mma_u8s8(h4, fa[0][0] & MH, fa[0][1] & MH, fa[0][2] & MH, fa[0][3] & MH, fx0.z, fx0.w);
       mma_u8s8(g4, fa[1][0] & M, fa[1][1] & M, fa[1][2] & M, fa[1][3] & M, fx1.x, fx1.y);
-      mma_u8s8(g4, (fa[1][0] >> 4) & M, (fa[1][1] >> 4) & M, (fa[1][2] >> 4) & M, (fa[1][3] >> 4) & M, fx1.z, fx1.w);
-      int sx = __dp4a((int)fx0.x, 0x01010101, 0);
-      sx = __dp4a((int)fx0.y, 0x01010101, sx);
-      sx = __dp4a((int)fx0.z, 0x01010101, sx);
-      sx = __dp4a((int)fx0.w, 0x01010101, sx);
-      sx = __dp4a((int)fx1.x, 0x01010101, sx);
-      sx = __dp4a((int)fx1.y, 0x01010101, sx);
-      sx = __dp4a((int)fx1.z, 0x01010101, sx);
-      sx = __dp4a((int)fx1.w, 0x01010101, sx);
-      sx += __shfl_xor_sync(0xffffffffu, sx, 1);
-      sx += __shfl_xor_sync(0xffffffffu, sx, 2);
-      const int sx0 = __shfl_sync(0xffffffffu, sx, 8 * q), sx1 = __shfl_sync(0xffffffffu, sx, 8 * q + 4);
+      mma_u8s8(h4, fa[1][0] & MH, fa[1][1] & MH, fa[1][2] & MH, fa[1][3] & MH, fx1.z, fx1.w);
+      // digit sums of this group for my two accumulator columns (2q, 2q + 1): {D2, D1} for q = 0, {D0, -} for q = 1
+      // (the other quad positions' columns are not in use and weigh nothing in the end)
+      const int sx0 = fsx.x, sx1 = fsx.y;
+#pragma unroll
+      for (int e = 0; e < 4; e++) g4[e] += h4[e] >> 4;
       facc[0] = fmaf(s0, (float)(g4[0] - z0 * sx0), facc[0]);
       facc[1] = fmaf(s0, (float)(g4[1] - z0 * sx1), facc[1]);
       facc[2] = fmaf(s1, (float)(g4[2] - z1 * sx0), facc[2]);
@@ -573,33 +597,29 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int kind
     if (active && !c.bad) {
       const unsigned char* sbase = c.ring + (size_t)c.stage * p.stage_bytes;
       // my units in this tile: blocks next_b, next_b + Wk, ... while (b, wr) comes before (n_b, n_r)
-      while (next_b < g.nblk && (next_b < n_b || (next_b == n_b && wr < n_r))) {
+      const int end_b = min(g.nblk, n_b + (wr < n_r ? 1 : 0));
+      for (; next_b < end_b; next_b += g.Wk) {
         const unsigned char* u = sbase + (next_b * g.bb + my_off - tile_off);
-        fx0 = make_uint4(0u, 0u, 0u, 0u);
-        fx1 = fx0;
+        // (B columns beyond NCOL repeat the last one: their accumulator columns weigh nothing in the end)
         if (WD == W_BF16) {
-          if (gq < NCOL) {
-            const uint4* xp = reinterpret_cast<const uint4*>(xcol + ((size_t)next_b * BC + 16 * q) * 2);
-            fx0 = xp[0];
-            fx1 = xp[1];
-          }
+          const uint4* xp = reinterpret_cast<const uint4*>(xcol + ((size_t)next_b * BC + 16 * q) * 2);
+          fx0 = xp[0];
+          fx1 = xp[1];
         } else if (WD == W_INT8) {
-          if (gq < NCOL) fx0 = *reinterpret_cast<const uint4*>(xcol + (size_t)next_b * BC + 16 * q);
+          fx0 = *reinterpret_cast<const uint4*>(xcol + (size_t)next_b * BC + 16 * q);
         } else {
-          if (gq < NCOL) {
-            const uint4* xp = reinterpret_cast<const uint4*>(xcol + (size_t)next_b * BC + 32 * q);
-            fx0 = xp[0];
-            fx1 = xp[1];
-          }
+          const uint4* xp = reinterpret_cast<const uint4*>(xcol + (size_t)next_b * BC + 32 * q);
+          fx0 = xp[0];
+          fx1 = xp[1];
           // {scale, zero} of my two fragment rows for this group (= this column block)
           const unsigned* szp = reinterpret_cast<const unsigned*>(u + urows * 64);
           fsz0 = szp[min(gq, urows - 1)];
           fsz1 = szp[min(gq + 8, urows - 1)];
+          fsx = *reinterpret_cast<const int4*>(c.xs + 3 * (size_t)K + 32 * next_b + 16 * (q & 1));
         }
 #pragma unroll
         for (int j = 0; j < NA; j++) ldmatrix_x4(fa[j], u + lane_off + j * step_stride);
         flush();
-        next_b += g.Wk;
       }
     }
     __syncwarp();
@@ -614,8 +634,8 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int kind
   // per-row result: sum of the B columns in use, with the digit weights for integer inputs
   float y0, y1;
   if (WD == W_BF16) {
-    y0 = facc[0] + facc[1];                            // (columns not in use are zero; the sum over the quad follows)
-    y1 = facc[2] + facc[3];
+    y0 = (q == 0) ? facc[0] + facc[1] : 0.f;           // columns 0 and 1: the high and low parts
+    y1 = (q == 0) ? facc[2] + facc[3] : 0.f;
   } else {
     // columns 2q and 2q+1 of this lane: digit weights 65536 (col 0), 256 (col 1), 1 (col 2), 0 otherwise
     const float w0 = (q == 0) ? 65536.f : (q == 1 ? 1.f : 0.f);
@@ -713,7 +733,7 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind_rt, int l) {
   if (np > 0) {
     const unsigned in_seq = seq_of(p, src_task);
     LoadResult lr;
-    if (WD == W_BF16) lr = load_input_bf16(p, c.sh, c.xs, c.cta, K, src, in_seq, src_task, normw, task);
+    if (WD != W_INT8) lr = load_input_1pass<WD>(p, c.sh, c.xs, c.cta, K, src, in_seq, src_task, normw, task);
     else lr = load_input<WD>(p, c.sh, c.xs, c.cta, K, src, in_seq, src_task, normw, task,
                              kind == OP_DOWN ? p.m_amax : nullptr, c.nblk);
     rnorm = lr.rnorm;
@@ -750,7 +770,7 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind_rt, int l) {
     }
     const float resid = __uint_as_float(rraw.x);
     float sc0 = __half2float(sh0) * rnorm, sc1 = __half2float(sh1) * rnorm;
-    if (d.wdtype != W_BF16) { sc0 *= c.xscale; sc1 *= c.xscale; }
+    if (d.wdtype == W_INT8) { sc0 *= c.xscale; sc1 *= c.xscale; }
     c.bad = cons_sync_or(c.bad);
     if (c.bad) return false;
 
@@ -810,7 +830,7 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind_rt, int l) {
       }
     }
   }
-  if (WD != W_BF16 && kind == OP_GATEUP) {
+  if (WD == W_INT8 && kind == OP_GATEUP) {
     // publish this block's max |m|: the down projection scales its integer input by the maximum over all blocks
     gu_amax = warp_max_nonneg(gu_amax);
     if (c.lane == 0) c.sh->cand_val[c.warp] = gu_amax;
