@@ -131,6 +131,8 @@ int orc_argmax(const float* v, int n) {
  *   wdtype 2: int4 [rows][cols/2], element j in byte j/2 (even j: bits 0-3, odd j: bits 4-7),
  *             asymmetric, per row and group of `group` consecutive columns an fp16 scale and an
  *             integer-valued fp16 zero point: w = s * (q - z)
+ *   wdtype 3: int8 [rows][cols], symmetric, per row and group of `group` consecutive columns an fp16
+ *             scale: w = s * q  ("dequantize per group", Section 7)
  * The dequantised value is formed in fp32; both products are exact there (11-bit by <=8-bit
  * significands), so dequantised weights are comparable bit for bit.
  * -------------------------------------------------------------------------------------------- */
@@ -140,6 +142,10 @@ float orc_dequant(int wdtype, const void* W, const uint16_t* scale, const uint16
     size_t idx = (size_t)o * (size_t)cols + (size_t)j;
     if (wdtype == 0) return orc_bf16_to_f32(((const uint16_t*)W)[idx]);
     if (wdtype == 1) return orc_f16_to_f32(scale[o]) * (float)((const int8_t*)W)[idx];
+    if (wdtype == 3) {
+        size_t gi = (size_t)o * (size_t)(cols / group) + (size_t)(j / group);
+        return orc_f16_to_f32(scale[gi]) * (float)((const int8_t*)W)[idx];
+    }
     {
         uint8_t byte = ((const uint8_t*)W)[idx >> 1];
         int q = (j & 1) ? (byte >> 4) : (byte & 0x0f);
@@ -194,6 +200,33 @@ void orc_quantize_int8(const uint16_t* W_bf16, int rows, int cols, int8_t* q, ui
             if (r > 127.0f) r = 127.0f;
             if (r < -127.0f) r = -127.0f;
             q[(size_t)o * cols + j] = (int8_t)r;
+        }
+    }
+}
+
+/* int8, symmetric, per output row and group of `group` consecutive columns: the per-row rule applied to
+ * each group: s = fp16(amax/127) (1 if the group is all zero); q = clamp(rint(w / s), -127, 127). */
+void orc_quantize_int8_grouped(const uint16_t* W_bf16, int rows, int cols, int group, int8_t* q, uint16_t* scale) {
+    int ng = cols / group;
+#pragma omp parallel for schedule(static)
+    for (int o = 0; o < rows; o++) {
+        const uint16_t* w = W_bf16 + (size_t)o * cols;
+        for (int g = 0; g < ng; g++) {
+            float amax = 0.0f;
+            for (int j = g * group; j < (g + 1) * group; j++) {
+                float a = fabsf(orc_bf16_to_f32(w[j]));
+                if (a > amax) amax = a;
+            }
+            uint16_t sh = (amax == 0.0f) ? orc_f32_to_f16(1.0f) : orc_f32_to_f16(amax / 127.0f);
+            float s = orc_f16_to_f32(sh);
+            if (s == 0.0f) { sh = orc_f32_to_f16(1.0f); s = 1.0f; }
+            scale[(size_t)o * ng + g] = sh;
+            for (int j = g * group; j < (g + 1) * group; j++) {
+                float r = rintf(orc_bf16_to_f32(w[j]) / s);
+                if (r > 127.0f) r = 127.0f;
+                if (r < -127.0f) r = -127.0f;
+                q[(size_t)o * cols + j] = (int8_t)r;
+            }
         }
     }
 }
@@ -312,8 +345,8 @@ typedef struct {
     int32_t tied_embeddings;
     float rms_eps;
     float rope_theta;
-    int32_t wdtype;        /* 0 bf16, 1 int8, 2 int4: applies to the seven per-layer linears only */
-    int32_t group_size;    /* int4 group length along the input dimension */
+    int32_t wdtype;        /* 0 bf16, 1 int8, 2 int4, 3 grouped int8: applies to the seven per-layer linears only */
+    int32_t group_size;    /* int4 / grouped int8: group length along the input dimension */
     int32_t round_kv;      /* 1: cache entries rounded to bf16 (the contract); 0: test-only, see below */
     int32_t quantize_lm_head; /* 0: the LM head stays bf16 (the reading taken of the paper); 1: it is quantised like
                                  the per-layer linears (wdtype, group_size) -- the other reading of "linear GEMV

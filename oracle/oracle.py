@@ -20,7 +20,7 @@ _SRC = os.path.join(_HERE, "oracle.c")
 _LIB = os.path.join(_HERE, "liboracle.so")
 
 KINDS = ("wq", "wk", "wv", "wo", "wgate", "wup", "wdown")
-W_BF16, W_INT8, W_INT4 = 0, 1, 2
+W_BF16, W_INT8, W_INT4, W_INT8G = 0, 1, 2, 3
 
 
 def build(force: bool = False) -> str:
@@ -156,12 +156,13 @@ def argmax(v) -> int:
 
 
 def gemv(wdtype: int, W, x, scale=None, zero=None, group: int = 128) -> np.ndarray:
-    """y = deq(W) x.  W: uint16 [rows][cols] (bf16 bits), int8 [rows][cols] or uint8 [rows][cols/2]."""
+    """y = deq(W) x.  W: uint16 [rows][cols] (bf16 bits), int8 [rows][cols] (per-row or grouped scales) or uint8
+    [rows][cols/2]."""
     x = _c(x, np.float32)
     cols = x.size
     if wdtype == W_BF16:
         W = _c(W, np.uint16)
-    elif wdtype == W_INT8:
+    elif wdtype in (W_INT8, W_INT8G):
         W = _c(W, np.int8)
     else:
         W = _c(W, np.uint8)
@@ -179,7 +180,7 @@ def dequant(wdtype: int, W, scale=None, zero=None, group: int = 128) -> np.ndarr
     if wdtype == W_BF16:
         W = _c(W, np.uint16)
         rows, cols = W.shape
-    elif wdtype == W_INT8:
+    elif wdtype in (W_INT8, W_INT8G):
         W = _c(W, np.int8)
         rows, cols = W.shape
     else:
@@ -202,6 +203,16 @@ def quantize_int8(W_bf16):
     q = np.empty((rows, cols), dtype=np.int8)
     s = np.empty(rows, dtype=np.uint16)
     lib().orc_quantize_int8(_p(W), C.c_int(rows), C.c_int(cols), _p(q), _p(s))
+    return q, s
+
+
+def quantize_int8_grouped(W_bf16, group: int = 128):
+    W = _c(W_bf16, np.uint16)
+    rows, cols = W.shape
+    assert cols % group == 0
+    q = np.empty((rows, cols), dtype=np.int8)
+    s = np.empty((rows, cols // group), dtype=np.uint16)
+    lib().orc_quantize_int8_grouped(_p(W), C.c_int(rows), C.c_int(cols), C.c_int(group), _p(q), _p(s))
     return q, s
 
 
@@ -316,7 +327,7 @@ class Model:
         w.final_norm = self._hold(weights["final_norm"], np.uint16)
         w.attn_norm = self._ptr_array(weights["attn_norm"], np.uint16)
         w.mlp_norm = self._ptr_array(weights["mlp_norm"], np.uint16)
-        wdt = {W_BF16: np.uint16, W_INT8: np.int8, W_INT4: np.uint8}[wdtype]
+        wdt = {W_BF16: np.uint16, W_INT8: np.int8, W_INT4: np.uint8, W_INT8G: np.int8}[wdtype]
         for i, kind in enumerate(KINDS):
             w.w[i] = self._ptr_array(weights[kind], wdt)
             if wdtype != W_BF16:
@@ -411,8 +422,8 @@ def quantize_weights(weights: Dict, wdtype: int, group: int = 128) -> Dict:
     for kind in KINDS:
         qs, ss, zs = [], [], []
         for W in weights[kind]:
-            if wdtype == W_INT8:
-                q, s = quantize_int8(W)
+            if wdtype in (W_INT8, W_INT8G):
+                q, s = quantize_int8(W) if wdtype == W_INT8 else quantize_int8_grouped(W, group)
                 qs.append(q)
                 ss.append(s)
             else:
@@ -434,6 +445,8 @@ def quantize_lm_head(weights: Dict, wdtype: int, group: int = 128, tied: bool = 
     W = weights["embed"] if (tied or weights.get("lm_head") is None) else weights["lm_head"]
     if wdtype == W_INT8:
         out["lm_head_q"], out["lm_head_scale"] = quantize_int8(W)
+    elif wdtype == W_INT8G:
+        out["lm_head_q"], out["lm_head_scale"] = quantize_int8_grouped(W, group)
     elif wdtype == W_INT4:
         out["lm_head_q"], out["lm_head_scale"], out["lm_head_zero"] = quantize_int4(W, group)
     return out

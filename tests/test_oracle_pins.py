@@ -273,6 +273,15 @@ def test_gemv_exact_integer_cases():
     ref = ((q4.astype(np.int64) - np.repeat(zvals, group, axis=1)) * x4.astype(np.int64)).sum(axis=1) * 0.25
     assert np.array_equal(y, ref.astype(np.float32))
     assert np.array_equal(orc.unpack_int4(packed), q4)
+    # grouped int8: a different power-of-two scale per (row, group); a scale taken from the wrong row or group, or
+    # applied per row, changes the integers
+    ng = cols4 // group
+    q8g = rng.integers(-127, 128, size=(rows, cols4)).astype(np.int8)
+    exps = rng.integers(-6, 3, size=(rows, ng))
+    s8g = (2.0 ** exps).astype(np.float16).view(np.uint16)
+    y = orc.gemv(orc.W_INT8G, q8g, x4, scale=s8g, group=group)
+    ref = ((q8g.astype(np.int64) * x4.astype(np.int64)).reshape(rows, ng, group).sum(axis=2) * 2.0 ** exps).sum(axis=1)
+    assert np.array_equal(y, ref.astype(np.float32))
 
 
 def test_silu_values():
@@ -315,6 +324,19 @@ def test_int8_quantiser_hand_row():
     assert np.allclose(d[0], [0.10010290, -0.04965734, 0.02522278, 0.0], atol=1e-8)
 
 
+def test_grouped_int8_quantiser_hand_groups():
+    # two groups of four with very different ranges: each gets the per-row rule on its own
+    W = np.array([[0x3DCD, 0xBD4D, 0x3CCD, 0x0000, 0x3A83, 0xBA03, 0x0000, 0x3983]], dtype=np.uint16)
+    q, s = orc.quantize_int8_grouped(W, group=4)
+    assert s.shape == (1, 2) and s[0, 0] == 0x1275                     # fp16(0.10009766 / 127), as the per-row pin
+    assert q[0, :4].tolist() == [127, -63, 32, 0]
+    # second group: 0x3A83 = 0.0010004044 is its maximum -> code 127; half of it -> -63 or -64; a quarter -> 32
+    assert q[0, 4] == 127 and q[0, 5] in (-63, -64) and q[0, 6] == 0 and q[0, 7] in (31, 32)
+    assert s[0, 1] == np.float16(np.float32(0.0010004044) / np.float32(127)).view(np.uint16)
+    d = orc.dequant(orc.W_INT8G, q, s, group=4)
+    assert np.allclose(d[0, :4], [0.10010290, -0.04965734, 0.02522278, 0.0], atol=1e-8)
+
+
 def test_int4_quantiser_hand_group():
     vals = np.array([[-0.03002930, 0.0, 0.01501465, 0.04492188]], dtype=np.float32)
     W = bf16_bits(vals)
@@ -342,9 +364,20 @@ def test_quantisers_vs_numpy_float16_and_error_bounds():
     assert np.array_equal(q, np.clip(np.rint(Wv / sf[:, None]), -127, 127).astype(np.int8))
     d = orc.dequant(orc.W_INT8, q, s)
     assert (np.abs(d - Wv) <= sf[:, None] * 0.5 * (1 + 1e-6)).all()
+    # grouped int8: the per-row rule per (row, group); with one group per row it IS the per-row quantiser
+    qg, sg = orc.quantize_int8_grouped(W, group)
+    Wg = Wv.reshape(rows, cols // group, group)
+    amaxg = np.abs(Wg).max(axis=2)
+    sg_ref = np.where(amaxg == 0, np.float16(1.0), (amaxg / np.float32(127)).astype(np.float16))
+    assert np.array_equal(sg, sg_ref.view(np.uint16))
+    sgf = sg_ref.astype(np.float32)
+    assert np.array_equal(qg.reshape(Wg.shape), np.clip(np.rint(Wg / sgf[:, :, None]), -127, 127).astype(np.int8))
+    dg = orc.dequant(orc.W_INT8G, qg, sg, group=group).reshape(Wg.shape)
+    assert (np.abs(dg - Wg) <= sgf[:, :, None] * 0.5 * (1 + 1e-6)).all()
+    q1, s1 = orc.quantize_int8_grouped(W, cols)
+    assert np.array_equal(q1, q) and np.array_equal(s1[:, 0], s)
     p, s4, z4 = orc.quantize_int4(W, group)
     codes = orc.unpack_int4(p)
-    Wg = Wv.reshape(rows, cols // group, group)
     mn = np.minimum(Wg.min(axis=2), 0)
     mx = np.maximum(Wg.max(axis=2), 0)
     s4_ref = np.where(mx == mn, np.float16(1.0), ((mx - mn) / np.float32(15)).astype(np.float16))
