@@ -34,6 +34,8 @@ WORKLOADS = {
     "llama3_8b_bf16_pos0": ("llama3_8b", "bf16", 0),
     "llama3_8b_int8_pos0": ("llama3_8b", "int8", 0),
     "llama3_8b_int4_pos0": ("llama3_8b", "int4", 0),
+    "llama3_8b_int8g_pos0": ("llama3_8b", "int8g", 0),
+    "tinyllama_1b_int8g_pos0": ("tinyllama_1b", "int8g", 0),
     "llama3_8b_bf16_pos4096": ("llama3_8b", "bf16", 4096),
     "llama3_8b_int8_pos4096": ("llama3_8b", "int8", 4096),
     "tinyllama_1b_int8_pos512": ("tinyllama_1b", "int8", 512),
@@ -58,7 +60,7 @@ OTHER = ["llama3_8b_int8_pos0", "tinyllama_1b_bf16_pos0", "tinyllama_1b_int8_pos
          "smollm2_135m_bf16_pos0", "tinyllama_1b_bf16_pos1024", "tinyllama_1b_int8_pos512", "llama3_8b_int8_pos4096",
          "llama3_8b_bf16_pos4096", "llama32_1b_bf16_pos0", "llama32_1b_int8_pos0", "tinyllama_1b_int8_qhead_pos0",
          "llama3_8b_int8_qhead_pos0", "paper_small_bf16_pos0", "paper_small_int8_pos0", "paper_small_int4_pos0",
-         "llama3_8b_int4_pos0"]
+         "llama3_8b_int4_pos0", "tinyllama_1b_int8g_pos0", "llama3_8b_int8g_pos0"]
 # device-resident multi-token runs (amk_decode_greedy: the token is fed back on the device): (shape, dtype, steps)
 SUSTAINED = [("smollm2_135m", "bf16", 256), ("tinyllama_1b", "bf16", 256)]
 METRIC = "batch-1 decode us/token; achieved HBM GB/s vs B200 measured peak"
@@ -218,7 +220,7 @@ def time_e2e(dec, shape, tok, pos, kv, steps, warmup):
     return dt / steps * 1e6, 4, 4 + 4 * shape.vocab
 
 
-WDT = {"bf16": 0, "int8": 1, "int4": 2}
+WDT = {"bf16": 0, "int8": 1, "int4": 2, "int8g": 3}
 
 
 class OracleSample:

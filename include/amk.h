@@ -41,7 +41,7 @@ typedef enum {
   AMK_ERR_BAD_TOKEN = 8    /* token < 0 or token >= vocab                                               */
 } amk_status;
 
-typedef enum { AMK_W_BF16 = 0, AMK_W_INT8 = 1, AMK_W_INT4 = 2 } amk_wdtype;
+typedef enum { AMK_W_BF16 = 0, AMK_W_INT8 = 1, AMK_W_INT4 = 2, AMK_W_INT8_GROUPED = 3 } amk_wdtype;
 
 /* amk_config.flags */
 #define AMK_FLAG_DEBUG_HIDDEN 1u /* keep the residual stream after the embedding and after every layer */
@@ -92,7 +92,7 @@ typedef struct amk_config {
   float rms_eps;             /* RMSNorm epsilon (inside the square root)                               */
   float rope_theta;          /* rotary base; pairs (i, i + head_dim/2), no scaling                     */
   uint32_t wdtype;           /* amk_wdtype of the seven per-layer linears                              */
-  uint32_t group_size;       /* int4: 128 (the only supported value); ignored otherwise                */
+  uint32_t group_size;       /* int4, grouped int8: 128 (the only supported value); ignored otherwise  */
   uint32_t quantize_lm_head; /* 0: the LM head stays bf16 (tied or not), as the paper says of the tied
                                 embedding matrix.  1 (int8 / int4 models only): the LM head GEMV streams a
                                 copy quantised like the layers (amk_weights.lm_head_q ...); the embedding
@@ -122,6 +122,8 @@ typedef struct amk_config {
  *   int8 : int8 [out][in]; scale fp16 [out]                       w = scale * q, q in [-127, 127]
  *   int4 : uint8 [out][in/2], element j in byte j/2 (even j: bits 0-3); scale fp16 [out][in/128];
  *          zero fp16 [out][in/128] holding an integer 0..15        w = scale * (q - zero)
+ *   grouped int8 : int8 [out][in]; scale fp16 [out][in/128]       w = scale * q, q in [-127, 127]
+ *          (the paper's ring variant dequantises "per group", Section 7; the group length is the int4 one)
  */
 typedef struct amk_weights {
   const void* embed;                        /* bf16 [V][H]                                            */
@@ -133,7 +135,8 @@ typedef struct amk_weights {
   const void* const* scale[AMK_LIN_COUNT];  /* [L] each; NULL arrays for bf16                         */
   const void* const* zero[AMK_LIN_COUNT];   /* [L] each; int4 only                                    */
   /* quantize_lm_head = 1 only: the LM head matrix (the embedding matrix when tied) quantised like a layer
-   * linear of [V][H]: codes, fp16 scales (int8 [V]; int4 [V][H/128]) and, for int4, fp16 zero points */
+   * linear of [V][H]: codes, fp16 scales (int8 [V]; int4 and grouped int8 [V][H/128]) and, for int4, fp16 zero
+   * points */
   const void* lm_head_q;
   const void* lm_head_scale;
   const void* lm_head_zero;
@@ -259,10 +262,13 @@ amk_status amk_destroy(amk_handle* h);
  *   int4: per row and group of 128 columns, mn = min(w, 0), mx = max(w, 0); s = fp16((mx - mn) / 15)
  *         (1 if mx == mn); z = clamp(rint(-mn / s), 0, 15); q = clamp(rint(w / s) + z, 0, 15);
  *         two codes per byte, even column in the low nibble; z stored as an fp16 integer.
- * All pointers DEVICE; w_bf16 is [rows][cols] bf16.  cols % 128 == 0 for int4.  Asynchronous.
+ *   grouped int8: the int8 rule per row and group of 128 columns; scale_out is fp16 [rows][cols/128].
+ * All pointers DEVICE; w_bf16 is [rows][cols] bf16.  cols % 128 == 0 for int4 and grouped int8.  Asynchronous.
  */
 amk_status amk_quantize_int8(const void* w_bf16, int64_t rows, int64_t cols, void* q_out, void* scale_out,
                              void* cuda_stream);
+amk_status amk_quantize_int8_grouped(const void* w_bf16, int64_t rows, int64_t cols, void* q_out, void* scale_out,
+                                     void* cuda_stream);
 amk_status amk_quantize_int4(const void* w_bf16, int64_t rows, int64_t cols, void* packed_out, void* scale_out,
                              void* zero_out, void* cuda_stream);
 

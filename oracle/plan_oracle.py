@@ -8,7 +8,7 @@ model is decided by brute force -- an explicit graph of (task, block) events for
 reachability -- instead of the checker's rule about all-to-all joins.
 
 is_safe(words, model) -> (bool, reason).  `model` is a dict with hidden, n_layers, n_q_heads, n_kv_heads,
-head_dim, mlp, vocab, wdtype (0 bf16, 1 int8, 2 int4), stage_bytes, n_blocks, and optionally lm_wdtype (the LM
+head_dim, mlp, vocab, wdtype (0 bf16, 1 int8, 2 int4, 3 grouped int8), stage_bytes, n_blocks, and optionally lm_wdtype (the LM
 head's dtype when it is quantised like the layers; 0 otherwise).
 """
 from collections import deque
@@ -25,11 +25,13 @@ def _cdiv(a, b):
 
 
 def _unit_bytes(wd, rows):
-    """A work unit = the rows of one row-warp over one column block (64 columns; 128 for int4)."""
+    """A work unit = the rows of one row-warp over one column block (64 columns; 128 for int4 and grouped int8)."""
     if wd == 0:
         return rows * 128                      # 64 bf16
     if wd == 1:
         return rows * 64                       # 64 int8
+    if wd == 3:
+        return (rows * 132 + 15) // 16 * 16    # 128 int8 + {fp16 scale, pad} per row, padded to 16 bytes
     return (rows * 68 + 15) // 16 * 16         # 128 nibbles + {scale, zero} fp16 per row, padded to 16 bytes
 
 
@@ -43,7 +45,7 @@ def _pass_tiles(rows, k, wd, stage):
     g = _cdiv(rows, wr)
     wr = _cdiv(rows, g)
     g_last = rows - (wr - 1) * g
-    nblk = k // (128 if wd == 2 else 64)
+    nblk = k // (128 if wd in (2, 3) else 64)
     ub, ubl = _unit_bytes(wd, g), _unit_bytes(wd, g_last)
     block_bytes = (wr - 1) * ub + ubl
     n_units = wr * nblk

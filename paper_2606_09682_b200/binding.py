@@ -18,7 +18,7 @@ LIB_PATH = os.environ.get("AMK_LIB") or os.path.join(_HERE, "libamk.so")      # 
 AMK_ABI_VERSION = 2
 AMK_OK, AMK_ERR_INVALID_ARG, AMK_ERR_UNSUPPORTED, AMK_ERR_CUDA, AMK_ERR_OOM = 0, 1, 2, 3, 4
 AMK_ERR_TIMEOUT, AMK_ERR_ABORTED, AMK_ERR_BAD_POS, AMK_ERR_BAD_TOKEN = 5, 6, 7, 8
-AMK_W_BF16, AMK_W_INT8, AMK_W_INT4 = 0, 1, 2
+AMK_W_BF16, AMK_W_INT8, AMK_W_INT4, AMK_W_INT8_GROUPED = 0, 1, 2, 3
 AMK_FLAG_DEBUG_HIDDEN = 1
 AMK_FLAG_TRACE = 2
 AMK_FLAG_MEASURED_SPLIT = 4
@@ -26,7 +26,7 @@ AMK_FLAG_TRACE_CYCLES = 8
 AMK_TRACE_EVENTS = 12
 AMK_LIN_Q, AMK_LIN_K, AMK_LIN_V, AMK_LIN_O, AMK_LIN_GATE, AMK_LIN_UP, AMK_LIN_DOWN, AMK_LIN_LM_HEAD = range(8)
 KINDS = ("wq", "wk", "wv", "wo", "wgate", "wup", "wdown")
-WDTYPES = {"bf16": AMK_W_BF16, "int8": AMK_W_INT8, "int4": AMK_W_INT4}
+WDTYPES = {"bf16": AMK_W_BF16, "int8": AMK_W_INT8, "int4": AMK_W_INT4, "int8g": AMK_W_INT8_GROUPED}
 
 
 class amk_config(C.Structure):
@@ -79,6 +79,7 @@ def _load() -> C.CDLL:
         "amk_last_kernel_ns": (C.c_int, [vp, C.POINTER(C.c_uint64)]),
         "amk_destroy": (C.c_int, [vp]),
         "amk_quantize_int8": (C.c_int, [vp, i64, i64, vp, vp, vp]),
+        "amk_quantize_int8_grouped": (C.c_int, [vp, i64, i64, vp, vp, vp]),
         "amk_quantize_int4": (C.c_int, [vp, i64, i64, vp, vp, vp, vp]),
         "amk_argmax_static": (C.c_int, [vp, i64, vp, C.c_char_p, sz, vp]),
         "amk_plan_export": (C.c_int, [C.POINTER(amk_config), vp, sz, C.POINTER(sz)]),
@@ -93,7 +94,7 @@ def _load() -> C.CDLL:
 lib = _load()
 EXPORTS = ("amk_status_str", "amk_packed_bytes", "amk_workspace_bytes", "amk_kv_bytes", "amk_create",
            "amk_decode_step", "amk_decode_greedy", "amk_last_status", "amk_plan_info", "amk_debug_hidden",
-           "amk_debug_trace", "amk_debug_unpack", "amk_debug_drop_signal", "amk_debug_set_step_count", "amk_last_kernel_ns", "amk_destroy", "amk_quantize_int8", "amk_quantize_int4",
+           "amk_debug_trace", "amk_debug_unpack", "amk_debug_drop_signal", "amk_debug_set_step_count", "amk_last_kernel_ns", "amk_destroy", "amk_quantize_int8", "amk_quantize_int8_grouped", "amk_quantize_int4",
            "amk_argmax_static", "amk_plan_export", "amk_plan_check")
 
 
@@ -120,7 +121,7 @@ def make_config(shape, wdtype: str = "bf16", flags: int = 0, wait_timeout_us: in
     c.tied_embeddings = int(shape.tied)
     c.rms_eps, c.rope_theta = shape.rms_eps, shape.rope_theta
     c.wdtype = WDTYPES[wdtype]
-    c.group_size = group_size if wdtype == "int4" else 0
+    c.group_size = group_size if wdtype in ("int4", "int8g") else 0
     c.wait_timeout_us, c.flags = wait_timeout_us, flags
     c.stage_bytes, c.n_stages, c.max_inflight = stage_bytes, n_stages, max_inflight
     c.sync_mode, c.n_blocks, c.l2_ahead = sync_mode, n_blocks, l2_ahead
@@ -157,6 +158,17 @@ def amk_quantize_int8(w: torch.Tensor):
     q = torch.empty((rows, cols), dtype=torch.int8, device=w.device)
     s = torch.empty((rows,), dtype=torch.float16, device=w.device)
     _check(lib.amk_quantize_int8(w.data_ptr(), rows, cols, q.data_ptr(), s.data_ptr(), _stream()), "amk_quantize_int8")
+    return q, s
+
+
+def amk_quantize_int8_grouped(w: torch.Tensor):
+    """bf16 [rows][cols] (cuda) -> (int8 [rows][cols], fp16 scale [rows][cols/128])."""
+    assert w.is_cuda and w.dtype == torch.bfloat16 and w.is_contiguous()
+    rows, cols = w.shape
+    q = torch.empty((rows, cols), dtype=torch.int8, device=w.device)
+    s = torch.empty((rows, cols // 128), dtype=torch.float16, device=w.device)
+    _check(lib.amk_quantize_int8_grouped(w.data_ptr(), rows, cols, q.data_ptr(), s.data_ptr(), _stream()),
+           "amk_quantize_int8_grouped")
     return q, s
 
 
@@ -217,6 +229,8 @@ def quantize_weights(weights: Dict, wdtype: str) -> Dict:
         for w in weights[kind]:
             if wdtype == "int8":
                 q, s = amk_quantize_int8(w)
+            elif wdtype == "int8g":
+                q, s = amk_quantize_int8_grouped(w)
             else:
                 q, s, z = amk_quantize_int4(w)
                 zs.append(z)
@@ -235,6 +249,8 @@ def quantize_lm_head(weights: Dict, wdtype: str, tied: bool) -> Dict:
     w = weights["embed"] if (tied or weights.get("lm_head") is None) else weights["lm_head"]
     if wdtype == "int8":
         out["lm_head_q"], out["lm_head_scale"] = amk_quantize_int8(w)
+    elif wdtype == "int8g":
+        out["lm_head_q"], out["lm_head_scale"] = amk_quantize_int8_grouped(w)
     elif wdtype == "int4":
         out["lm_head_q"], out["lm_head_scale"], out["lm_head_zero"] = amk_quantize_int4(w)
     return out
@@ -363,6 +379,9 @@ class Decoder:
         elif wd == "int8":
             out = torch.zeros((rows, cols), dtype=torch.int8, device=self.device)
             scale = torch.zeros((rows,), dtype=torch.float16, device=self.device)
+        elif wd == "int8g":
+            out = torch.zeros((rows, cols), dtype=torch.int8, device=self.device)
+            scale = torch.zeros((rows, cols // 128), dtype=torch.float16, device=self.device)
         else:
             out = torch.zeros((rows, cols // 2), dtype=torch.uint8, device=self.device)
             scale = torch.zeros((rows, cols // 128), dtype=torch.float16, device=self.device)

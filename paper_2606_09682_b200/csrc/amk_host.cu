@@ -68,7 +68,7 @@ amk_status check_config(const amk_config* c) {
   if (c->l2_ahead > 33u) return AMK_ERR_INVALID_ARG;
   if (!c->hidden || !c->n_layers || !c->n_q_heads || !c->n_kv_heads || !c->mlp || !c->vocab || !c->max_seq)
     return AMK_ERR_INVALID_ARG;
-  if (c->wdtype > AMK_W_INT4 || c->sync_mode > 2) return AMK_ERR_INVALID_ARG;
+  if (c->wdtype > AMK_W_INT8_GROUPED || c->sync_mode > 2) return AMK_ERR_INVALID_ARG;
   if (5ull * c->n_layers + 1 > 2047ull) return AMK_ERR_UNSUPPORTED;      // a tile entry keeps its task in 11 bits
   if (c->n_blocks > (uint32_t)kMaxBlocks) return AMK_ERR_INVALID_ARG;
   if (c->head_dim != 64 && c->head_dim != 128) return AMK_ERR_UNSUPPORTED;
@@ -76,11 +76,11 @@ amk_status check_config(const amk_config* c) {
   if (c->n_q_heads / c->n_kv_heads > (uint32_t)kMaxRep) return AMK_ERR_UNSUPPORTED;
   if (c->quantize_lm_head > 1) return AMK_ERR_INVALID_ARG;
   if (c->quantize_lm_head && c->wdtype == AMK_W_BF16) return AMK_ERR_UNSUPPORTED;   // nothing to quantise it like
-  const uint32_t kdiv = (c->wdtype == AMK_W_INT4) ? 128 : 64;
+  const uint32_t kdiv = grouped((int)c->wdtype) ? 128 : 64;
   const uint32_t qdim = c->n_q_heads * c->head_dim;
   if (c->hidden % kdiv || c->mlp % kdiv || qdim % kdiv) return AMK_ERR_UNSUPPORTED;
   if (c->hidden > 16u * kConsumerThreads) return AMK_ERR_UNSUPPORTED;   // a normed input is gathered in one batch
-  if (c->wdtype == AMK_W_INT4 && c->group_size != 128) return AMK_ERR_UNSUPPORTED;
+  if (grouped((int)c->wdtype) && c->group_size != 128) return AMK_ERR_UNSUPPORTED;
   if ((uint64_t)c->vocab * c->hidden > (1ull << 40)) return AMK_ERR_UNSUPPORTED;
   if (c->stage_bytes && (c->stage_bytes % 1024 || c->stage_bytes < 8192 || c->stage_bytes > 65536))
     return AMK_ERR_INVALID_ARG;
@@ -268,8 +268,8 @@ amk_status amk_packed_bytes(const amk_config* cfg, size_t* bytes) {
   amk_status st = check_config(cfg);
   if (st != AMK_OK) return st;
   const Plan pl = make_plan(cfg, resolve_blocks(cfg), nullptr, false, nullptr, nullptr);
-  // int4 work units are padded to 16 bytes, so the total depends a little on the split: leave room
-  *bytes = pl.packed_total + (cfg->wdtype == AMK_W_INT4 ? pl.packed_total / 64 : 0);
+  // work units with scales inside are padded to 16 bytes, so the total depends a little on the split: leave room
+  *bytes = pl.packed_total + (grouped((int)cfg->wdtype) ? pl.packed_total / 64 : 0);
   return AMK_OK;
 }
 
@@ -427,7 +427,7 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     size_t kmax = (size_t)(H > I ? H : I);
     if ((size_t)qd > kmax) kmax = qd;
     size_t act = kmax * (cfg->wdtype == AMK_W_BF16 ? 4 : 3);   // bf16 high + low halves, or three int8 digits
-    if (cfg->wdtype == AMK_W_INT4) act += kmax / 4;            // + 32 bytes per group of 128: digit sums and scale
+    if (cfg->wdtype != AMK_W_BF16) act += (kmax + 127) / 128 * 32;   // + 32 bytes per group of 128: digit sums and scale
     if (!cfg->quantize_lm_head && (size_t)H * 4 > act) act = (size_t)H * 4;   // a bf16 LM head in an integer model
     // attention scratch: q vectors, per-warp partial outputs, the new K / V rows, the scores of the longest chunk
     int lc_max = 0, c_max = 0;
@@ -808,6 +808,14 @@ amk_status amk_quantize_int8(const void* w_bf16, int64_t rows, int64_t cols, voi
                              void* cuda_stream) {
   if (!w_bf16 || !q_out || !scale_out || rows < 0 || cols <= 0 || rows > 0x7fffffff) return AMK_ERR_INVALID_ARG;
   return launch_quantize_int8(w_bf16, rows, cols, q_out, scale_out, (cudaStream_t)cuda_stream) == cudaSuccess
+             ? AMK_OK
+             : AMK_ERR_CUDA;
+}
+
+amk_status amk_quantize_int8_grouped(const void* w_bf16, int64_t rows, int64_t cols, void* q_out, void* scale_out,
+                                     void* cuda_stream) {
+  if (!w_bf16 || !q_out || !scale_out || rows < 0 || cols <= 0 || cols % 128) return AMK_ERR_INVALID_ARG;
+  return launch_quantize_int8_grouped(w_bf16, rows, cols, q_out, scale_out, (cudaStream_t)cuda_stream) == cudaSuccess
              ? AMK_OK
              : AMK_ERR_CUDA;
 }

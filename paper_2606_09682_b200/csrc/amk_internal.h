@@ -139,6 +139,7 @@ cudaError_t launch_pack(const PackOp& d, const PackSrc& src, unsigned char* pack
 cudaError_t launch_calibrate(const unsigned char* src, size_t bytes_per_block, int n_blocks, size_t smem_bytes,
                              unsigned* smid_out, unsigned long long* ns_out, cudaStream_t stream);
 cudaError_t launch_quantize_int8(const void* w, int64_t rows, int64_t cols, void* q, void* scale, cudaStream_t s);
+cudaError_t launch_quantize_int8_grouped(const void* w, int64_t rows, int64_t cols, void* q, void* scale, cudaStream_t s);
 cudaError_t launch_quantize_int4(const void* w, int64_t rows, int64_t cols, void* packed, void* scale, void* zero,
                                  cudaStream_t s);
 

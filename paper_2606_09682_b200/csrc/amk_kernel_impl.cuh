@@ -62,7 +62,6 @@ struct Ctx {
   int stage;             // ring stage of the next tile this warp walks
   unsigned parity;       // its phase parity
   int token;
-  float xscale;          // int8 / int4: scale of the digit representation of the current input vector
   bool bad;              // this thread saw a failure; agreed on at the next consumer barrier
 };
 
@@ -251,8 +250,10 @@ __device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi) {      // {b
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
 }
+// (integer weights: called by whole warps -- the warp's 32 items are one group of 128 elements sharing a scale;
+//  `valid` is false for the lanes beyond the end of a vector whose length is not a multiple of 128, which pass zeros)
 template <int WD>
-__device__ __forceinline__ void store_item(unsigned char* xs, int n4, int it, const float (&a)[4], float inv = 0.f) {
+__device__ __forceinline__ void store_item(unsigned char* xs, int n4, int it, const float (&a)[4], bool valid = true) {
   if (WD == W_BF16) {
     // two B columns: bf16(a) and bf16(a - bf16(a)); their sum is a to 2^-17 (a third column would make it exact
     // and measured 1.3 % slower at the TinyLlama shape for an error far below the others')
@@ -264,13 +265,10 @@ __device__ __forceinline__ void store_item(unsigned char* xs, int n4, int it, co
   } else {
     // X = d2 * 65536 + d1 * 256 + d0 with every digit in [-128, 127] (see kDigitBias)
     unsigned* D2 = reinterpret_cast<unsigned*>(xs);                  // columns of K bytes = n4 items of 4 bytes
-    float gmax = 0.f;
-    if (WD == W_INT4) {
-      // int4: a scale of its own for every group of 128 elements, which is exactly a warp's 32 items (items are
-      // dealt out warp by warp and K is a multiple of 128): one warp-wide maximum, no pass over the whole vector
-      gmax = warp_max_nonneg(fmaxf(fmaxf(fabsf(a[0]), fabsf(a[1])), fmaxf(fabsf(a[2]), fabsf(a[3]))));
-      inv = gmax > 0.f ? __fdividef(kDigitScale, gmax) : 0.f;
-    }
+    // a scale of its own for every group of 128 elements, which is exactly a warp's 32 items (items are dealt out
+    // warp by warp): one warp-wide maximum, no pass over the whole vector
+    const float gmax = warp_max_nonneg(fmaxf(fmaxf(fabsf(a[0]), fabsf(a[1])), fmaxf(fabsf(a[2]), fabsf(a[3]))));
+    const float inv = gmax > 0.f ? __fdividef(kDigitScale, gmax) : 0.f;
     unsigned t[4];
 #pragma unroll
     for (int e = 0; e < 4; e++) t[e] = __float_as_uint(fmaf(a[e], inv, kDigitBias));
@@ -278,17 +276,24 @@ __device__ __forceinline__ void store_item(unsigned char* xs, int n4, int it, co
     const unsigned w0 = __byte_perm(p01, p23, 0x5410) ^ 0x80808080u;
     const unsigned w1 = __byte_perm(p01, p23, 0x7632) ^ 0x80808080u;
     const unsigned w2 = (__byte_perm(__byte_perm(t[0], t[1], 0x0062), __byte_perm(t[2], t[3], 0x0062), 0x5410) + 0x40404040u) ^ 0x80808080u;
-    D2[2 * n4 + it] = w0;
-    D2[n4 + it] = w1;
-    D2[it] = w2;
-    if (WD == W_INT4) {
-      // The zero point of a weight group meets the sum of the input's integers X over the group (see consume_pass):
-      // one warp-wide integer sum (below 2^29), split into signed base-256 digits like the elements themselves so
-      // that each meets the accumulator column of its weight.  The group's entry of the table behind the digit
-      // columns, laid out by accumulator column pair: {A2, A1, scale, -} {A0, 0, scale, -}.
-      const int sx = (int)(__reduce_add_sync(0xffffffffu, (t[0] + t[1]) + (t[2] + t[3])) - 128u * 0x4B408080u);
-      const int s0 = (sx << 24) >> 24, r1 = (sx - s0) >> 8;
-      const int s1 = (r1 << 24) >> 24, s2 = (r1 - s1) >> 8;
+    if (valid) {
+      D2[2 * n4 + it] = w0;
+      D2[n4 + it] = w1;
+      D2[it] = w2;
+    }
+    {
+      // The group's entry of the table behind the digit columns, laid out by accumulator column pair:
+      // {A2, A1, scale, -} {A0, 0, scale, -}.  int4: the zero point of a weight group meets the sum of the input's
+      // integers X over the group (see consume_pass): one warp-wide integer sum (below 2^29), split into signed
+      // base-256 digits A like the elements themselves so that each meets the accumulator column of its weight.
+      int s0 = 0, s1 = 0, s2 = 0;
+      if (WD == W_INT4) {
+        const int sx = (int)(__reduce_add_sync(0xffffffffu, (t[0] + t[1]) + (t[2] + t[3])) - 128u * 0x4B408080u);
+        s0 = (sx << 24) >> 24;
+        const int r1 = (sx - s0) >> 8;
+        s1 = (r1 << 24) >> 24;
+        s2 = (r1 - s1) >> 8;
+      }
       const int lane = threadIdx.x & 31;
       if (lane < 2) {
         const int sc = __float_as_int(gmax * (1.0f / kDigitScale));
@@ -354,23 +359,22 @@ __device__ __forceinline__ bool gather_batch(const KParams& p, Item (&raw)[kBatc
 }
 
 struct LoadResult {
-  float xscale;      // int8 / int4: scale of the digit representation
-  float rnorm;       // bf16 weights, normed input: 1/rms, to be applied to the outputs (1 otherwise)
+  float rnorm;       // normed input: 1/rms, to be applied to the outputs (1 otherwise)
   bool bad;
 };
 
-// bf16 and int4 weights: every item is converted as soon as it has arrived.  RMSNorm's 1/rms is one scalar for the
+// Every item is converted as soon as it has arrived.  RMSNorm's 1/rms is one scalar for the
 // whole vector, so W (r * x * g) = r * (W (x * g)): the items go to shared memory as x * g while the sum of squares
 // is still being collected, and r is applied to the outputs in the epilogue -- no second pass over the input and no
-// block-wide reduction between the arrival of the input and the first multiply.  (int4: the digits' scale is per
-// group of 128 elements, like the weights' own, and meets them in the same multiply.)
+// block-wide reduction between the arrival of the input and the first multiply.  (Integer weights: the digits' scale
+// is per group of 128 elements and meets the group's integer sums in one multiply-add, see consume_pass.)
 template <int WD>
 __device__ __forceinline__ LoadResult load_input_1pass(const KParams& p, SmemHeader* sh, unsigned char* xs, int cta, int K,
                                                        const ActPair* src, unsigned seq, int src_task,
                                                        const unsigned short* normw, int task) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n4 = K >> 2;                               // items of four elements
-  LoadResult res{1.0f, 1.0f, false};
+  LoadResult res{1.0f, false};
   Item raw[kBatch];
   // norm weights of my items: requested before the gather, so that their latency (they come from HBM, being
   // read once per token) is not added to the join's (a normed input is one batch per thread)
@@ -383,14 +387,18 @@ __device__ __forceinline__ LoadResult load_input_1pass(const KParams& p, SmemHea
     }
   }
   float ss = 0.f;
+  // (integer weights: the conversion works warp-wide, so a warp stays together through a ragged last group)
+  constexpr int kWhole = (WD == W_BF16) ? 0 : 31;
 #pragma unroll 1
-  for (int i0 = tid; i0 < n4; i0 += kBatch * kConsumerThreads) {
+  for (int i0 = tid; i0 - (lane & kWhole) < n4; i0 += kBatch * kConsumerThreads) {
     res.bad |= gather_batch(p, raw, i0, n4, src, seq, src_task, cta, task);
 #pragma unroll
     for (int i = 0; i < kBatch; i++) {
       const int it = i0 + i * kConsumerThreads;
-      if (it < n4) {
+      if (it - (lane & kWhole) < n4) {
+        const bool valid = it < n4;
         float a[4] = {raw[i].val(0), raw[i].val(1), raw[i].val(2), raw[i].val(3)};
+        if (WD != W_BF16 && !valid) a[0] = a[1] = a[2] = a[3] = 0.f;
         if (normw) {
           ss = fmaf(a[0], a[0], ss);
           ss = fmaf(a[1], a[1], ss);
@@ -401,7 +409,7 @@ __device__ __forceinline__ LoadResult load_input_1pass(const KParams& p, SmemHea
           a[2] *= bf16_lo(gwt[i].y);
           a[3] *= bf16_hi(gwt[i].y);
         }
-        store_item<WD>(xs, n4, it, a);
+        store_item<WD>(xs, n4, it, a, valid);
       }
     }
   }
@@ -417,101 +425,6 @@ __device__ __forceinline__ LoadResult load_input_1pass(const KParams& p, SmemHea
     for (int w = 0; w < kConsumerWarps; w++) tot += sh->warp_part[0][w];
     res.rnorm = rsqrtf(__fdividef(tot, (float)K) + p.eps);       // (2 ulp: the same factor on every output)
   }
-  return res;
-}
-
-// int8 weights (one integer accumulation over the whole row): the input becomes three signed digits of a / scale
-// with one scale, which needs the maximum of the whole (normed) vector first.  A vector short enough for one batch per thread (every normed input) is held in
-// registers across the block reduction; the down projection's long input comes with its producers' maxima.
-template <int WD>
-__device__ __forceinline__ LoadResult load_input(const KParams& p, SmemHeader* sh, unsigned char* xs, int cta, int K,
-                                                 const ActPair* src, unsigned seq, int src_task,
-                                                 const unsigned short* normw, int task, const ActPair* amax_src,
-                                                 int nblk) {
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int n4 = K >> 2;                               // items of four elements
-  LoadResult res{1.0f, 1.0f, false};
-  Item raw[kBatch];
-  const bool held = n4 <= kBatch * kConsumerThreads;
-  float r = 1.0f, inv = 0.f;
-  // `amax_src`: the producers of this (un-normed) input also published the maximum of their part, so the vector
-  // need not be read twice: the first batch is requested, the maxima are combined meanwhile.
-  const bool have_first = held || amax_src != nullptr;
-  {
-    float ss = 0.f, amax = 0.f;
-    if (amax_src) {
-      // the blocks' maxima are requested before the gather (they were published with the values), looked at after
-      uint2 ar = make_uint2(0u, seq);
-      if (tid < nblk) ar = ld_pair(amax_src + tid);
-      res.bad |= gather_batch(p, raw, tid, n4, src, seq, src_task, cta, task);
-      if (tid < nblk && ar.y != seq) {
-        ar = poll_pair_slow(p, amax_src + tid, seq, src_task);
-        if (ar.y != seq) res.bad = true;
-      }
-      amax = fabsf(__uint_as_float(ar.x));
-      for (int b = tid + kConsumerThreads; b < nblk; b += kConsumerThreads)
-        amax = fmaxf(amax, fabsf(read_act(p, res.bad, amax_src + b, seq, src_task)));
-    }
-    // norm weights of my items: requested before the gather (see load_input_bf16)
-    uint2 gwt[kBatch];
-    if (normw) {
-#pragma unroll
-      for (int i = 0; i < kBatch; i++) {
-        const int it = tid + i * kConsumerThreads;
-        gwt[i] = (it < n4) ? __ldg(reinterpret_cast<const uint2*>(normw) + it) : make_uint2(0u, 0u);
-      }
-    }
-#pragma unroll 1
-    for (int i0 = tid; i0 < n4 && !amax_src; i0 += kBatch * kConsumerThreads) {
-      res.bad |= gather_batch(p, raw, i0, n4, src, seq, src_task, cta, task);
-#pragma unroll
-      for (int i = 0; i < kBatch; i++) {
-        const int it = i0 + i * kConsumerThreads;
-        if (it < n4) {
-          float a[4] = {raw[i].val(0), raw[i].val(1), raw[i].val(2), raw[i].val(3)};
-          if (normw) {                                 // (normed inputs are always held)
-            ss = fmaf(a[0], a[0], ss);
-            ss = fmaf(a[1], a[1], ss);
-            ss = fmaf(a[2], a[2], ss);
-            ss = fmaf(a[3], a[3], ss);
-            a[0] *= bf16_lo(gwt[i].x);                 // norm weight now, 1/rms after the sum
-            a[1] *= bf16_hi(gwt[i].x);
-            a[2] *= bf16_lo(gwt[i].y);
-            a[3] *= bf16_hi(gwt[i].y);
-#pragma unroll
-            for (int e = 0; e < 4; e++) raw[i].e[e] = (raw[i].e[e] & 0xffffffff00000000ull) | __float_as_uint(a[e]);
-          }
-          amax = fmaxf(amax, fmaxf(fmaxf(fabsf(a[0]), fabsf(a[1])), fmaxf(fabsf(a[2]), fabsf(a[3]))));
-        }
-      }
-    }
-    if (tid == 0) stamp(p, cta, task, AMK_TR_JOINED);
-    ss = warp_sum_nonneg(ss);
-    amax = warp_max_nonneg(amax);
-    if (lane == 0) { sh->warp_part[0][warp] = ss; sh->warp_part[1][warp] = amax; }
-    res.bad = cons_sync_or(res.bad);
-    float tot = 0.f, mx = 0.f;
-#pragma unroll
-    for (int w = 0; w < kConsumerWarps; w++) { tot += sh->warp_part[0][w]; mx = fmaxf(mx, sh->warp_part[1][w]); }
-    if (normw) r = rsqrtf(__fdividef(tot, (float)K) + p.eps);   // (2 ulp: the same factor on every element)
-    mx *= r;
-    inv = mx > 0.f ? __fdividef(kDigitScale, mx) : 0.f;
-    res.xscale = mx * (1.0f / kDigitScale);
-  }
-  const float rinv = r * inv;
-#pragma unroll 1
-  for (int i0 = tid; i0 < n4; i0 += kBatch * kConsumerThreads) {
-    if (!(have_first && i0 == tid)) res.bad |= gather_batch(p, raw, i0, n4, src, seq, src_task, cta, task);
-#pragma unroll
-    for (int i = 0; i < kBatch; i++) {
-      const int it = i0 + i * kConsumerThreads;
-      if (it < n4) {
-        const float a[4] = {raw[i].val(0), raw[i].val(1), raw[i].val(2), raw[i].val(3)};
-        store_item<WD>(xs, n4, it, a, rinv);
-      }
-    }
-  }
-  res.bad = cons_sync_or(res.bad);
   return res;
 }
 
@@ -533,7 +446,7 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int kind
   const unsigned lane_off = (unsigned)(((c.lane >> 4) * urows + mrow) * 16);   // chunk half h = lane / 16
   const unsigned step_stride = (unsigned)(2 * urows * 16);                     // two chunks per k step
   const int S = p.n_stages;
-  constexpr int BC = (WD == W_INT4) ? 128 : 64;
+  constexpr int BC = grouped(WD) ? 128 : 64;
   // B columns in use: int8 / int4 three digits; bf16 high + low parts
   constexpr int NCOL = (WD == W_BF16) ? 2 : 3;
   const unsigned char* xcol = c.xs + (size_t)min(gq, NCOL - 1) * K * (WD == W_BF16 ? 2 : 1);
@@ -541,8 +454,7 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int kind
   // All fragments of a unit are loaded before its first MMA, and two accumulator sets are used in turn, so
   // that consecutive MMAs do not wait for each other.
   float facc[4] = {0.f, 0.f, 0.f, 0.f}, facc2[4] = {0.f, 0.f, 0.f, 0.f};
-  int iacc[4] = {0, 0, 0, 0}, iacc2[4] = {0, 0, 0, 0};
-  constexpr int NA = (WD == W_BF16) ? 4 : 2;         // ldmatrix.x4 loads per unit
+  constexpr int NA = (WD == W_BF16 || WD == W_INT8G) ? 4 : 2;         // ldmatrix.x4 loads per unit
   unsigned fa[NA][4];                                // pending unit: weight fragments,
   uint4 fx0 = make_uint4(0u, 0u, 0u, 0u), fx1 = fx0; // input fragments,
   unsigned fsz0 = 0u, fsz1 = 0u;                     // int4: {scale, zero} of my two rows,
@@ -554,8 +466,31 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int kind
       mma_bf16(facc, fa[2], fx1.x, fx1.y);
       mma_bf16(facc2, fa[3], fx1.z, fx1.w);
     } else if (WD == W_INT8) {
-      mma_s8(iacc, fa[0][0], fa[0][1], fa[0][2], fa[0][3], fx0.x, fx0.y);
-      mma_s8(iacc2, fa[1][0], fa[1][1], fa[1][2], fa[1][3], fx0.z, fx0.w);
+      // 64 columns of one input group: exact integer sums, then the group's input scale (the row's weight scale
+      // meets the finished sum in the epilogue)
+      int g4[4] = {0, 0, 0, 0}, h4[4] = {0, 0, 0, 0};
+      mma_s8(g4, fa[0][0], fa[0][1], fa[0][2], fa[0][3], fx0.x, fx0.y);
+      mma_s8(h4, fa[1][0], fa[1][1], fa[1][2], fa[1][3], fx0.z, fx0.w);
+      const float xsc = __int_as_float(fsx.z);
+      facc[0] = fmaf(xsc, (float)(g4[0] + h4[0]), facc[0]);
+      facc[1] = fmaf(xsc, (float)(g4[1] + h4[1]), facc[1]);
+      facc[2] = fmaf(xsc, (float)(g4[2] + h4[2]), facc[2]);
+      facc[3] = fmaf(xsc, (float)(g4[3] + h4[3]), facc[3]);
+    } else if (WD == W_INT8G) {
+      // one group of 128 columns: exact integer sums in two chains, then the weights' group scale times the
+      // input's group scale in one multiply-add per accumulator
+      int g4[4] = {0, 0, 0, 0}, h4[4] = {0, 0, 0, 0};
+      mma_s8(g4, fa[0][0], fa[0][1], fa[0][2], fa[0][3], fx0.x, fx0.y);
+      mma_s8(h4, fa[1][0], fa[1][1], fa[1][2], fa[1][3], fx0.z, fx0.w);
+      mma_s8(g4, fa[2][0], fa[2][1], fa[2][2], fa[2][3], fx1.x, fx1.y);
+      mma_s8(h4, fa[3][0], fa[3][1], fa[3][2], fa[3][3], fx1.z, fx1.w);
+      const float xsc = __int_as_float(fsx.z);
+      const float s0 = __half2float(__ushort_as_half((unsigned short)(fsz0 & 0xffffu))) * xsc;
+      const float s1 = __half2float(__ushort_as_half((unsigned short)(fsz1 & 0xffffu))) * xsc;
+      facc[0] = fmaf(s0, (float)(g4[0] + h4[0]), facc[0]);
+      facc[1] = fmaf(s0, (float)(g4[1] + h4[1]), facc[1]);
+      facc[2] = fmaf(s1, (float)(g4[2] + h4[2]), facc[2]);
+      facc[3] = fmaf(s1, (float)(g4[3] + h4[3]), facc[3]);
     } else {
       // sum over k of s (q_k - z) x_k = s (sum q_k x_k - z sum x_k): the codes go to the tensor cores as unsigned
       // bytes, and the zero point meets the sum of the input's digits over the group, which the input's loader
@@ -607,12 +542,13 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int kind
           fx1 = xp[1];
         } else if (WD == W_INT8) {
           fx0 = *reinterpret_cast<const uint4*>(xcol + (size_t)next_b * BC + 16 * q);
+          fsx.z = *reinterpret_cast<const int*>(c.xs + 3 * (size_t)K + 32 * (next_b >> 1) + 8);   // the group's scale
         } else {
           const uint4* xp = reinterpret_cast<const uint4*>(xcol + (size_t)next_b * BC + 32 * q);
           fx0 = xp[0];
           fx1 = xp[1];
           // {scale, zero} of my two fragment rows for this group (= this column block)
-          const unsigned* szp = reinterpret_cast<const unsigned*>(u + urows * 64);
+          const unsigned* szp = reinterpret_cast<const unsigned*>(u + urows * (WD == W_INT4 ? 64 : 128));
           fsz0 = szp[min(gq, urows - 1)];
           fsz1 = szp[min(gq + 8, urows - 1)];
           fsx = *reinterpret_cast<const int4*>(c.xs + 3 * (size_t)K + 32 * next_b + 16 * (q & 1));
@@ -629,7 +565,7 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int kind
     t_r = n_r;
   }
 #pragma unroll
-  for (int e = 0; e < 4; e++) { facc[e] += facc2[e]; iacc[e] += iacc2[e]; }
+  for (int e = 0; e < 4; e++) facc[e] += facc2[e];
   if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_TILES_DONE);
   // per-row result: sum of the B columns in use, with the digit weights for integer inputs
   float y0, y1;
@@ -640,13 +576,8 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int kind
     // columns 2q and 2q+1 of this lane: digit weights 65536 (col 0), 256 (col 1), 1 (col 2), 0 otherwise
     const float w0 = (q == 0) ? 65536.f : (q == 1 ? 1.f : 0.f);
     const float w1 = (q == 0) ? 256.f : 0.f;
-    if (WD == W_INT8) {
-      y0 = w0 * (float)iacc[0] + w1 * (float)iacc[1];
-      y1 = w0 * (float)iacc[2] + w1 * (float)iacc[3];
-    } else {
-      y0 = w0 * facc[0] + w1 * facc[1];
-      y1 = w0 * facc[2] + w1 * facc[3];
-    }
+    y0 = w0 * facc[0] + w1 * facc[1];
+    y1 = w0 * facc[2] + w1 * facc[3];
   }
   y0 += __shfl_xor_sync(0xffffffffu, y0, 1);
   y0 += __shfl_xor_sync(0xffffffffu, y0, 2);
@@ -732,12 +663,8 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind_rt, int l) {
   if (src_task >= 0 && !wait_phase(c, src_task)) return false;
   if (np > 0) {
     const unsigned in_seq = seq_of(p, src_task);
-    LoadResult lr;
-    if (WD != W_INT8) lr = load_input_1pass<WD>(p, c.sh, c.xs, c.cta, K, src, in_seq, src_task, normw, task);
-    else lr = load_input<WD>(p, c.sh, c.xs, c.cta, K, src, in_seq, src_task, normw, task,
-                             kind == OP_DOWN ? p.m_amax : nullptr, c.nblk);
+    const LoadResult lr = load_input_1pass<WD>(p, c.sh, c.xs, c.cta, K, src, in_seq, src_task, normw, task);
     rnorm = lr.rnorm;
-    c.xscale = lr.xscale;
     c.bad = lr.bad;
     if (c.bad) return false;
   }
@@ -747,7 +674,6 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind_rt, int l) {
   float best_val = -CUDART_INF_F;
   int best_idx = 0x7fffffff;
   const bool drop = dropped(p, task, c.cta);
-  float gu_amax = 0.f;                                // gate/up of an integer-weight model: max |output| of this block
   for (int ps = 0; ps < np; ps++) {
     const int R = pass_rows(sl.rows, ps);
     const int gw = (ps == np - 1) ? 1 : 0;             // which precomputed geometry: a full pass or the last one
@@ -770,7 +696,6 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind_rt, int l) {
     }
     const float resid = __uint_as_float(rraw.x);
     float sc0 = __half2float(sh0) * rnorm, sc1 = __half2float(sh1) * rnorm;
-    if (d.wdtype == W_INT8) { sc0 *= c.xscale; sc1 *= c.xscale; }
     c.bad = cons_sync_or(c.bad);
     if (c.bad) return false;
 
@@ -786,7 +711,6 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind_rt, int l) {
         up *= sc1;
         const float mv = silu_f(gt) * up;
         st_pair(p.m + (vrow0 >> 1) + c.tid, mv, my_seq);
-        gu_amax = fmaxf(gu_amax, fabsf(mv));
       } else {
         float y = 0.f;
         for (int k = 0; k < g.Wk; k++) y += red[k * R + c.tid];
@@ -828,19 +752,6 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind_rt, int l) {
             break;
         }
       }
-    }
-  }
-  if (WD == W_INT8 && kind == OP_GATEUP) {
-    // publish this block's max |m|: the down projection scales its integer input by the maximum over all blocks
-    gu_amax = warp_max_nonneg(gu_amax);
-    if (c.lane == 0) c.sh->cand_val[c.warp] = gu_amax;
-    c.bad = cons_sync_or(c.bad);
-    if (c.bad) return false;
-    if (c.tid == 0 && !drop) {
-      float mx = 0.f;
-#pragma unroll
-      for (int w = 0; w < kConsumerWarps; w++) mx = fmaxf(mx, c.sh->cand_val[w]);
-      st_pair(p.m_amax + c.cta, mx, my_seq);
     }
   }
   if (c.tid == 0) stamp(p, c.cta, task, AMK_TR_COMPUTED);
@@ -1513,7 +1424,7 @@ template <int WD>
 __device__ __noinline__ void lm_head_task(const KParams& p, SmemHeader* sh, unsigned char* xs, unsigned char* ring,
                                           int cta, int nblk, int stage, unsigned parity, int token) {
   const int tid = threadIdx.x;
-  Ctx c{p, sh, xs, ring, tid, tid >> 5, tid & 31, cta, nblk, stage, parity, token, 1.0f, false};
+  Ctx c{p, sh, xs, ring, tid, tid >> 5, tid & 31, cta, nblk, stage, parity, token, false};
   gemv_op<WD, true>(c, (int)OP_LMHEAD, p.L);
 }
 
@@ -1700,7 +1611,7 @@ __global__ void __launch_bounds__(kThreads, 1) AMK_KERNEL(const __grid_constant_
       if (p.flags & AMK_FLAG_DEBUG_HIDDEN) p.hidden[e] = v;
     }
   }
-  Ctx c{p, sh, xs, ring, tid, warp, lane, cta, nblk, 0, 0u, token, 1.0f, false};
+  Ctx c{p, sh, xs, ring, tid, warp, lane, cta, nblk, 0, 0u, token, false};
   // the block's queue: tasks 5 l + {0..4} = QKV, attention, O, gate/up, down of layer l, then the LM head
   // (one call site each, so that the per-thread state stays in registers)
   const int n_layer_tasks = 5 * p.L;
@@ -1791,10 +1702,12 @@ static DecodeKernel pick_kernel(int wdtype, int hd) {
   if (hd == 64) {
     if (wdtype == W_BF16) return AMK_KERNEL<W_BF16, 64>;
     if (wdtype == W_INT8) return AMK_KERNEL<W_INT8, 64>;
+    if (wdtype == W_INT8G) return AMK_KERNEL<W_INT8G, 64>;
     return AMK_KERNEL<W_INT4, 64>;
   }
   if (wdtype == W_BF16) return AMK_KERNEL<W_BF16, 128>;
   if (wdtype == W_INT8) return AMK_KERNEL<W_INT8, 128>;
+  if (wdtype == W_INT8G) return AMK_KERNEL<W_INT8G, 128>;
   return AMK_KERNEL<W_INT4, 128>;
 }
 

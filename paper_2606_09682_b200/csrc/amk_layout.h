@@ -4,7 +4,7 @@
 // `slot` owns a contiguous run of "units" (1 row, or 2 rows where rows must stay together).  Inside a
 // block the rows are processed in passes of at most kPassRows rows.  In a pass the consumer warps form
 // a Wr x Wk grid: row-warp wr owns G <= 16 consecutive rows (one m16 tensor-core tile), k-warp wk owns
-// every Wk-th column block (64 columns; 128 for int4 = one quantisation group).  The bytes of a pass are
+// every Wk-th column block (64 columns; 128 for int4 and grouped int8 = one quantisation group).  The bytes of a pass are
 // stored block-major: for column block b, the work units (b, wr = 0..Wr-1) one after another.  A work
 // unit -- the rows of one row-warp in one column block -- is contiguous, and a ring tile is a run of
 // `upt` consecutive units, so each block's weight stream is a sequence of contiguous byte runs that one
@@ -14,8 +14,8 @@
 // along K) of row r sits at (c * rows + r) * 16, so the eight rows of an 8x8 matrix are 128 contiguous
 // bytes (no bank conflicts).  The k order inside a block is permuted (col_of_k) so that the activation
 // values one lane feeds to the tensor core -- its B fragments for every k step of the block -- are
-// contiguous in the natural column order.  An int4 unit ends with fp16 {scale, zero} per row (its block
-// is one group).
+// contiguous in the natural column order.  An int4 / grouped-int8 unit ends with {fp16 scale, 16-bit zero point
+// (0 for grouped int8)} per row (its block is one group).
 #pragma once
 #include <stdint.h>
 
@@ -38,16 +38,18 @@ constexpr int kAttnMinChunk = 32;             // fewest cache positions per spli
 constexpr int kMaxChunks = 64;
 
 enum OpKind : int { OP_QKV = 0, OP_O = 1, OP_GATEUP = 2, OP_DOWN = 3, OP_LMHEAD = 4 };
-enum WDtype : int { W_BF16 = 0, W_INT8 = 1, W_INT4 = 2 };
+enum WDtype : int { W_BF16 = 0, W_INT8 = 1, W_INT4 = 2, W_INT8G = 3 };
+AMK_HD constexpr bool grouped(int wdtype) { return wdtype == W_INT4 || wdtype == W_INT8G; }   // scales inside the units
 
 AMK_HD int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
-AMK_HD int block_cols(int wdtype) { return wdtype == W_INT4 ? 128 : 64; }        // columns per column block
-AMK_HD int block_chunks(int wdtype) { return wdtype == W_BF16 ? 8 : 4; }          // 16-byte chunks per row per block
-// bytes of a work unit holding `rows` rows (int4: codes, then 4 bytes {scale, zero} per row, padded to 16)
+AMK_HD int block_cols(int wdtype) { return grouped(wdtype) ? 128 : 64; }          // columns per column block
+AMK_HD int block_chunks(int wdtype) { return (wdtype == W_BF16 || wdtype == W_INT8G) ? 8 : 4; }   // 16-byte chunks per row per block
+// bytes of a work unit holding `rows` rows (grouped: codes, then 4 bytes {scale, zero} per row, padded to 16)
 AMK_HD int unit_bytes(int wdtype, int rows) {
   if (wdtype == W_BF16) return rows * 128;
   if (wdtype == W_INT8) return rows * 64;
+  if (wdtype == W_INT8G) return (rows * 132 + 15) & ~15;
   return (rows * 68 + 15) & ~15;
 }
 
@@ -57,7 +59,7 @@ AMK_HD int unit_bytes(int wdtype, int rows) {
 // q * (block_cols / 4).
 //   bf16: k = 16 s + 8 h + 2 q + j  (s<4, h<2, q<4, j<2)  ->  col 16 q + 4 s + 2 h + j
 //   int8: k = 32 s + 16 h + 4 q + j (s<2, h<2, q<4, j<4)  ->  col 16 q + 8 s + 4 h + j
-//   int4: k = 32 s + 16 h + 4 q + j (s<4, h<2, q<4, j<4)  ->  col 32 q + 8 s + 4 h + j
+//   int4, grouped int8: k = 32 s + 16 h + 4 q + j (s<4, h<2, q<4, j<4)  ->  col 32 q + 8 s + 4 h + j
 AMK_HD int col_of_k(int wdtype, int k) {
   if (wdtype == W_BF16) {
     const int s = k >> 4, h = (k >> 3) & 1, q = (k >> 1) & 3, j = k & 1;
@@ -69,11 +71,11 @@ AMK_HD int col_of_k(int wdtype, int k) {
 
 // Where logical k of a row is stored inside its unit: the 16-byte chunk, and the element inside the chunk
 // (bf16: 2-byte element; int8: byte; int4: nibble, low nibble of a byte first).
-//   bf16 / int8: k-major.   int4: one ldmatrix word (8 nibbles) of chunk 2 (s >> 1) + h expands into the
+//   bf16 / int8 / grouped int8: k-major.   int4: one ldmatrix word (8 nibbles) of chunk 2 (s >> 1) + h expands into the
 //   fragment registers of k steps s = 2x (even nibbles) and s = 2x + 1 (odd nibbles).
 AMK_HD void place_of_k(int wdtype, int k, int* chunk, int* elem) {
   if (wdtype == W_BF16) { *chunk = k >> 3; *elem = k & 7; return; }
-  if (wdtype == W_INT8) { *chunk = k >> 4; *elem = k & 15; return; }
+  if (wdtype == W_INT8 || wdtype == W_INT8G) { *chunk = k >> 4; *elem = k & 15; return; }
   const int s = k >> 5, h = (k >> 4) & 1, q = (k >> 2) & 3, j = k & 3;
   *chunk = 2 * (s >> 1) + h;
   *elem = 8 * q + 2 * j + (s & 1);

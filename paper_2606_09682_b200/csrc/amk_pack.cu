@@ -12,7 +12,7 @@ namespace {
 
 struct RowSrc {
   unsigned char* w;             // row start in the canonical matrix (nullptr: this row is not wanted)
-  unsigned short* scale;        // int8: &scale[row]; int4: &scale[row][0]
+  unsigned short* scale;        // int8: &scale[row]; int4, grouped int8: &scale[row][0]
   unsigned short* zero;         // int4: &zero[row][0]
 };
 
@@ -27,15 +27,15 @@ __device__ __forceinline__ RowSrc row_source(const OpShape& d, const PackSrc& s,
     row = vrow >> 1;
   }
   const size_t K = (size_t)d.K;
-  const size_t rowb = d.wdtype == W_BF16 ? K * 2 : (d.wdtype == W_INT8 ? K : K / 2);
+  const size_t rowb = d.wdtype == W_BF16 ? K * 2 : (d.wdtype == W_INT4 ? K / 2 : K);
   RowSrc r;
   r.w = s.w[which] ? (unsigned char*)s.w[which] + (size_t)row * rowb : nullptr;
   r.scale = nullptr;
   r.zero = nullptr;
   if (d.wdtype == W_INT8 && s.scale[which]) r.scale = (unsigned short*)s.scale[which] + row;
-  if (d.wdtype == W_INT4) {
+  if (grouped(d.wdtype)) {
     if (s.scale[which]) r.scale = (unsigned short*)s.scale[which] + (size_t)row * (K / 128);
-    if (s.zero[which]) r.zero = (unsigned short*)s.zero[which] + (size_t)row * (K / 128);
+    if (d.wdtype == W_INT4 && s.zero[which]) r.zero = (unsigned short*)s.zero[which] + (size_t)row * (K / 128);
   }
   return r;
 }
@@ -82,18 +82,25 @@ __global__ void pack_kernel(const PackOp d, const PackSrc s, unsigned char* pack
         else w32[col >> 1] = v[q];
       }
       if (!inverse) *chunk = make_uint4(v[0], v[1], v[2], v[3]);
-    } else if (wd == W_INT8) {
-      // chunk c = 2 s + hh holds logical k = 32 s + 16 hh + 4 q + j: for q = 0..3 the word at column 16 q + 8 s + 4 hh
-      const int sidx = c >> 1, hh = c & 1;
+    } else if (wd == W_INT8 || wd == W_INT8G) {
+      // chunk c = 2 s + hh holds logical k = 32 s + 16 hh + 4 q + j: for q = 0..3 the word at column
+      // (16 | 32 grouped) q + 8 s + 4 hh
+      const int sidx = c >> 1, hh = c & 1, qs = (wd == W_INT8) ? 16 : 32;
       unsigned* w32 = reinterpret_cast<unsigned*>(src.w);
       unsigned v[4];
       if (inverse) { const uint4 t = *chunk; v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w; }
       for (int q = 0; q < 4; q++) {
-        const int col = col0 + 16 * q + 8 * sidx + 4 * hh;
+        const int col = col0 + qs * q + 8 * sidx + 4 * hh;
         if (!inverse) v[q] = w32[col >> 2];
         else w32[col >> 2] = v[q];
       }
       if (!inverse) *chunk = make_uint4(v[0], v[1], v[2], v[3]);
+      if (wd == W_INT8G && c == 0) {
+        // {fp16 scale, 0} of this row's group (= this block) after the unit's code bytes
+        unsigned* sz = reinterpret_cast<unsigned*>(unit + (size_t)urows * 128 + (size_t)gi * 4);
+        if (!inverse) { if (src.scale) *sz = (unsigned)src.scale[b]; }
+        else if (src.scale) src.scale[b] = (unsigned short)(*sz & 0xffffu);
+      }
     } else {
       // chunk c = 2 x + hh; word q, nibble 2 j + sb holds logical k of step s = 2 x + sb: column 32 q + 8 s + 4 hh + j
       const int x = c >> 1, hh = c & 1;
@@ -172,6 +179,33 @@ __global__ void quantize_int8_kernel(const unsigned short* __restrict__ w, int64
   }
 }
 
+// grouped int8: one warp per (row, group of 128), the per-row rule on the group; lane handles 4 consecutive columns
+__global__ void quantize_int8_grouped_kernel(const unsigned short* __restrict__ w, int64_t rows, int64_t cols,
+                                             signed char* __restrict__ q, __half* __restrict__ scale) {
+  const int64_t ng = cols / 128;
+  const int64_t wid = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (wid >= rows * ng) return;
+  const int lane = threadIdx.x & 31;
+  const int64_t row = wid / ng, g = wid - row * ng;
+  const unsigned short* wp = w + row * cols + g * 128 + lane * 4;
+  float v[4];
+  float amax = 0.f;
+#pragma unroll
+  for (int e = 0; e < 4; e++) { v[e] = bf16_at(wp, e); amax = fmaxf(amax, fabsf(v[e])); }
+  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+  __half h = (amax == 0.f) ? __float2half_rn(1.0f) : __float2half_rn(__fdiv_rn(amax, 127.0f));
+  float s = __half2float(h);
+  if (s == 0.f) { h = __float2half_rn(1.0f); s = 1.0f; }
+  signed char* out = q + row * cols + g * 128 + lane * 4;
+#pragma unroll
+  for (int e = 0; e < 4; e++) {
+    float r = rintf(__fdiv_rn(v[e], s));
+    r = fminf(fmaxf(r, -127.0f), 127.0f);
+    out[e] = (signed char)(int)r;
+  }
+  if (lane == 0) scale[row * ng + g] = h;
+}
+
 // one warp per (row, group of 128): lane handles 4 consecutive columns = 2 output bytes
 __global__ void quantize_int4_kernel(const unsigned short* __restrict__ w, int64_t rows, int64_t cols,
                                      unsigned char* __restrict__ packed, __half* __restrict__ scale,
@@ -221,6 +255,15 @@ cudaError_t launch_pack(const PackOp& d, const PackSrc& src, unsigned char* pack
 cudaError_t launch_quantize_int8(const void* w, int64_t rows, int64_t cols, void* q, void* scale, cudaStream_t s) {
   if (rows <= 0) return cudaSuccess;
   quantize_int8_kernel<<<(unsigned)rows, 256, 0, s>>>((const unsigned short*)w, cols, (signed char*)q, (__half*)scale);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_quantize_int8_grouped(const void* w, int64_t rows, int64_t cols, void* q, void* scale, cudaStream_t s) {
+  if (rows <= 0) return cudaSuccess;
+  const int64_t warps = rows * (cols / 128);
+  const int wpb = 8;
+  quantize_int8_grouped_kernel<<<(unsigned)((warps + wpb - 1) / wpb), wpb * 32, 0, s>>>(
+      (const unsigned short*)w, rows, cols, (signed char*)q, (__half*)scale);
   return cudaGetLastError();
 }
 

@@ -165,6 +165,8 @@ def streamed_bytes(shape: ModelShape, wdtype: str = "bf16", pos: int = 0, group:
         wl, sc = 1.0 * lin, 2.0 * rows
     elif wdtype == "int4":
         wl, sc = 0.5 * lin, 4.0 * lin / group
+    elif wdtype == "int8g":                                          # grouped int8: {fp16 scale, pad} per row and group
+        wl, sc = 1.0 * lin, 4.0 * lin / group
     else:
         raise ValueError(wdtype)
     head, head_sc = 2.0 * V * H, 0.0
@@ -172,6 +174,8 @@ def streamed_bytes(shape: ModelShape, wdtype: str = "bf16", pos: int = 0, group:
         head, head_sc = 1.0 * V * H, 2.0 * V
     elif quantize_lm_head and wdtype == "int4":
         head, head_sc = 0.5 * V * H, 4.0 * V * H / group
+    elif quantize_lm_head and wdtype == "int8g":
+        head, head_sc = 1.0 * V * H, 4.0 * V * H / group
     weights = L * wl + head + 2.0 * (2 * L + 1) * H + 2.0 * H            # linears + LM head + norms + one embedding row
     scales = L * sc + head_sc
     kv = 2.0 * L * nkv * hd * 2 * pos + 2.0 * L * nkv * hd * 2

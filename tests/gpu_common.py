@@ -9,7 +9,7 @@ from paper_2606_09682_b200 import inputs as inp
 HIDDEN_TOL = 5e-3      # rel-L2 per layer hidden state
 LOGITS_TOL = 1e-2      # rel-L2 on logits
 ARGMAX_GAP = 1e-2      # the greedy token must match bit-exactly when the oracle's top-2 gap exceeds this
-WD = {"bf16": orc.W_BF16, "int8": orc.W_INT8, "int4": orc.W_INT4}
+WD = {"bf16": orc.W_BF16, "int8": orc.W_INT8, "int4": orc.W_INT4, "int8g": orc.W_INT8G}
 LAST = {}                # the last compared step's raw outputs, for callers that need them
 
 

@@ -102,14 +102,14 @@ int main(int argc, char** argv) {
               for (int k = 0; k < bc; k++) {
                 int ch, el;
                 place_of_k(wd, k, &ch, &el);
-                const long long byte = uo + ((long long)ch * urows + i) * 16 + (wd == W_BF16 ? el * 2 : (wd == W_INT8 ? el : el / 2));
+                const long long byte = uo + ((long long)ch * urows + i) * 16 + (wd == W_BF16 ? el * 2 : (wd == W_INT4 ? el / 2 : el));
                 if (byte >= (long long)mark.size()) { printf("element outside the pass\n"); return 1; }
                 mark[byte] = 1;
                 if (wd == W_BF16) mark[byte + 1] = 1;
                 seen[(size_t)row * K + (size_t)next_b * bc + col_of_k(wd, k)]++;
               }
-              if (wd == W_INT4) {
-                const long long sz = uo + (long long)urows * 64 + i * 4;
+              if (grouped(wd)) {
+                const long long sz = uo + (long long)urows * (wd == W_INT4 ? 64 : 128) + i * 4;
                 for (int e = 0; e < 4; e++) mark[sz + e] = 1;
               }
             }
@@ -123,7 +123,7 @@ int main(int argc, char** argv) {
       // every byte except unit padding is used
       long long used = 0;
       for (unsigned char m : mark) used += m;
-      const long long expect = (long long)R * g.nblk * (wd == W_BF16 ? 128 : (wd == W_INT8 ? 64 : 68));
+      const long long expect = (long long)R * g.nblk * (wd == W_BF16 ? 128 : (wd == W_INT8 ? 64 : (wd == W_INT4 ? 68 : 132)));
       if (used != expect) { printf("bytes used %lld, expected %lld\n", used, expect); return 1; }
       sbytes += pass_bytes(g);
     }

@@ -61,9 +61,9 @@ def test_struct_mirror_matches_header(amk, tmp_path):
 def test_size_queries_and_argument_checks(amk):
     for name in ("smollm2_135m", "tinyllama_1b", "llama3_8b"):
         s = inp.SHAPES[name]
-        for wd in ("bf16", "int8", "int4"):
+        for wd in ("bf16", "int8", "int4", "int8g"):
             cfg = amk.make_config(s, wd)
-            if wd == "int4" and name == "smollm2_135m":       # hidden 576 is not a multiple of the group size 128
+            if wd in ("int4", "int8g") and name == "smollm2_135m":       # hidden 576 is not a multiple of the group size 128
                 with pytest.raises(amk.AmkError) as e:
                     amk.amk_packed_bytes(cfg)
                 assert e.value.code == amk.AMK_ERR_UNSUPPORTED
@@ -72,7 +72,7 @@ def test_size_queries_and_argument_checks(amk):
             b = inp.streamed_bytes(s, wd, 0)
             # packed buffer = streamed weights and scales + a canonical embedding copy (+ alignment padding)
             expect = b["weights"] + b["scales"] - 2.0 * s.hidden + 2.0 * s.vocab * s.hidden
-            slack = 0.02 if wd == "int4" else 1e-3        # int4 work units are padded to 16 bytes
+            slack = 0.02 if wd in ("int4", "int8g") else 1e-3        # units with scales inside are padded to 16 bytes
             assert 0 <= pb - expect < slack * expect + 1e6, (name, wd, pb, expect)
             assert amk.amk_kv_bytes(cfg) == 2 * s.n_layers * s.n_kv_heads * s.max_seq * s.head_dim * 2
             assert amk.amk_workspace_bytes(cfg) > 0
@@ -129,6 +129,7 @@ def layout_check(tmp_path_factory):
     (960, 576, 0, 1, 148), (3072, 576, 0, 2, 148), (576, 1536, 0, 1, 148),                                  # SmolLM2 shape
     (6144, 4096, 1, 1, 148), (28672, 4096, 1, 2, 148), (4096, 14336, 1, 1, 148),                            # Llama-3-8B int8
     (2560, 2048, 2, 1, 148), (11264, 2048, 2, 2, 148), (2048, 5632, 2, 1, 148),                             # TinyLlama int4
+    (2560, 2048, 3, 1, 148), (11264, 2048, 3, 2, 148), (2048, 5632, 3, 1, 148), (300, 384, 3, 1, 132),      # grouped int8
     (1003, 192, 0, 1, 148), (7, 64, 0, 1, 148), (300, 320, 1, 1, 132), (5000, 1024, 0, 1, 7),               # odd cases
     (128256, 4096, 0, 1, 148), (49152, 576, 0, 1, 148),                                                     # LM heads
 ])

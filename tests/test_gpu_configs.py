@@ -101,7 +101,8 @@ def test_smollm2_shape_256_greedy_steps(amk):
     dec.close()
 
 
-@pytest.mark.parametrize("wdtype,pos", [("bf16", 0), ("bf16", 1024), ("int8", 0), ("int8", 512), ("int4", 0), ("int4", 512)])
+@pytest.mark.parametrize("wdtype,pos", [("bf16", 0), ("bf16", 1024), ("int8", 0), ("int8", 512), ("int4", 0), ("int4", 512),
+                                        ("int8g", 0), ("int8g", 300)])
 def test_tinyllama_shape(amk, wdtype, pos):
     shape, w, _, dec = _build(amk, "tinyllama_1b", wdtype, 0xA3C2)
     model, _ = gc.oracle_model(shape, w, wdtype)
@@ -112,7 +113,7 @@ def test_tinyllama_shape(amk, wdtype, pos):
     dec.close()
 
 
-@pytest.mark.parametrize("wdtype,pos", [("int8", 0), ("int4", 200)])
+@pytest.mark.parametrize("wdtype,pos", [("int8", 0), ("int4", 200), ("int8g", 0)])
 def test_tinyllama_shape_quantised_lm_head(amk, wdtype, pos):
     shape, w, _, dec = _build(amk, "tinyllama_1b", wdtype, 0xA3C2, quantize_lm_head=True)
     model, _ = gc.oracle_model(shape, w, wdtype, quantize_lm_head=True)
@@ -147,7 +148,8 @@ def test_llama32_1b_shape(amk, wdtype, pos):
     dec.close()
 
 
-@pytest.mark.parametrize("wdtype,pos", [("bf16", 0), ("bf16", 4096), ("int8", 0), ("int8", 4096), ("int4", 0), ("int4", 2500)])
+@pytest.mark.parametrize("wdtype,pos", [("bf16", 0), ("bf16", 4096), ("int8", 0), ("int8", 4096), ("int4", 0), ("int4", 2500),
+                                        ("int8g", 0)])
 def test_llama3_8b_shape_whole_step_layer_by_layer(amk, wdtype, pos):
     shape, w, wq, dec = _build(amk, "llama3_8b", wdtype, 0xA3C4)
     kv_g = inp.make_kv_prefill(shape, 0xA3C4, pos, device="cuda")

@@ -27,6 +27,7 @@ def _setup(name, wdtype, seed, std=0.05, norm_jitter=0.1, quantize_lm_head=False
     ("mini", "bf16"), ("mini_ragged", "bf16"), ("mini_hd128", "bf16"), ("mini_wide", "bf16"),
     ("mini", "int8"), ("mini_ragged", "int8"), ("mini_hd128", "int8"),
     ("mini", "int4"), ("mini_hd128", "int4"), ("mini_wide", "int4"),
+    ("mini", "int8g"), ("mini_hd128", "int8g"), ("mini_wide", "int8g"),
 ])
 def test_multi_step_decode_matches_oracle(name, wdtype):
     shape, dec, model = _setup(name, wdtype, seed=21)
@@ -43,7 +44,7 @@ def test_multi_step_decode_matches_oracle(name, wdtype):
 
 
 @pytest.mark.parametrize("name,wdtype", [("mini", "int8"), ("mini_ragged", "int8"), ("mini_wide", "int4"),
-                                         ("mini_hd128", "int4")])
+                                         ("mini_hd128", "int4"), ("mini_wide", "int8g")])
 def test_quantised_lm_head(name, wdtype):
     """quantize_lm_head = 1: the LM head GEMV streams codes quantised like the layers (a quantised copy of the
     embedding matrix for the tied mini_ragged shape), against the oracle with the same reading switched on."""
@@ -70,7 +71,8 @@ def test_prefilled_cache_split_k(name, pos):
     dec.close()
 
 
-@pytest.mark.parametrize("name,wdtype", [("mini", "bf16"), ("mini_hd128", "int8"), ("mini_ragged", "bf16"), ("mini_wide", "int4")])
+@pytest.mark.parametrize("name,wdtype", [("mini", "bf16"), ("mini_hd128", "int8"), ("mini_ragged", "bf16"), ("mini_wide", "int4"),
+                                         ("mini_hd128", "int8g")])
 def test_chunk_boundaries_and_last_position(name, wdtype):
     """Positions around the 32-position chunk boundary -- a last chunk that holds nothing but the new row
     (pos = 32, 64), chunks that end exactly at the boundary (pos = 31, 63), one position only in the cache

@@ -38,6 +38,10 @@ def test_quantisers_bit_exact_against_oracle(amk, rows, cols):
     qo, so = orc.quantize_int8(wb)
     assert np.array_equal(q.cpu().numpy(), qo)
     assert np.array_equal(inp.bits(s), so)
+    qg, sg = amk.amk_quantize_int8_grouped(w)
+    qgo, sgo = orc.quantize_int8_grouped(wb, 128)
+    assert np.array_equal(qg.cpu().numpy(), qgo)
+    assert np.array_equal(inp.bits(sg), sgo)
     p, s4, z4 = amk.amk_quantize_int4(w)
     po, s4o, z4o = orc.quantize_int4(wb, 128)
     assert np.array_equal(p.cpu().numpy(), po)
@@ -46,7 +50,8 @@ def test_quantisers_bit_exact_against_oracle(amk, rows, cols):
 
 
 @pytest.mark.parametrize("name,wdtype", [("mini_wide", "bf16"), ("mini_ragged", "bf16"), ("mini_wide", "int8"),
-                                         ("mini_ragged", "int8"), ("mini_wide", "int4"), ("mini_hd128", "int4")])
+                                         ("mini_ragged", "int8"), ("mini_wide", "int4"), ("mini_hd128", "int4"),
+                                         ("mini_wide", "int8g"), ("mini_hd128", "int8g")])
 def test_packed_layout_unpacks_bit_exact(amk, name, wdtype):
     shape = inp.SHAPES[name]
     w = inp.make_weights(shape, 41, device="cuda")

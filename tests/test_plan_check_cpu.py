@@ -11,10 +11,12 @@ from oracle import plan_oracle
 from paper_2606_09682_b200 import binding as amk
 from paper_2606_09682_b200 import inputs as inp
 
-WD = {"bf16": 0, "int8": 1, "int4": 2}
+WD = {"bf16": 0, "int8": 1, "int4": 2, "int8g": 3}
 CASES = [("mini", "bf16", 148), ("mini_ragged", "int8", 132), ("mini_hd128", "int4", 7), ("mini_wide", "int4", 148),
-         ("tinyllama_1b", "int8", 148), ("smollm2_135m", "bf16", 148), ("llama3_8b", "bf16", 148)]
-QHEAD_CASES = [("mini_ragged", "int8", 132), ("mini_wide", "int4", 148), ("tinyllama_1b", "int8", 148)]
+         ("tinyllama_1b", "int8", 148), ("smollm2_135m", "bf16", 148), ("llama3_8b", "bf16", 148),
+         ("mini_wide", "int8g", 148), ("tinyllama_1b", "int8g", 148)]
+QHEAD_CASES = [("mini_ragged", "int8", 132), ("mini_wide", "int4", 148), ("tinyllama_1b", "int8", 148),
+               ("mini_hd128", "int8g", 148)]
 
 
 def _plan(name, wdtype, n_blocks, **kw):
