@@ -25,11 +25,12 @@ def _cdiv(a, b):
 
 
 def _unit_bytes(wd, rows):
-    """A work unit = the rows of one row-warp over one column block (64 columns; 128 for int4 and grouped int8)."""
+    """A work unit = the rows of one row-warp over one column block (64 columns for bf16; 128 for the integer dtypes,
+    an int8 matrix's last block zero-filled when K is 64 short of a multiple of 128)."""
     if wd == 0:
         return rows * 128                      # 64 bf16
     if wd == 1:
-        return rows * 64                       # 64 int8
+        return rows * 128                      # 128 int8
     if wd == 3:
         return (rows * 132 + 15) // 16 * 16    # 128 int8 + {fp16 scale, pad} per row, padded to 16 bytes
     return (rows * 68 + 15) // 16 * 16         # 128 nibbles + {scale, zero} fp16 per row, padded to 16 bytes
@@ -45,7 +46,7 @@ def _pass_tiles(rows, k, wd, stage):
     g = _cdiv(rows, wr)
     wr = _cdiv(rows, g)
     g_last = rows - (wr - 1) * g
-    nblk = k // (128 if wd in (2, 3) else 64)
+    nblk = _cdiv(k, 64 if wd == 0 else 128)
     ub, ubl = _unit_bytes(wd, g), _unit_bytes(wd, g_last)
     block_bytes = (wr - 1) * ub + ubl
     n_units = wr * nblk

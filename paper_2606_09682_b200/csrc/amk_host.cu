@@ -426,8 +426,9 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     const size_t hdr = (sizeof(SmemHeader) + 127) & ~(size_t)127;
     size_t kmax = (size_t)(H > I ? H : I);
     if ((size_t)qd > kmax) kmax = qd;
-    size_t act = kmax * (cfg->wdtype == AMK_W_BF16 ? 4 : 3);   // bf16 high + low halves, or three int8 digits
-    if (cfg->wdtype != AMK_W_BF16) act += (kmax + 127) / 128 * 32;   // + 32 bytes per group of 128: digit sums and scale
+    size_t act = kmax * 4;                                     // bf16 high + low halves
+    if (cfg->wdtype != AMK_W_BF16)                             // or three int8 digit columns of whole groups of 128
+      act = (kmax + 127) / 128 * (3 * 128 + 32);               //   + 32 bytes per group: digit sums and scale
     if (!cfg->quantize_lm_head && (size_t)H * 4 > act) act = (size_t)H * 4;   // a bf16 LM head in an integer model
     // attention scratch: q vectors, per-warp partial outputs, the new K / V rows, the scores of the longest chunk
     int lc_max = 0, c_max = 0;

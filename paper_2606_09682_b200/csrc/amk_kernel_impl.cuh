@@ -250,10 +250,11 @@ __device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi) {      // {b
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
 }
-// (integer weights: called by whole warps -- the warp's 32 items are one group of 128 elements sharing a scale;
-//  `valid` is false for the lanes beyond the end of a vector whose length is not a multiple of 128, which pass zeros)
+// (integer weights: called by whole warps -- the warp's 32 items are one group of 128 elements sharing a scale; the
+//  lanes beyond the end of a vector whose length is not a multiple of 128 pass zeros.)
+//  `n4`: items per column (integer weights: of the column length rounded up to whole groups, the tail zero).
 template <int WD>
-__device__ __forceinline__ void store_item(unsigned char* xs, int n4, int it, const float (&a)[4], bool valid = true) {
+__device__ __forceinline__ void store_item(unsigned char* xs, int n4, int it, const float (&a)[4]) {
   if (WD == W_BF16) {
     // two B columns: bf16(a) and bf16(a - bf16(a)); their sum is a to 2^-17 (a third column would make it exact
     // and measured 1.3 % slower at the TinyLlama shape for an error far below the others')
@@ -276,11 +277,9 @@ __device__ __forceinline__ void store_item(unsigned char* xs, int n4, int it, co
     const unsigned w0 = __byte_perm(p01, p23, 0x5410) ^ 0x80808080u;
     const unsigned w1 = __byte_perm(p01, p23, 0x7632) ^ 0x80808080u;
     const unsigned w2 = (__byte_perm(__byte_perm(t[0], t[1], 0x0062), __byte_perm(t[2], t[3], 0x0062), 0x5410) + 0x40404040u) ^ 0x80808080u;
-    if (valid) {
-      D2[2 * n4 + it] = w0;
-      D2[n4 + it] = w1;
-      D2[it] = w2;
-    }
+    D2[2 * n4 + it] = w0;
+    D2[n4 + it] = w1;
+    D2[it] = w2;
     {
       // The group's entry of the table behind the digit columns, laid out by accumulator column pair:
       // {A2, A1, scale, -} {A0, 0, scale, -}.  int4: the zero point of a weight group meets the sum of the input's
@@ -374,6 +373,7 @@ __device__ __forceinline__ LoadResult load_input_1pass(const KParams& p, SmemHea
                                                        const unsigned short* normw, int task) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n4 = K >> 2;                               // items of four elements
+  const int n4s = (WD == W_BF16) ? n4 : ((n4 + 31) & ~31);   // items per shared-memory column (whole groups)
   LoadResult res{1.0f, false};
   Item raw[kBatch];
   // norm weights of my items: requested before the gather, so that their latency (they come from HBM, being
@@ -409,7 +409,7 @@ __device__ __forceinline__ LoadResult load_input_1pass(const KParams& p, SmemHea
           a[2] *= bf16_lo(gwt[i].y);
           a[3] *= bf16_hi(gwt[i].y);
         }
-        store_item<WD>(xs, n4, it, a, valid);
+        store_item<WD>(xs, n4s, it, a);
       }
     }
   }
@@ -446,15 +446,16 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int kind
   const unsigned lane_off = (unsigned)(((c.lane >> 4) * urows + mrow) * 16);   // chunk half h = lane / 16
   const unsigned step_stride = (unsigned)(2 * urows * 16);                     // two chunks per k step
   const int S = p.n_stages;
-  constexpr int BC = grouped(WD) ? 128 : 64;
+  constexpr int BC = block_cols(WD);
   // B columns in use: int8 / int4 three digits; bf16 high + low parts
   constexpr int NCOL = (WD == W_BF16) ? 2 : 3;
-  const unsigned char* xcol = c.xs + (size_t)min(gq, NCOL - 1) * K * (WD == W_BF16 ? 2 : 1);
+  const int Ks = (WD == W_BF16) ? 2 * K : ((K + 127) & ~127);       // bytes per input column in shared memory
+  const unsigned char* xcol = c.xs + (size_t)min(gq, NCOL - 1) * Ks;
 
   // All fragments of a unit are loaded before its first MMA, and two accumulator sets are used in turn, so
   // that consecutive MMAs do not wait for each other.
   float facc[4] = {0.f, 0.f, 0.f, 0.f}, facc2[4] = {0.f, 0.f, 0.f, 0.f};
-  constexpr int NA = (WD == W_BF16 || WD == W_INT8G) ? 4 : 2;         // ldmatrix.x4 loads per unit
+  constexpr int NA = (WD == W_INT4) ? 2 : 4;         // ldmatrix.x4 loads per unit
   unsigned fa[NA][4];                                // pending unit: weight fragments,
   uint4 fx0 = make_uint4(0u, 0u, 0u, 0u), fx1 = fx0; // input fragments,
   unsigned fsz0 = 0u, fsz1 = 0u;                     // int4: {scale, zero} of my two rows,
@@ -465,28 +466,18 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int kind
       mma_bf16(facc2, fa[1], fx0.z, fx0.w);
       mma_bf16(facc, fa[2], fx1.x, fx1.y);
       mma_bf16(facc2, fa[3], fx1.z, fx1.w);
-    } else if (WD == W_INT8) {
-      // 64 columns of one input group: exact integer sums, then the group's input scale (the row's weight scale
-      // meets the finished sum in the epilogue)
-      int g4[4] = {0, 0, 0, 0}, h4[4] = {0, 0, 0, 0};
-      mma_s8(g4, fa[0][0], fa[0][1], fa[0][2], fa[0][3], fx0.x, fx0.y);
-      mma_s8(h4, fa[1][0], fa[1][1], fa[1][2], fa[1][3], fx0.z, fx0.w);
-      const float xsc = __int_as_float(fsx.z);
-      facc[0] = fmaf(xsc, (float)(g4[0] + h4[0]), facc[0]);
-      facc[1] = fmaf(xsc, (float)(g4[1] + h4[1]), facc[1]);
-      facc[2] = fmaf(xsc, (float)(g4[2] + h4[2]), facc[2]);
-      facc[3] = fmaf(xsc, (float)(g4[3] + h4[3]), facc[3]);
-    } else if (WD == W_INT8G) {
-      // one group of 128 columns: exact integer sums in two chains, then the weights' group scale times the
-      // input's group scale in one multiply-add per accumulator
+    } else if (WD == W_INT8 || WD == W_INT8G) {
+      // one group of 128 columns: exact integer sums in two chains, then the input's group scale -- times the
+      // weights' group scale for grouped int8; a per-row weight scale meets the finished sum in the epilogue --
+      // in one multiply-add per accumulator
       int g4[4] = {0, 0, 0, 0}, h4[4] = {0, 0, 0, 0};
       mma_s8(g4, fa[0][0], fa[0][1], fa[0][2], fa[0][3], fx0.x, fx0.y);
       mma_s8(h4, fa[1][0], fa[1][1], fa[1][2], fa[1][3], fx0.z, fx0.w);
       mma_s8(g4, fa[2][0], fa[2][1], fa[2][2], fa[2][3], fx1.x, fx1.y);
       mma_s8(h4, fa[3][0], fa[3][1], fa[3][2], fa[3][3], fx1.z, fx1.w);
       const float xsc = __int_as_float(fsx.z);
-      const float s0 = __half2float(__ushort_as_half((unsigned short)(fsz0 & 0xffffu))) * xsc;
-      const float s1 = __half2float(__ushort_as_half((unsigned short)(fsz1 & 0xffffu))) * xsc;
+      const float s0 = (WD == W_INT8) ? xsc : __half2float(__ushort_as_half((unsigned short)(fsz0 & 0xffffu))) * xsc;
+      const float s1 = (WD == W_INT8) ? xsc : __half2float(__ushort_as_half((unsigned short)(fsz1 & 0xffffu))) * xsc;
       facc[0] = fmaf(s0, (float)(g4[0] + h4[0]), facc[0]);
       facc[1] = fmaf(s0, (float)(g4[1] + h4[1]), facc[1]);
       facc[2] = fmaf(s1, (float)(g4[2] + h4[2]), facc[2]);
@@ -540,18 +531,17 @@ __device__ __forceinline__ void consume_pass(Ctx& c, const PassGeom& g, int kind
           const uint4* xp = reinterpret_cast<const uint4*>(xcol + ((size_t)next_b * BC + 16 * q) * 2);
           fx0 = xp[0];
           fx1 = xp[1];
-        } else if (WD == W_INT8) {
-          fx0 = *reinterpret_cast<const uint4*>(xcol + (size_t)next_b * BC + 16 * q);
-          fsx.z = *reinterpret_cast<const int*>(c.xs + 3 * (size_t)K + 32 * (next_b >> 1) + 8);   // the group's scale
         } else {
           const uint4* xp = reinterpret_cast<const uint4*>(xcol + (size_t)next_b * BC + 32 * q);
           fx0 = xp[0];
           fx1 = xp[1];
-          // {scale, zero} of my two fragment rows for this group (= this column block)
-          const unsigned* szp = reinterpret_cast<const unsigned*>(u + urows * (WD == W_INT4 ? 64 : 128));
-          fsz0 = szp[min(gq, urows - 1)];
-          fsz1 = szp[min(gq + 8, urows - 1)];
-          fsx = *reinterpret_cast<const int4*>(c.xs + 3 * (size_t)K + 32 * next_b + 16 * (q & 1));
+          if (WD != W_INT8) {
+            // {scale, zero} of my two fragment rows for this group (= this column block)
+            const unsigned* szp = reinterpret_cast<const unsigned*>(u + urows * (WD == W_INT4 ? 64 : 128));
+            fsz0 = szp[min(gq, urows - 1)];
+            fsz1 = szp[min(gq + 8, urows - 1)];
+          }
+          fsx = *reinterpret_cast<const int4*>(c.xs + 3 * (size_t)Ks + 32 * next_b + 16 * (q & 1));
         }
 #pragma unroll
         for (int j = 0; j < NA; j++) ldmatrix_x4(fa[j], u + lane_off + j * step_stride);

@@ -4,7 +4,8 @@
 // `slot` owns a contiguous run of "units" (1 row, or 2 rows where rows must stay together).  Inside a
 // block the rows are processed in passes of at most kPassRows rows.  In a pass the consumer warps form
 // a Wr x Wk grid: row-warp wr owns G <= 16 consecutive rows (one m16 tensor-core tile), k-warp wk owns
-// every Wk-th column block (64 columns; 128 for int4 and grouped int8 = one quantisation group).  The bytes of a pass are
+// every Wk-th column block (64 columns for bf16; 128 for the integer dtypes = one quantisation group; an int8 matrix
+// whose K is 64 short of a multiple of 128 gets its last block filled up with zero codes).  The bytes of a pass are
 // stored block-major: for column block b, the work units (b, wr = 0..Wr-1) one after another.  A work
 // unit -- the rows of one row-warp in one column block -- is contiguous, and a ring tile is a run of
 // `upt` consecutive units, so each block's weight stream is a sequence of contiguous byte runs that one
@@ -43,12 +44,12 @@ AMK_HD constexpr bool grouped(int wdtype) { return wdtype == W_INT4 || wdtype ==
 
 AMK_HD int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
-AMK_HD int block_cols(int wdtype) { return grouped(wdtype) ? 128 : 64; }          // columns per column block
-AMK_HD int block_chunks(int wdtype) { return (wdtype == W_BF16 || wdtype == W_INT8G) ? 8 : 4; }   // 16-byte chunks per row per block
+AMK_HD constexpr int block_cols(int wdtype) { return wdtype == W_BF16 ? 64 : 128; }   // columns per column block
+AMK_HD int block_chunks(int wdtype) { return wdtype == W_INT4 ? 4 : 8; }           // 16-byte chunks per row per block
 // bytes of a work unit holding `rows` rows (grouped: codes, then 4 bytes {scale, zero} per row, padded to 16)
 AMK_HD int unit_bytes(int wdtype, int rows) {
   if (wdtype == W_BF16) return rows * 128;
-  if (wdtype == W_INT8) return rows * 64;
+  if (wdtype == W_INT8) return rows * 128;
   if (wdtype == W_INT8G) return (rows * 132 + 15) & ~15;
   return (rows * 68 + 15) & ~15;
 }
@@ -58,15 +59,14 @@ AMK_HD int unit_bytes(int wdtype, int rows) {
 // fragment half h, the values j; its whole supply for a block is the contiguous column run starting at
 // q * (block_cols / 4).
 //   bf16: k = 16 s + 8 h + 2 q + j  (s<4, h<2, q<4, j<2)  ->  col 16 q + 4 s + 2 h + j
-//   int8: k = 32 s + 16 h + 4 q + j (s<2, h<2, q<4, j<4)  ->  col 16 q + 8 s + 4 h + j
-//   int4, grouped int8: k = 32 s + 16 h + 4 q + j (s<4, h<2, q<4, j<4)  ->  col 32 q + 8 s + 4 h + j
+//   int8, int4, grouped int8: k = 32 s + 16 h + 4 q + j (s<4, h<2, q<4, j<4)  ->  col 32 q + 8 s + 4 h + j
 AMK_HD int col_of_k(int wdtype, int k) {
   if (wdtype == W_BF16) {
     const int s = k >> 4, h = (k >> 3) & 1, q = (k >> 1) & 3, j = k & 1;
     return 16 * q + 4 * s + 2 * h + j;
   }
   const int s = k >> 5, h = (k >> 4) & 1, q = (k >> 2) & 3, j = k & 3;
-  return (wdtype == W_INT8 ? 16 : 32) * q + 8 * s + 4 * h + j;
+  return 32 * q + 8 * s + 4 * h + j;
 }
 
 // Where logical k of a row is stored inside its unit: the 16-byte chunk, and the element inside the chunk
@@ -145,7 +145,7 @@ AMK_HD PassGeom pass_geom(int R, int K, int wdtype, int stage_bytes) {
   g.Wr = ceil_div(R, G);
   g.g_last = R - (g.Wr - 1) * G;
   g.Wk = kConsumerWarps / g.Wr;
-  g.nblk = K / block_cols(wdtype);
+  g.nblk = ceil_div(K, block_cols(wdtype));
   if (g.Wk > g.nblk) g.Wk = g.nblk;
   g.n_units = g.Wr * g.nblk;
   g.ub_full = unit_bytes(wdtype, G);

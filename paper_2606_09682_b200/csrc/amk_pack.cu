@@ -84,13 +84,14 @@ __global__ void pack_kernel(const PackOp d, const PackSrc s, unsigned char* pack
       if (!inverse) *chunk = make_uint4(v[0], v[1], v[2], v[3]);
     } else if (wd == W_INT8 || wd == W_INT8G) {
       // chunk c = 2 s + hh holds logical k = 32 s + 16 hh + 4 q + j: for q = 0..3 the word at column
-      // (16 | 32 grouped) q + 8 s + 4 hh
-      const int sidx = c >> 1, hh = c & 1, qs = (wd == W_INT8) ? 16 : 32;
+      // 32 q + 8 s + 4 hh (zero codes beyond K: an int8 matrix's last block may be half full)
+      const int sidx = c >> 1, hh = c & 1;
       unsigned* w32 = reinterpret_cast<unsigned*>(src.w);
       unsigned v[4];
       if (inverse) { const uint4 t = *chunk; v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w; }
       for (int q = 0; q < 4; q++) {
-        const int col = col0 + qs * q + 8 * sidx + 4 * hh;
+        const int col = col0 + 32 * q + 8 * sidx + 4 * hh;
+        if (col >= K) { if (!inverse) v[q] = 0u; continue; }
         if (!inverse) v[q] = w32[col >> 2];
         else w32[col >> 2] = v[q];
       }

@@ -29,7 +29,7 @@ int main(int argc, char** argv) {
   if (bounds[0] != 0 || bounds[N] != rows / unit_rows) { printf("bad bounds\n"); return 1; }
   const int bc = block_cols(wd), cpb = block_chunks(wd);
   const int epc = bc / cpb;                     // elements per 16-byte chunk
-  if (K % bc) { printf("K not a multiple of the column block\n"); return 1; }
+  if (K % bc && !(wd == W_INT8 && K % bc == 64)) { printf("K not a multiple of the column block\n"); return 1; }
   // the in-block permutation
   {
     std::vector<int> col_seen(bc, 0), place_seen(bc, 0);
@@ -106,6 +106,7 @@ int main(int argc, char** argv) {
                 if (byte >= (long long)mark.size()) { printf("element outside the pass\n"); return 1; }
                 mark[byte] = 1;
                 if (wd == W_BF16) mark[byte + 1] = 1;
+                if (next_b * bc + col_of_k(wd, k) >= K) continue;         // (zero fill of an int8 matrix's half-full last block)
                 seen[(size_t)row * K + (size_t)next_b * bc + col_of_k(wd, k)]++;
               }
               if (grouped(wd)) {
@@ -123,7 +124,7 @@ int main(int argc, char** argv) {
       // every byte except unit padding is used
       long long used = 0;
       for (unsigned char m : mark) used += m;
-      const long long expect = (long long)R * g.nblk * (wd == W_BF16 ? 128 : (wd == W_INT8 ? 64 : (wd == W_INT4 ? 68 : 132)));
+      const long long expect = (long long)R * g.nblk * (wd == W_INT4 ? 68 : (wd == W_INT8G ? 132 : 128));
       if (used != expect) { printf("bytes used %lld, expected %lld\n", used, expect); return 1; }
       sbytes += pass_bytes(g);
     }
