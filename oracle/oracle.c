@@ -117,6 +117,40 @@ void orc_rope(float* u, int hd, int pos, double theta) {
 /* SiLU: z * sigmoid(z). */
 float orc_silu(float z) { return (float)((double)z / (1.0 + exp(-(double)z))); }
 
+/* ----------------------------------------------------------------------------------------------
+ * fp8 "e4m3" (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; no infinities; the one NaN is
+ * magnitude code 0x7f; largest finite value 448 = code 0x7e): the element type of the optional 8-bit KV
+ * cache.  Narrowing is round-to-nearest-even with saturation: every finite value beyond 448 (and either
+ * infinity) becomes +-448; NaN stays NaN.
+ * -------------------------------------------------------------------------------------------- */
+float orc_e4m3_to_f32(uint8_t code) {
+    int e = (code >> 3) & 0xf, m = code & 7;
+    double v;
+    if (e == 0xf && m == 7) return (code & 0x80) ? -NAN : NAN;
+    if (e == 0) v = ldexp((double)m, -9);                     /* subnormal: m/8 * 2^-6 */
+    else v = ldexp(1.0 + (double)m / 8.0, e - 7);
+    return (float)((code & 0x80) ? -v : v);
+}
+
+uint8_t orc_f32_to_e4m3(float x) {
+    uint8_t sign = signbit(x) ? 0x80 : 0x00;
+    double a = fabs((double)x);
+    if (isnan(x)) return (uint8_t)(sign | 0x7f);
+    if (a > 448.0) return (uint8_t)(sign | 0x7e);             /* saturate (464 and beyond would need code 0x7f) */
+    if (a < ldexp(1.0, -6)) {                                 /* subnormal range: multiples of 2^-9; rint ties to even */
+        int q = (int)rint(ldexp(a, 9));                       /* 0..8; 8 is the smallest normal, code 0x08 */
+        return (uint8_t)(sign | q);
+    }
+    int ex;
+    double f = frexp(a, &ex);                                 /* a = f * 2^ex, f in [0.5, 1) */
+    int E = ex - 1;                                           /* a = (2f) * 2^E, 2f in [1, 2) */
+    int m = (int)rint((2.0 * f - 1.0) * 8.0);                 /* 0..8, ties to even */
+    if (m == 8) { m = 0; E += 1; }
+    int code = ((E + 7) << 3) | m;
+    if (code > 0x7e) code = 0x7e;
+    return (uint8_t)(sign | code);
+}
+
 /* Index of the largest entry; the lowest index wins an exact tie. */
 int orc_argmax(const float* v, int n) {
     int best = 0;
@@ -272,18 +306,31 @@ void orc_quantize_int4(const uint16_t* W_bf16, int rows, int cols, int group, ui
  * Attention for one query head over cache positions [j0, j1)
  * -------------------------------------------------------------------------------------------- */
 
-/* Plain softmax attention.  K, V: [n_pos][hd] bf16 rows of one kv head.  Reading (paper silent):
- * scores scaled by 1/sqrt(hd), every position j0 <= j < j1 attended, no other mask.
+/* One cache element as fp32.  The cache is an array of 16-bit words whatever its element type: a bf16 bit
+ * pattern (kv_dtype 0), or an e4m3 code in the low byte (kv_dtype 1). */
+static float kv_to_f32(int kv_dtype, uint16_t word) {
+    return kv_dtype == 1 ? orc_e4m3_to_f32((uint8_t)word) : orc_bf16_to_f32(word);
+}
+
+/* Plain softmax attention.  K, V: [n_pos][hd] rows of one kv head, bf16 (orc_attention_head) or of the given
+ * cache element type (orc_attention_head_kv).  Reading (paper silent): scores scaled by 1/sqrt(hd), every
+ * position j0 <= j < j1 attended, no other mask.
  * Optionally returns the softmax weights (w_out, length j1-j0, may be NULL). */
+void orc_attention_head_kv(int kv_dtype, const float* q, const uint16_t* K, const uint16_t* V, int hd, int j0, int j1,
+                           float* o, double* w_out);
 void orc_attention_head(const float* q, const uint16_t* K, const uint16_t* V, int hd, int j0, int j1,
                         float* o, double* w_out) {
+    orc_attention_head_kv(0, q, K, V, hd, j0, j1, o, w_out);
+}
+void orc_attention_head_kv(int kv_dtype, const float* q, const uint16_t* K, const uint16_t* V, int hd, int j0, int j1,
+                           float* o, double* w_out) {
     int n = j1 - j0;
     double* s = (double*)malloc(sizeof(double) * (size_t)n);
     double inv = 1.0 / sqrt((double)hd);
     double M = -INFINITY;
     for (int j = j0; j < j1; j++) {
         double d = 0.0;
-        for (int t = 0; t < hd; t++) d += (double)q[t] * (double)orc_bf16_to_f32(K[(size_t)j * hd + t]);
+        for (int t = 0; t < hd; t++) d += (double)q[t] * (double)kv_to_f32(kv_dtype, K[(size_t)j * hd + t]);
         s[j - j0] = d * inv;
         if (s[j - j0] > M) M = s[j - j0];
     }
@@ -291,7 +338,7 @@ void orc_attention_head(const float* q, const uint16_t* K, const uint16_t* V, in
     for (int j = 0; j < n; j++) { s[j] = exp(s[j] - M); Z += s[j]; }
     for (int t = 0; t < hd; t++) {
         double acc = 0.0;
-        for (int j = 0; j < n; j++) acc += (s[j] / Z) * (double)orc_bf16_to_f32(V[(size_t)(j + j0) * hd + t]);
+        for (int j = 0; j < n; j++) acc += (s[j] / Z) * (double)kv_to_f32(kv_dtype, V[(size_t)(j + j0) * hd + t]);
         o[t] = (float)acc;
     }
     if (w_out) for (int j = 0; j < n; j++) w_out[j] = s[j] / Z;
@@ -347,10 +394,12 @@ typedef struct {
     float rope_theta;
     int32_t wdtype;        /* 0 bf16, 1 int8, 2 int4, 3 grouped int8: applies to the seven per-layer linears only */
     int32_t group_size;    /* int4 / grouped int8: group length along the input dimension */
-    int32_t round_kv;      /* 1: cache entries rounded to bf16 (the contract); 0: test-only, see below */
+    int32_t round_kv;      /* 1: cache entries rounded to the cache element type (the contract); 0: test-only, see below */
     int32_t quantize_lm_head; /* 0: the LM head stays bf16 (the reading taken of the paper); 1: it is quantised like
                                  the per-layer linears (wdtype, group_size) -- the other reading of "linear GEMV
                                  weights move to int8 / int4" for an untied head; the embedding gather stays bf16 */
+    int32_t kv_dtype;      /* element type of the KV cache: 0 bf16 (what the paper's kernels keep, Section 5), 1 fp8 e4m3
+                              (a variant: the same step with the cache rounded to 8 bits instead of 16) */
 } orc_config;
 
 /* Canonical weights.  Per-layer arrays are indexed [layer]; linears are indexed by
@@ -402,24 +451,28 @@ static void linear(const orc_config* c, const orc_weights* w, int kind, int laye
  * tied, and it stays bf16 in the quantised variants (tied or not).
  */
 
-/* Distance between two bf16 values in representable steps (sign-magnitude bit patterns ordered as integers). */
-static int bf16_steps_apart(uint16_t a, uint16_t b) {
-    int ia = (a & 0x8000u) ? -(int)(a & 0x7fffu) : (int)(a & 0x7fffu);
-    int ib = (b & 0x8000u) ? -(int)(b & 0x7fffu) : (int)(b & 0x7fffu);
+/* Distance between two bf16 (or, sign_bit = 0x80, e4m3) values in representable steps (sign-magnitude bit
+ * patterns ordered as integers). */
+static int steps_apart(uint16_t a, uint16_t b, uint16_t sign_bit) {
+    uint16_t mag = (uint16_t)(sign_bit - 1);
+    int ia = (a & sign_bit) ? -(int)(a & mag) : (int)(a & mag);
+    int ib = (b & sign_bit) ? -(int)(b & mag) : (int)(b & mag);
     return ia > ib ? ia - ib : ib - ia;
 }
 
-/* The cache entry appended for one fp32 value.  The contract is round-to-nearest-even to bf16.  Two correct
+/* The cache entry appended for one fp32 value.  The contract is round-to-nearest-even to bf16 (to e4m3 with
+ * saturation for an fp8 cache; the entry is then the code in a 16-bit word).  Two correct
  * implementations whose fp32 values differ in the last bits (another summation order) may land on either side
  * of a rounding boundary, i.e. on neighbouring bf16 values: both are valid cache entries.  A caller that
  * compares another implementation with this one can pass that implementation's entry as `pref`: it is adopted
  * only if it is this oracle's own rounding or one of its two neighbours, so that everything computed FROM the
  * cache afterwards is compared like with like; otherwise the oracle keeps its own.  `own` always receives the
  * oracle's own rounding. */
-static uint16_t cache_entry(float value, const uint16_t* pref, uint16_t* own, int* adopted) {
-    uint16_t r = orc_f32_to_bf16(value);
+static uint16_t cache_entry(int kv_dtype, float value, const uint16_t* pref, uint16_t* own, int* adopted) {
+    uint16_t r = kv_dtype == 1 ? (uint16_t)orc_f32_to_e4m3(value) : orc_f32_to_bf16(value);
     if (own) *own = r;
-    if (pref && *pref != r && bf16_steps_apart(*pref, r) <= 1) { if (adopted) (*adopted)++; return *pref; }
+    if (pref && *pref != r && (kv_dtype != 1 || (*pref & 0x7f) != 0x7f) &&
+        steps_apart(*pref, r, kv_dtype == 1 ? 0x80 : 0x8000) <= 1) { if (adopted) (*adopted)++; return *pref; }
     return r;
 }
 
@@ -473,9 +526,9 @@ int orc_decode_step_rows(const orc_config* c, const orc_weights* w, int token, i
             const size_t rbase = ((size_t)l * nkv + g) * hd, rhalf = (size_t)L * nkv * hd;
             for (int d = 0; d < hd; d++) {
                 if (c->round_kv) {
-                    kv_cache[base + d] = cache_entry(k[g * hd + d], rows_pref ? rows_pref + rbase + d : NULL,
+                    kv_cache[base + d] = cache_entry(c->kv_dtype, k[g * hd + d], rows_pref ? rows_pref + rbase + d : NULL,
                                                      rows_own ? rows_own + rbase + d : NULL, n_adopted);
-                    kv_cache[kv_half + base + d] = cache_entry(v[g * hd + d], rows_pref ? rows_pref + rhalf + rbase + d : NULL,
+                    kv_cache[kv_half + base + d] = cache_entry(c->kv_dtype, v[g * hd + d], rows_pref ? rows_pref + rhalf + rbase + d : NULL,
                                                                rows_own ? rows_own + rhalf + rbase + d : NULL, n_adopted);
                 } else {
                     kv_f32[base + d] = k[g * hd + d];
@@ -489,7 +542,7 @@ int orc_decode_step_rows(const orc_config* c, const orc_weights* w, int token, i
             int g = h / n_rep;
             size_t base = ((size_t)l * nkv + g) * S * hd;
             if (c->round_kv) {
-                orc_attention_head(q + (size_t)h * hd, kv_cache + base, kv_cache + kv_half + base, hd, 0, pos + 1,
+                orc_attention_head_kv(c->kv_dtype, q + (size_t)h * hd, kv_cache + base, kv_cache + kv_half + base, hd, 0, pos + 1,
                                    o + (size_t)h * hd, NULL);
             } else {
                 /* same definition on the fp32 shadow cache */
@@ -572,9 +625,9 @@ int orc_layer_step_rows(const orc_config* c, const orc_weights* w, int layer, in
         size_t base = (((size_t)l * nkv + g) * S + (size_t)pos) * hd;
         const size_t rbase = (size_t)g * hd, rhalf = (size_t)nkv * hd;
         for (int d = 0; d < hd; d++) {
-            kv_cache[base + d] = cache_entry(k[g * hd + d], rows_pref ? rows_pref + rbase + d : NULL,
+            kv_cache[base + d] = cache_entry(c->kv_dtype, k[g * hd + d], rows_pref ? rows_pref + rbase + d : NULL,
                                              rows_own ? rows_own + rbase + d : NULL, n_adopted);
-            kv_cache[kv_half + base + d] = cache_entry(v[g * hd + d], rows_pref ? rows_pref + rhalf + rbase + d : NULL,
+            kv_cache[kv_half + base + d] = cache_entry(c->kv_dtype, v[g * hd + d], rows_pref ? rows_pref + rhalf + rbase + d : NULL,
                                                        rows_own ? rows_own + rhalf + rbase + d : NULL, n_adopted);
         }
     }
@@ -582,7 +635,7 @@ int orc_layer_step_rows(const orc_config* c, const orc_weights* w, int layer, in
     for (int h = 0; h < nq; h++) {
         int g = h / n_rep;
         size_t base = ((size_t)l * nkv + g) * S * hd;
-        orc_attention_head(q + (size_t)h * hd, kv_cache + base, kv_cache + kv_half + base, hd, 0, pos + 1,
+        orc_attention_head_kv(c->kv_dtype, q + (size_t)h * hd, kv_cache + base, kv_cache + kv_half + base, hd, 0, pos + 1,
                            o + (size_t)h * hd, NULL);
     }
     linear(c, w, 3, l, H, nq * hd, o, t);

@@ -21,6 +21,7 @@ _LIB = os.path.join(_HERE, "liboracle.so")
 
 KINDS = ("wq", "wk", "wv", "wo", "wgate", "wup", "wdown")
 W_BF16, W_INT8, W_INT4, W_INT8G = 0, 1, 2, 3
+KV_BF16, KV_E4M3 = 0, 1      # cache element type; the cache array holds 16-bit words either way (an e4m3 code in the low byte)
 
 
 def build(force: bool = False) -> str:
@@ -37,7 +38,8 @@ class _Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("hidden", "n_layers", "n_q_heads", "n_kv_heads", "head_dim",
                                          "mlp", "vocab", "max_seq", "tied_embeddings")] + [
         ("rms_eps", C.c_float), ("rope_theta", C.c_float),
-        ("wdtype", C.c_int32), ("group_size", C.c_int32), ("round_kv", C.c_int32), ("quantize_lm_head", C.c_int32)]
+        ("wdtype", C.c_int32), ("group_size", C.c_int32), ("round_kv", C.c_int32), ("quantize_lm_head", C.c_int32),
+        ("kv_dtype", C.c_int32)]
 
 
 _PP = C.POINTER(C.c_void_p)
@@ -66,6 +68,10 @@ def lib() -> C.CDLL:
         L.orc_f16_to_f32.argtypes = [C.c_uint16]
         L.orc_f32_to_f16.restype = C.c_uint16
         L.orc_f32_to_f16.argtypes = [C.c_float]
+        L.orc_e4m3_to_f32.restype = C.c_float
+        L.orc_e4m3_to_f32.argtypes = [C.c_uint8]
+        L.orc_f32_to_e4m3.restype = C.c_uint8
+        L.orc_f32_to_e4m3.argtypes = [C.c_float]
         L.orc_silu.restype = C.c_float
         L.orc_silu.argtypes = [C.c_float]
         L.orc_argmax.restype = C.c_int
@@ -106,6 +112,26 @@ def f32_to_bf16(x) -> np.ndarray:
     v = np.asarray(x, dtype=np.float32)
     out = np.empty(v.shape, dtype=np.uint16)
     f = lib().orc_f32_to_bf16
+    fi, fo = v.ravel(), out.ravel()
+    for i in range(fi.size):
+        fo[i] = f(float(fi[i]))
+    return out
+
+
+def e4m3_to_f32(codes) -> np.ndarray:
+    b = np.asarray(codes, dtype=np.uint8)
+    out = np.empty(b.shape, dtype=np.float32)
+    f = lib().orc_e4m3_to_f32
+    fi, fo = b.ravel(), out.ravel()
+    for i in range(fi.size):
+        fo[i] = f(int(fi[i]))
+    return out
+
+
+def f32_to_e4m3(x) -> np.ndarray:
+    v = np.asarray(x, dtype=np.float32)
+    out = np.empty(v.shape, dtype=np.uint8)
+    f = lib().orc_f32_to_e4m3
     fi, fo = v.ravel(), out.ravel()
     for i in range(fi.size):
         fo[i] = f(float(fi[i]))
@@ -311,8 +337,9 @@ class Model:
     """
 
     def __init__(self, shape, weights: Dict, wdtype: int = W_BF16, group: int = 128, round_kv: bool = True,
-                 quantize_lm_head: bool = False):
-        """``quantize_lm_head``: the LM head is read from ``weights["lm_head_q"]`` / ``["lm_head_scale"]`` /
+                 quantize_lm_head: bool = False, kv_dtype: int = KV_BF16):
+        """``kv_dtype``: KV_BF16, or KV_E4M3 (cache entries rounded to fp8 e4m3; the cache array then holds the codes).
+        ``quantize_lm_head``: the LM head is read from ``weights["lm_head_q"]`` / ``["lm_head_scale"]`` /
         ``["lm_head_zero"]`` (see ``quantize_lm_head``), quantised like the layers."""
         self.shape = Shape.of(shape)
         s = self.shape
@@ -320,7 +347,8 @@ class Model:
         self._keep: List[np.ndarray] = []
         qlm = bool(quantize_lm_head) and wdtype != W_BF16
         self.cfg = _Config(s.hidden, s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, s.mlp, s.vocab,
-                           s.max_seq, int(s.tied), s.rms_eps, s.rope_theta, wdtype, group, int(round_kv), int(qlm))
+                           s.max_seq, int(s.tied), s.rms_eps, s.rope_theta, wdtype, group, int(round_kv), int(qlm),
+                           int(kv_dtype))
         w = _Weights()
         w.embed = self._hold(weights["embed"], np.uint16)
         w.lm_head = None if s.tied else self._hold(weights["lm_head"], np.uint16)

@@ -28,9 +28,23 @@ def round_bf16(x64):
     return t.to(torch.float64).numpy()
 
 
-def dense_forward(shape, W, tokens, round_kv=True):
+def e4m3_codes(x64):
+    """fp64 -> fp32 -> e4m3 codes through torch's conversion (round to nearest even; callers stay below 448)."""
+    t = torch.tensor(np.asarray(x64, dtype=np.float64)).to(torch.float32).to(torch.float8_e4m3fn)
+    return t.view(torch.uint8).numpy()
+
+
+def e4m3_values(codes):
+    return torch.from_numpy(np.ascontiguousarray(codes, dtype=np.uint8)).view(torch.float8_e4m3fn).to(torch.float64).numpy()
+
+
+def dense_forward(shape, W, tokens, round_kv=True, e4m3_cache=None):
     """Logits [T][V] and hidden [T][L+1][H] for the whole token prefix, recomputed from scratch.
-    W: dict of float64 matrices (already dequantised)."""
+    W: dict of float64 matrices (already dequantised).
+    ``e4m3_cache``: the step-by-step implementation's fp8 cache as codes [2][L][n_kv][S][hd].  fp8 steps are coarse
+    (2^-4 relative), so two correct computations of a key that differ in the last fp32 bits may round to neighbouring
+    codes and then differ visibly downstream; here each cached code must be this dense form's own rounding of its own
+    fp64 key / value or a neighbour of it, and the dense form then carries on with the cached code's value."""
     T = len(tokens)
     H, nq, nkv, hd = shape.hidden, shape.n_q_heads, shape.n_kv_heads, shape.head_dim
     n_rep = nq // nkv
@@ -55,7 +69,16 @@ def dense_forward(shape, W, tokens, round_kv=True):
         Q = rot((A @ W["wq"][l].T).reshape(T, nq, hd))
         K = rot((A @ W["wk"][l].T).reshape(T, nkv, hd))
         Vv = (A @ W["wv"][l].T).reshape(T, nkv, hd)
-        if round_kv:
+        if e4m3_cache is not None:
+            for which, U in ((0, K), (1, Vv)):
+                got = np.transpose(e4m3_cache[which, l, :, :T, :], (1, 0, 2)).astype(np.uint8)      # [T][n_kv][hd]
+                own = e4m3_codes(U)
+                mag = lambda c: np.where(c & 0x80, -(c & 0x7F).astype(np.int32), (c & 0x7F).astype(np.int32))
+                apart = np.abs(mag(got) - mag(own))
+                assert apart.max() <= 1, (l, which, int(apart.max()))
+                assert (apart != 0).mean() < 0.01                     # neighbours are the rare exception
+                U[...] = e4m3_values(got)
+        elif round_kv:
             K, Vv = round_bf16(K), round_bf16(Vv)
         O = np.zeros((T, nq, hd))
         for h in range(nq):
@@ -142,6 +165,38 @@ def test_decode_with_cache_equals_dense_recompute(name, norm_jitter):
     kvv = kv.reshape(2, shape.n_layers, shape.n_kv_heads, S, hd)
     assert not kvv[:, :, :, len(toks):, :].any()
     assert kvv[:, :, :, :len(toks), :].any()
+
+
+@pytest.mark.parametrize("name,wdtype", [("toy", orc.W_BF16), ("toy_ragged", orc.W_BF16), ("toy", orc.W_INT8)])
+def test_fp8_cache_decode_equals_dense_recompute_on_the_cached_codes(name, wdtype):
+    """kv_dtype = e4m3: every appended cache entry is the e4m3 rounding (torch's, on an independent fp64 forward)
+    of the rotated key / the value or its neighbour; attention reads the decoded codes; everything downstream
+    equals the dense form computed from those codes.  The cache differs from the bf16 cache's values."""
+    shape = inp.SHAPES[name]
+    group = 32 if name == "toy" else 8
+    w = inp.make_weights(shape, seed=19, std=0.25 if name == "toy" else 0.08, norm_jitter=0.1)
+    wq = orc.quantize_weights(inp.weights_to_numpy(w), wdtype, group)
+    model = orc.Model(shape, wq, wdtype=wdtype, group=group, kv_dtype=orc.KV_E4M3)
+    model16 = orc.Model(shape, wq, wdtype=wdtype, group=group)
+    toks = greedy_tokens(8, shape.vocab, 9)
+    kv, kv16 = model.new_cache(), model16.new_cache()
+    outs = []
+    for t, tok in enumerate(toks):
+        outs.append(model.decode_step(tok, t, kv))
+        l16, _, h16 = model16.decode_step(tok, t, kv16)
+    assert kv.max() <= 0xFF                                          # codes in the low byte
+    L, G, S, hd = shape.n_layers, shape.n_kv_heads, shape.max_seq, shape.head_dim
+    codes = kv.reshape(2, L, G, S, hd)
+    logits_d, hidden_d = dense_forward(shape, to_f64(wq, shape, wdtype, group), toks, e4m3_cache=codes)
+    for t in range(len(toks)):
+        logits, nxt, hidden = outs[t]
+        assert rel_l2(hidden, hidden_d[t]) < 2e-5
+        assert rel_l2(logits, logits_d[t]) < 2e-5
+    assert not codes[:, :, :, len(toks):, :].any()                   # slots beyond the last position untouched
+    assert rel_l2(outs[-1][0], l16) > 1e-3                           # not the bf16 cache's result
+    # position 0 of layer 0: the attention output is the decoded cached v (softmax over one position)
+    assert np.array_equal(orc.e4m3_to_f32(codes[1, 0, :, 0, :].astype(np.uint8)),
+                          e4m3_values(codes[1, 0, :, 0, :]).astype(np.float32))
 
 
 @pytest.mark.parametrize("wdtype", [orc.W_INT8, orc.W_INT4, orc.W_INT8G])
@@ -235,13 +290,14 @@ def _bump(bits, steps):
     return (np.asarray(bits, dtype=np.uint16) + np.uint16(steps)).astype(np.uint16)
 
 
-def test_preferred_cache_rows_are_adopted_only_next_to_the_own_rounding():
+@pytest.mark.parametrize("kv_dtype", [orc.KV_BF16, orc.KV_E4M3])
+def test_preferred_cache_rows_are_adopted_only_next_to_the_own_rounding(kv_dtype):
     """decode_step(rows_pref=...): another implementation's appended rows are taken where they are the oracle's
-    own rounding or a neighbouring bf16 value, and attention then reads them; anything further away is refused.
-    Pinned at position 0, where the attention output is the cached V row, against the dense form."""
+    own rounding or a neighbouring bf16 (e4m3) value, and attention then reads them; anything further away is
+    refused.  Pinned at position 0, where the attention output is the cached V row, against the dense form."""
     shape = inp.SHAPES["toy"]
     wnp = inp.weights_to_numpy(inp.make_weights(shape, seed=14, std=0.25))
-    model = orc.Model(shape, wnp)
+    model = orc.Model(shape, wnp, kv_dtype=kv_dtype)
     tok = 42
     L, G, S, hd = shape.n_layers, shape.n_kv_heads, shape.max_seq, shape.head_dim
     kv0 = model.new_cache()
@@ -267,7 +323,7 @@ def test_preferred_cache_rows_are_adopted_only_next_to_the_own_rounding():
     # the dense form of layer 0 with the adopted V row
     W = to_f64(wnp, shape)
     x0 = W["embed"][tok]
-    v = f64(pref[1, 0]).reshape(G, hd)
+    v = (f64(pref[1, 0]) if kv_dtype == orc.KV_BF16 else e4m3_values(pref[1, 0])).reshape(G, hd)
     n_rep = shape.n_q_heads // G
     o = np.concatenate([v[h // n_rep] for h in range(shape.n_q_heads)])
     x_attn = x0 + o @ W["wo"][0].T

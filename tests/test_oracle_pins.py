@@ -450,3 +450,41 @@ def test_streamed_bytes_table():
     b = streamed_bytes(SHAPES["llama3_8b"], "int8", 4096)
     assert abs((b["weights"] + b["scales"]) / 1e6 - 8033.29) < 0.01
     assert abs(2.0 * 32 * 8 * 128 * 2 * 4096 / 1e6 - 536.87) < 0.01
+
+
+# ------------------------------------------------------------------------------------------------
+# fp8 e4m3 (the element type of the optional 8-bit KV cache)
+# ------------------------------------------------------------------------------------------------
+
+def test_e4m3_to_f32_exhaustive_vs_torch():
+    codes = np.arange(256, dtype=np.uint8)
+    ours = orc.e4m3_to_f32(codes)
+    ref = torch.from_numpy(codes.copy()).view(torch.float8_e4m3fn).to(torch.float32).numpy()
+    nan = np.isnan(ref)
+    assert nan.sum() == 2 and nan[0x7F] and nan[0xFF] and np.isnan(ours[nan]).all()
+    assert np.array_equal(ours[~nan].view(np.uint32), ref[~nan].view(np.uint32))       # bit for bit, -0 included
+    assert ours[0x7E] == 448.0 and ours[0x01] == 2.0 ** -9 and ours[0x08] == 2.0 ** -6
+
+
+def test_f32_to_e4m3_vs_torch_ties_and_saturation():
+    rng = np.random.default_rng(77)
+    vals = [rng.standard_normal(20000).astype(np.float32) * s for s in (1e-3, 1e-2, 1.0, 30.0, 200.0)]
+    # every representable value, every midpoint between neighbours (ties), and values a hair to either side
+    rep = orc.e4m3_to_f32(np.arange(0x7F, dtype=np.uint8)).astype(np.float64)
+    mid = (rep[:-1] + rep[1:]) / 2
+    edge = np.concatenate([rep, mid, mid * (1 + 1e-6), mid * (1 - 1e-6)]).astype(np.float32)
+    x = np.concatenate(vals + [edge, -edge, np.array([0.0, -0.0], dtype=np.float32)])
+    x = x[np.abs(x) <= 464.0]                         # beyond the tie above 448 torch gives NaN, the contract here saturates
+    ours = orc.f32_to_e4m3(x)
+    ref = torch.from_numpy(x.copy()).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert np.array_equal(ours, ref)
+    # round trip of every finite code, ties to even at hand-worked midpoints, saturation, NaN
+    codes = np.array([c for c in range(256) if (c & 0x7F) != 0x7F], dtype=np.uint8)
+    assert np.array_equal(orc.f32_to_e4m3(orc.e4m3_to_f32(codes)), codes)
+    assert orc.f32_to_e4m3(np.float32(2.0 ** -10))[()] == 0x00            # half the smallest subnormal: tie -> even (0)
+    assert orc.f32_to_e4m3(np.float32(3 * 2.0 ** -10))[()] == 0x02        # 1.5 subnormal steps: tie -> even (2)
+    assert orc.f32_to_e4m3(np.float32(1.0625))[()] == 0x38                # 1 + 1/16: tie between 1.0 and 1.125 -> 1.0
+    assert orc.f32_to_e4m3(np.float32(1.1875))[()] == 0x3A                # tie between 1.125 and 1.25 -> 1.25 (even)
+    assert orc.f32_to_e4m3(np.float32(464.0))[()] == 0x7E and orc.f32_to_e4m3(np.float32(465.0))[()] == 0x7E
+    assert orc.f32_to_e4m3(np.float32(1e30))[()] == 0x7E and orc.f32_to_e4m3(np.float32(-np.inf))[()] == 0xFE
+    assert orc.f32_to_e4m3(np.float32(np.nan))[()] & 0x7F == 0x7F
