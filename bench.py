@@ -53,14 +53,32 @@ WORKLOADS = {
     # quantize_lm_head = 1: the LM head streamed as int8 too (the other reading of the paper for an untied head)
     "tinyllama_1b_int8_qhead_pos0": ("tinyllama_1b", "int8", 0),
     "llama3_8b_int8_qhead_pos0": ("llama3_8b", "int8", 0),
+    # an fp8 (e4m3) KV cache: half the cache bytes at long positions
+    "tinyllama_1b_bf16_fp8kv_pos1024": ("tinyllama_1b", "bf16", 1024),
+    "llama3_8b_int8_fp8kv_pos4096": ("llama3_8b", "int8", 4096),
 }
 QHEAD = {"tinyllama_1b_int8_qhead_pos0", "llama3_8b_int8_qhead_pos0"}
+FP8KV = {"tinyllama_1b_bf16_fp8kv_pos1024", "llama3_8b_int8_fp8kv_pos4096"}
+
+
+def kv_dtype_of(workload: str) -> str:
+    return "fp8" if workload in FP8KV else "bf16"
+
+
+def kv_words(t) -> np.ndarray:
+    """A cache tensor as the oracle keeps it: one 16-bit word per element (a bf16 bit pattern, or an e4m3 code)."""
+    if t.dtype == torch.uint8:
+        return t.contiguous().cpu().numpy().astype(np.uint16)
+    return inp.bits(t)
+
+
 DEFAULT_WORKLOAD = "llama3_8b_bf16_pos0"      # the largest single-GPU configuration
 OTHER = ["llama3_8b_int8_pos0", "tinyllama_1b_bf16_pos0", "tinyllama_1b_int8_pos0", "tinyllama_1b_int4_pos0",
          "smollm2_135m_bf16_pos0", "tinyllama_1b_bf16_pos1024", "tinyllama_1b_int8_pos512", "llama3_8b_int8_pos4096",
          "llama3_8b_bf16_pos4096", "llama32_1b_bf16_pos0", "llama32_1b_int8_pos0", "tinyllama_1b_int8_qhead_pos0",
          "llama3_8b_int8_qhead_pos0", "paper_small_bf16_pos0", "paper_small_int8_pos0", "paper_small_int4_pos0",
-         "llama3_8b_int4_pos0", "tinyllama_1b_int8g_pos0", "llama3_8b_int8g_pos0"]
+         "llama3_8b_int4_pos0", "tinyllama_1b_int8g_pos0", "llama3_8b_int8g_pos0", "tinyllama_1b_bf16_fp8kv_pos1024",
+         "llama3_8b_int8_fp8kv_pos4096"]
 # device-resident multi-token runs (amk_decode_greedy: the token is fed back on the device): (shape, dtype, steps)
 SUSTAINED = [("smollm2_135m", "bf16", 256), ("tinyllama_1b", "bf16", 256)]
 METRIC = "batch-1 decode us/token; achieved HBM GB/s vs B200 measured peak"
@@ -160,14 +178,15 @@ def build_decoder(workload: str, device, sync_mode: int = 0):
     if qhead:
         wq = amk.quantize_lm_head(wq, wd, shape.tied)
     dec = amk.Decoder(shape, wq, wd, flags=amk.AMK_FLAG_DEBUG_HIDDEN, sync_mode=sync_mode, device=device,
-                      quantize_lm_head=qhead)
+                      quantize_lm_head=qhead, kv_dtype=kv_dtype_of(workload))
     keep = {k: w[k][0] for k in inp.KINDS}
     keep["qhead"] = qhead
+    keep["kv_dtype"] = kv_dtype_of(workload)
     keep.update(attn_norm=w["attn_norm"][0], mlp_norm=w["mlp_norm"][0], final_norm=w["final_norm"], embed=w["embed"],
                 lm_head=None if shape.tied else w["lm_head"])
     del w, wq
     torch.cuda.empty_cache()
-    kv = inp.make_kv_prefill(shape, SEED, pos, device=device)
+    kv = inp.make_kv_prefill(shape, SEED, pos, device=device, kv_dtype=kv_dtype_of(workload))
     tok = inp.make_token(shape, SEED)
     return shape, wd, pos, dec, kv, tok, keep
 
@@ -250,14 +269,16 @@ class OracleSample:
         self.qhead = bool(keep and keep.get("qhead"))
         if self.qhead:
             wq = orc.quantize_lm_head(wq, wdt, 128, tied=shape.tied)
-        self.model = orc.Model(s1, wq, wdtype=wdt, group=128, quantize_lm_head=self.qhead)
+        self.kv_dtype = (keep or {}).get("kv_dtype", "bf16")
+        self.model = orc.Model(s1, wq, wdtype=wdt, group=128, quantize_lm_head=self.qhead,
+                               kv_dtype=orc.KV_E4M3 if self.kv_dtype == "fp8" else orc.KV_BF16)
         self.kv = np.zeros(orc.kv_elems(s1), dtype=np.uint16)
         if pos > 0:
             if kv_gpu is None:
                 self.kv[:] = inp.bits(inp.make_kv_prefill(s1, SEED, pos, device="cpu"))
             else:       # layer 0's slice of the GPU run's pre-filled cache (a seeded input)
                 L, G, S, hd = shape.n_layers, shape.n_kv_heads, shape.max_seq, shape.head_dim
-                self.kv[:] = inp.bits(kv_gpu.view(2, L, G, S, hd)[:, 0].contiguous()).reshape(-1)
+                self.kv[:] = kv_words(kv_gpu.view(2, L, G, S, hd)[:, 0]).reshape(-1)
         self.tok = tok
         self.x0 = (wq["embed"][tok].astype(np.uint32) << 16).view(np.float32)
         self.cores = orc.num_threads()
@@ -298,7 +319,7 @@ def gate_and_kernel_time(shape, wd, pos, dec, kv, tok, keep, n_kernel=9):
     logits = dec.logits.cpu().numpy()
     tok_g = int(dec.next_token.item())
     L, G, S, hd = shape.n_layers, shape.n_kv_heads, shape.max_seq, shape.head_dim
-    rows = inp.bits(kv.view(2, L, G, S, hd)[:, 0, :, pos, :].contiguous())
+    rows = kv_words(kv.view(2, L, G, S, hd)[:, 0, :, pos, :])
     smp = OracleSample(shape, wd, pos, keep, tok, kv)
     parity = smp.gate(hidden, logits, tok_g, rows)
     ks = []
@@ -316,7 +337,7 @@ def run_one(workload, device, steps, warmup, peak, sync_mode=0, evict_l2=False):
     else:
         per, _ = time_device(dec, tok, pos, kv, steps, warmup)
     parity, kernel_us, _ = gate_and_kernel_time(shape, wd, pos, dec, kv, tok, keep)
-    b = inp.streamed_bytes(shape, wd, pos, quantize_lm_head=workload in QHEAD)
+    b = inp.streamed_bytes(shape, wd, pos, quantize_lm_head=workload in QHEAD, kv_dtype=kv_dtype_of(workload))
     us = float(np.mean(per))
     ach = b["total"] / (us * 1e-6) / 1e9
     res = {"workload": workload, "us_per_token": us if parity["pass"] else None, "median_us": float(np.median(per)),
@@ -389,7 +410,7 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     name, wd, pos = WORKLOADS[a.workload]
     shape = inp.SHAPES[name]
-    config = {"workload": f"{name} shape, {wd} weights{' (LM head quantised too)' if a.workload in QHEAD else ''}, batch 1, decode position {pos}, "
+    config = {"workload": f"{name} shape, {wd} weights{' (LM head quantised too)' if a.workload in QHEAD else ''}{', fp8 e4m3 KV cache' if a.workload in FP8KV else ''}, batch 1, decode position {pos}, "
                           f"{'pre-filled N(0,1) bf16 KV cache' if pos else 'empty KV cache'}, random-init N(0,0.02) weights",
               "l2": "inputs larger than L2: every step streams the whole weight set from HBM",
               "replicas": world}
@@ -474,7 +495,7 @@ def main():
 
     if rank == 0:
         peak, peak_src = measured_peak()
-        b = inp.streamed_bytes(shape, wd, pos, quantize_lm_head=a.workload in QHEAD)
+        b = inp.streamed_bytes(shape, wd, pos, quantize_lm_head=a.workload in QHEAD, kv_dtype=kv_dtype_of(a.workload))
         us = total_ms * 1e3 / a.steps
         achieved = b["total"] / (us * 1e-6) / 1e9
         plan = dec.plan()

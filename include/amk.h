@@ -27,7 +27,7 @@
 extern "C" {
 #endif
 
-#define AMK_ABI_VERSION 2u
+#define AMK_ABI_VERSION 3u
 
 typedef enum {
   AMK_OK = 0,
@@ -42,6 +42,9 @@ typedef enum {
 } amk_status;
 
 typedef enum { AMK_W_BF16 = 0, AMK_W_INT8 = 1, AMK_W_INT4 = 2, AMK_W_INT8_GROUPED = 3 } amk_wdtype;
+/* element type of the KV cache: bf16 (what the paper's kernels keep, Section 5), or fp8 e4m3 (a variant: the
+ * appended rows are rounded to nearest even, saturating at +-448, and attention reads the 8-bit entries) */
+typedef enum { AMK_KV_BF16 = 0, AMK_KV_FP8_E4M3 = 1 } amk_kvdtype;
 
 /* amk_config.flags */
 #define AMK_FLAG_DEBUG_HIDDEN 1u /* keep the residual stream after the embedding and after every layer */
@@ -112,6 +115,8 @@ typedef struct amk_config {
                                 no device).  The packed layout depends on it.                          */
   uint32_t l2_ahead;         /* ring tiles the producer requests into L2 beyond the ring (weight prefetch
                                 hint, as in the paper's Algorithm 1); 0 = automatic, 33 = off, max 32    */
+  uint32_t kv_dtype;         /* amk_kvdtype of the KV cache; the cache is K then V, each
+                                [L][n_kv][max_seq][head_dim] of that type                                */
 } amk_config;
 
 /*
@@ -186,9 +191,9 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* weights, void* p
  * inside one cooperative launch): embedding of `token`, L decoder layers at position `pos`, final norm,
  * LM head, greedy token.
  *   kv_cache_dev   DEVICE, caller-owned, amk_kv_bytes: K then V, each [L][n_kv_heads][max_seq][head_dim]
- *                  bf16, 16-byte aligned (rows are fetched with 16-byte bulk copies).  Entries [0, pos) must
- *                  be valid; the step writes slot `pos` of every layer (K after the rotation,
- *                  round-to-nearest-even) and reads [0, pos].
+ *                  of cfg.kv_dtype (bf16, or fp8 e4m3 bytes), 16-byte aligned (rows are fetched with 16-byte
+ *                  bulk copies).  Entries [0, pos) must be valid; the step writes slot `pos` of every layer
+ *                  (K after the rotation, round-to-nearest-even; fp8 saturates at +-448) and reads [0, pos].
  *   logits_dev     DEVICE float[vocab], 4-byte aligned, may be NULL
  *   next_token_dev DEVICE int32[1], 4-byte aligned, may be NULL; lowest index wins an exact tie
  * Asynchronous: returns after the launch.  Synchronous errors: INVALID_ARG (NULL handle or cache, misaligned

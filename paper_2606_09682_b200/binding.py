@@ -15,10 +15,12 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("AMK_LIB") or os.path.join(_HERE, "libamk.so")      # AMK_LIB: another build of the library
 
-AMK_ABI_VERSION = 2
+AMK_ABI_VERSION = 3
 AMK_OK, AMK_ERR_INVALID_ARG, AMK_ERR_UNSUPPORTED, AMK_ERR_CUDA, AMK_ERR_OOM = 0, 1, 2, 3, 4
 AMK_ERR_TIMEOUT, AMK_ERR_ABORTED, AMK_ERR_BAD_POS, AMK_ERR_BAD_TOKEN = 5, 6, 7, 8
 AMK_W_BF16, AMK_W_INT8, AMK_W_INT4, AMK_W_INT8_GROUPED = 0, 1, 2, 3
+AMK_KV_BF16, AMK_KV_FP8_E4M3 = 0, 1
+KVDTYPES = {"bf16": AMK_KV_BF16, "fp8": AMK_KV_FP8_E4M3}
 AMK_FLAG_DEBUG_HIDDEN = 1
 AMK_FLAG_TRACE = 2
 AMK_FLAG_MEASURED_SPLIT = 4
@@ -35,7 +37,7 @@ class amk_config(C.Structure):
                                           "tied_embeddings")] + [
         ("rms_eps", C.c_float), ("rope_theta", C.c_float)] + [
         (n, C.c_uint32) for n in ("wdtype", "group_size", "quantize_lm_head", "wait_timeout_us", "flags",
-                                  "stage_bytes", "n_stages", "max_inflight", "sync_mode", "n_blocks", "l2_ahead")]
+                                  "stage_bytes", "n_stages", "max_inflight", "sync_mode", "n_blocks", "l2_ahead", "kv_dtype")]
 
 
 _PP = C.POINTER(C.c_void_p)
@@ -111,7 +113,8 @@ def _check(code: int, what: str):
 
 def make_config(shape, wdtype: str = "bf16", flags: int = 0, wait_timeout_us: int = 0, stage_bytes: int = 0,
                 n_stages: int = 0, max_inflight: int = 0, group_size: int = 128, sync_mode: int = 1,
-                n_blocks: int = 0, l2_ahead: int = 0, quantize_lm_head: bool = False) -> amk_config:
+                n_blocks: int = 0, l2_ahead: int = 0, quantize_lm_head: bool = False,
+                kv_dtype: str = "bf16") -> amk_config:
     """``shape``: any object with hidden, n_layers, n_q_heads, n_kv_heads, head_dim, mlp, vocab, max_seq,
     tied, rms_eps, rope_theta attributes."""
     c = amk_config()
@@ -126,6 +129,7 @@ def make_config(shape, wdtype: str = "bf16", flags: int = 0, wait_timeout_us: in
     c.stage_bytes, c.n_stages, c.max_inflight = stage_bytes, n_stages, max_inflight
     c.sync_mode, c.n_blocks, c.l2_ahead = sync_mode, n_blocks, l2_ahead
     c.quantize_lm_head = int(bool(quantize_lm_head))
+    c.kv_dtype = KVDTYPES[kv_dtype]
     return c
 
 
@@ -271,14 +275,15 @@ class Decoder:
     def __init__(self, shape, weights: Dict, wdtype: str = "bf16", flags: int = 0, wait_timeout_us: int = 0,
                  stage_bytes: int = 0, n_stages: int = 0, max_inflight: int = 0, sync_mode: int = 1,
                  n_blocks: int = 0, l2_ahead: int = 0, device="cuda", guard_bytes: int = 0,
-                 quantize_lm_head: bool = False):
+                 quantize_lm_head: bool = False, kv_dtype: str = "bf16"):
         """``guard_bytes`` (a multiple of 256): the packed buffer, the workspace and the logits get that many bytes
         of a fixed pattern in front and behind, which ``guards_intact()`` checks -- a stand-in for a memory checker."""
         self.shape, self.wdtype = shape, wdtype
         self.device = torch.device(device)
         self.cfg = make_config(shape, wdtype, flags, wait_timeout_us, stage_bytes, n_stages, max_inflight,
                                sync_mode=sync_mode, n_blocks=n_blocks, l2_ahead=l2_ahead,
-                               quantize_lm_head=quantize_lm_head)
+                               quantize_lm_head=quantize_lm_head, kv_dtype=kv_dtype)
+        self.kv_dtype = kv_dtype
         self.quantize_lm_head = bool(quantize_lm_head)
         assert guard_bytes % 256 == 0
         self._guard = guard_bytes
@@ -326,11 +331,12 @@ class Decoder:
 
     def new_cache(self) -> torch.Tensor:
         n = amk_kv_bytes(self.cfg)
+        fp8 = self.kv_dtype == "fp8"
         if not self._guard:
-            return torch.zeros(n // 2, dtype=torch.bfloat16, device=self.device)
+            return torch.zeros(n if fp8 else n // 2, dtype=torch.uint8 if fp8 else torch.bfloat16, device=self.device)
         buf = self._alloc(n)
         buf.zero_()
-        return buf.view(torch.bfloat16)
+        return buf if fp8 else buf.view(torch.bfloat16)
 
     def plan(self) -> amk_plan:
         p = amk_plan()

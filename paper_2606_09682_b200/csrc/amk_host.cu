@@ -45,7 +45,7 @@ struct Plan {
 };
 
 struct WorkspaceLayout {
-  size_t status, phase_ctr, group_ctr, lm_ctr, next_ws, cand_val, cand_idx, x_a, x_b, qkv, o, m, m_amax, part, hidden, rope,
+  size_t status, phase_ctr, group_ctr, lm_ctr, next_ws, cand_val, cand_idx, x_a, x_b, qkv, o, m, part, hidden, rope,
       trace, ktime, slice_tab, bounds, smid_tab, calib, tile_begin, tiles, total;
 };
 
@@ -68,7 +68,7 @@ amk_status check_config(const amk_config* c) {
   if (c->l2_ahead > 33u) return AMK_ERR_INVALID_ARG;
   if (!c->hidden || !c->n_layers || !c->n_q_heads || !c->n_kv_heads || !c->mlp || !c->vocab || !c->max_seq)
     return AMK_ERR_INVALID_ARG;
-  if (c->wdtype > AMK_W_INT8_GROUPED || c->sync_mode > 2) return AMK_ERR_INVALID_ARG;
+  if (c->wdtype > AMK_W_INT8_GROUPED || c->sync_mode > 2 || c->kv_dtype > AMK_KV_FP8_E4M3) return AMK_ERR_INVALID_ARG;
   if (5ull * c->n_layers + 1 > 2047ull) return AMK_ERR_UNSUPPORTED;      // a tile entry keeps its task in 11 bits
   if (c->n_blocks > (uint32_t)kMaxBlocks) return AMK_ERR_INVALID_ARG;
   if (c->head_dim != 64 && c->head_dim != 128) return AMK_ERR_UNSUPPORTED;
@@ -207,7 +207,6 @@ WorkspaceLayout workspace_layout(const amk_config* c, const Plan& pl) {
   w.qkv = take((qd + 2 * kvd) * sizeof(ActPair));
   w.o = take(qd * sizeof(ActPair));
   w.m = take(I * sizeof(ActPair));
-  w.m_amax = take(kMaxBlocks * sizeof(ActPair));
   w.part = take((size_t)c->n_q_heads * kMaxChunks * (hd + 2) * sizeof(ActPair));
   w.hidden = take((L + 1) * H * 4);
   w.rope = take(S * (hd / 2) * sizeof(float2));
@@ -225,7 +224,7 @@ WorkspaceLayout workspace_layout(const amk_config* c, const Plan& pl) {
 }
 
 size_t kv_bytes_of(const amk_config* c) {
-  return 2ull * c->n_layers * c->n_kv_heads * c->max_seq * c->head_dim * 2ull;
+  return 2ull * c->n_layers * c->n_kv_heads * c->max_seq * c->head_dim * (c->kv_dtype == AMK_KV_FP8_E4M3 ? 1ull : 2ull);
 }
 
 }  // namespace
@@ -550,6 +549,7 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     // ---- kernel parameters that do not change from step to step ---------------------------------------
     KParams& p = h->base;
     p.H = H; p.L = L; p.nq = cfg->n_q_heads; p.nkv = cfg->n_kv_heads; p.hd = hd; p.I = I; p.V = cfg->vocab;
+    p.kv_esz = (cfg->kv_dtype == AMK_KV_FP8_E4M3) ? 1 : 2;
     p.S = cfg->max_seq; p.n_rep = n_rep; p.eps = cfg->rms_eps; p.flags = (int)cfg->flags;
     p.sync_mode = (cfg->sync_mode == 2) ? 0 : 1;      // kernel: 0 = counter joins as well, 1 = sequence numbers only
     for (int k = 0; k < 5; k++) p.shape[k] = h->pl.shape[k];
@@ -571,7 +571,6 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     p.rope = (const float2*)(h->ws + h->wl.rope);
     p.x_a = (ActPair*)(h->ws + h->wl.x_a); p.x_b = (ActPair*)(h->ws + h->wl.x_b);
     p.qkv = (ActPair*)(h->ws + h->wl.qkv); p.o = (ActPair*)(h->ws + h->wl.o); p.m = (ActPair*)(h->ws + h->wl.m);
-    p.m_amax = (ActPair*)(h->ws + h->wl.m_amax);
     p.part = (ActPair*)(h->ws + h->wl.part); p.hidden = (float*)(h->ws + h->wl.hidden);
     p.phase_ctr = (unsigned*)(h->ws + h->wl.phase_ctr); p.group_ctr = (unsigned*)(h->ws + h->wl.group_ctr);
     p.lm_ctr = (unsigned*)(h->ws + h->wl.lm_ctr); p.cand_val = (float*)(h->ws + h->wl.cand_val);
@@ -628,8 +627,8 @@ static amk_status launch_step(amk_handle* h, int32_t token, const int* token_ptr
   p.epoch = ++h->epoch;
   p.ctr_epoch = ++h->ctr_epoch;
   const size_t half = kv_bytes_of(&h->cfg) / 2;
-  p.kcache = (unsigned short*)kv;
-  p.vcache = (unsigned short*)((unsigned char*)kv + half);
+  p.kcache = (unsigned char*)kv;
+  p.vcache = (unsigned char*)kv + half;
   p.logits = logits;
   p.next_token = next_token;
   p.drop_phase = h->drop_phase;

@@ -81,8 +81,9 @@ struct KParams {
                                           // before the 32-bit sequence numbers could wrap)
   unsigned ctr_epoch;                     // steps since the counters were last zeroed
   // caller buffers
-  unsigned short* kcache;
-  unsigned short* vcache;
+  unsigned char* kcache;                  // K cache [L][n_kv][S][hd] of kv_esz-byte elements (2: bf16, 1: fp8 e4m3)
+  unsigned char* vcache;
+  int kv_esz;
   float* logits;
   int* next_token;
   // workspace
@@ -91,7 +92,6 @@ struct KParams {
   ActPair* qkv;
   ActPair* o;
   ActPair* m;
-  ActPair* m_amax;                        // [n_blocks] max |m| over each block's rows (integer-weight models)
   ActPair* part;                          // [nq][kMaxChunks][hd + 2]: a chunk's max, sum, unnormalised output
   float* hidden;                          // [(L+1)][H]
   unsigned* phase_ctr;                    // [5 L]

@@ -27,6 +27,7 @@
 // kernel's instruction footprint: with the stamps merely compiled in (and switched off at run time) a TinyLlama
 // step measured 4-9 % slower.  AMK_KERNEL / AMK_LAUNCH / AMK_ATTRS name the build's kernel and entry points.
 #include <cuda_fp16.h>
+#include <cuda_fp8.h>
 #include <cuda_runtime.h>
 #include <math_constants.h>
 
@@ -230,6 +231,32 @@ __device__ __forceinline__ float read_act(const KParams& p, bool& bad, const Act
     if (v.y != seq) bad = true;
   }
   return __uint_as_float(v.x);
+}
+
+// fp8 e4m3 cache entries: round to nearest even, saturating at +-448 (the hardware's conversion), and back (exact).
+__device__ __forceinline__ unsigned char f32_to_e4m3(float v) {
+  return (unsigned char)__nv_cvt_float_to_fp8(v, __NV_SATFINITE, __NV_E4M3);
+}
+__device__ __forceinline__ float e4m3_to_f32(unsigned char code) {
+  return __half2float(__half(__nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)code, __NV_E4M3)));
+}
+// Eight consecutive cache elements as fp32: 16 bytes of bf16, or 8 bytes of e4m3.
+template <bool FP8>
+__device__ __forceinline__ void cache8(const unsigned char* p8, float (&f)[8]) {
+  if (FP8) {
+    const uint2 w = *reinterpret_cast<const uint2*>(p8);
+    const unsigned v[2] = {w.x, w.y};
+#pragma unroll
+    for (int i = 0; i < 2; i++) {
+      const float2 a = __half22float2(__half2(__nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)(v[i] & 0xffffu), __NV_E4M3)));
+      const float2 b = __half22float2(__half2(__nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)(v[i] >> 16), __NV_E4M3)));
+      f[4 * i] = a.x; f[4 * i + 1] = a.y; f[4 * i + 2] = b.x; f[4 * i + 3] = b.y;
+    }
+  } else {
+    const uint4 w = *reinterpret_cast<const uint4*>(p8);
+    f[0] = bf16_lo(w.x); f[1] = bf16_hi(w.x); f[2] = bf16_lo(w.y); f[3] = bf16_hi(w.y);
+    f[4] = bf16_lo(w.z); f[5] = bf16_hi(w.z); f[6] = bf16_lo(w.w); f[7] = bf16_hi(w.w);
+  }
 }
 
 // (on the gate/up -> down critical path: the hardware's exp2 and reciprocal, ~1e-6 relative)
@@ -719,12 +746,21 @@ __device__ __forceinline__ bool gemv_op(Ctx& c, int kind_rt, int l) {
                 const bool is_v = vrow >= qd + kvd;
                 const int e = vrow - qd - (is_v ? kvd : 0);
                 const int g = e >> hs, dd = e & (p.hd - 1);
-                const unsigned short bits = f32_to_bf16_rne(y);
-                (is_v ? p.vcache : p.kcache)[((size_t)l * p.nkv + g) * p.S * p.hd + dd] = bits;
+                unsigned char* cache = is_v ? p.vcache : p.kcache;
+                const size_t idx = ((size_t)l * p.nkv + g) * p.S * p.hd + dd;
+                float stored;                              // the value the cache now holds
+                if (p.kv_esz == 2) {
+                  const unsigned short bits = f32_to_bf16_rne(y);
+                  reinterpret_cast<unsigned short*>(cache)[idx] = bits;
+                  stored = bf16_lo((unsigned)bits);
+                } else {
+                  const unsigned char code = f32_to_e4m3(y);
+                  cache[idx] = code;
+                  stored = e4m3_to_f32(code);
+                }
                 if (is_v) {
                   const unsigned oseq = seq_of(p, 5 * l + 1);
-                  for (int h = g * p.n_rep; h < (g + 1) * p.n_rep; h++)
-                    st_pair(p.o + (size_t)h * p.hd + dd, bf16_lo((unsigned)bits), oseq);
+                  for (int h = g * p.n_rep; h < (g + 1) * p.n_rep; h++) st_pair(p.o + (size_t)h * p.hd + dd, stored, oseq);
                 }
               }
             }
@@ -856,7 +892,7 @@ template <int HD>
 __device__ __noinline__ unsigned attn_general(const KParams& p, SmemHeader* sh, unsigned char* xs,
                                               const unsigned char* ring, int cta, int l, int g, int ch, int Lc, int C,
                                               bool bad_in, int stage, unsigned parity);
-template <int HD>
+template <int HD, bool FP8>
 __device__ __noinline__ unsigned attn_general_scalar(const KParams& p, SmemHeader* sh, unsigned char* xs,
                                                      const unsigned char* ring, int cta, int l, int g, int ch, int Lc,
                                                      int C, bool bad_in, int stage, unsigned parity);
@@ -897,6 +933,22 @@ __device__ __forceinline__ bool attn_task(const KParams& p, SmemHeader* sh, unsi
     const int ql = i & 3, ks = (i >> 2) % A.NKS, col = 2 * (n_rep & 3) + (i >> 2) / A.NKS;      // col in [2 (n_rep % 4), 8)
     A.qfrag[((A.n_sets - 1) * A.NKS + ks) * 32 + col * 4 + ql] = make_uint2(0u, 0u);
   }
+  // the new row's elements e and e + half: into the cache at its element type, and into shared memory as the bf16
+  // pattern of the value the cache now holds (an e4m3 value is exactly a bf16 value)
+  auto append2 = [&](unsigned char* cache, unsigned short* fresh, int e, float x0, float x1) {
+    unsigned short b0, b1;
+    const size_t at = (kvrow + p.pos) * HD;
+    if (p.kv_esz == 2) {
+      b0 = f32_to_bf16_rne(x0); b1 = f32_to_bf16_rne(x1);
+      unsigned short* dst = reinterpret_cast<unsigned short*>(cache) + at;
+      dst[e] = b0; dst[e + half] = b1;
+    } else {
+      const unsigned char c0 = f32_to_e4m3(x0), c1 = f32_to_e4m3(x1);
+      cache[at + e] = c0; cache[at + e + half] = c1;
+      b0 = f32_to_bf16_rne(e4m3_to_f32(c0)); b1 = f32_to_bf16_rne(e4m3_to_f32(c1));
+    }
+    fresh[e] = b0; fresh[e + half] = b1;
+  };
   for (int i = c.tid; i < n_items; i += kConsumerThreads) {
     const int h = i / half, e = i - h * half;
     const ActPair* base = (h < n_rep) ? p.qkv + (size_t)(g * n_rep + h) * HD
@@ -914,15 +966,9 @@ __device__ __forceinline__ bool attn_task(const KParams& p, SmemHeader* sh, unsi
       A.put_q(h, e, q0);                               // and as bf16 high / low parts in tensor-core B-fragment order
       A.put_q(h, e + half, q1);
     } else if (h == n_rep) {
-      const unsigned short k0 = f32_to_bf16_rne(a * cs.x - b * cs.y), k1 = f32_to_bf16_rne(b * cs.x + a * cs.y);
-      unsigned short* dst = p.kcache + (kvrow + p.pos) * HD;
-      dst[e] = k0; dst[e + half] = k1;
-      knew[e] = k0; knew[e + half] = k1;
+      append2(p.kcache, knew, e, a * cs.x - b * cs.y, b * cs.x + a * cs.y);
     } else {
-      const unsigned short v0 = f32_to_bf16_rne(a), v1 = f32_to_bf16_rne(b);
-      unsigned short* dst = p.vcache + (kvrow + p.pos) * HD;
-      dst[e] = v0; dst[e + half] = v1;
-      vnew[e] = v0; vnew[e + half] = v1;
+      append2(p.vcache, vnew, e, a, b);
     }
   }
   c.bad = cons_sync_or(c.bad);           // q and the new cache row are in shared memory
@@ -940,9 +986,12 @@ __device__ __forceinline__ bool attn_task(const KParams& p, SmemHeader* sh, unsi
   }
   // tensor-core kernel when the accumulators of all sets of four heads fit the registers (every shape measured
   // here: up to 8 q heads per kv head at head_dim 64, 4 at 128); otherwise the scalar one
-  const unsigned r = (A.n_sets * A.NKS <= 8)
+  // (an fp8 cache: the scalar kernel, which converts the 8-bit entries as it reads them)
+  const unsigned r = (p.kv_esz == 1)
+                         ? attn_general_scalar<HD, true>(p, sh, xs, ring, cta, l, g, ch, Lc, C, c.bad, stage, parity)
+                     : (A.n_sets * A.NKS <= 8)
                          ? attn_general<HD>(p, sh, xs, ring, cta, l, g, ch, Lc, C, c.bad, stage, parity)
-                         : attn_general_scalar<HD>(p, sh, xs, ring, cta, l, g, ch, Lc, C, c.bad, stage, parity);
+                         : attn_general_scalar<HD, false>(p, sh, xs, ring, cta, l, g, ch, Lc, C, c.bad, stage, parity);
   stage = (int)((r >> 1) & 0x7fu);
   parity = (r >> 8) & 1u;
   return (r & 1u) != 0u;
@@ -1226,7 +1275,7 @@ __device__ __noinline__ unsigned attn_general(const KParams& p, SmemHeader* sh, 
 //      are summed by shuffles, then across warps through shared memory.
 // The chunk's (max, sum, unnormalised output) is the final output for a single chunk, else a partial.
 // Returns bad | stage << 1 | parity << 8 (the ring position moves on by the tiles walked).
-template <int HD>
+template <int HD, bool FP8>
 __device__ __noinline__ unsigned attn_general_scalar(const KParams& p, SmemHeader* sh, unsigned char* xs,
                                                      const unsigned char* ring, int cta, int l, int g, int ch, int Lc,
                                                      int C, bool bad_in, int stage, unsigned parity) {
@@ -1243,7 +1292,8 @@ __device__ __noinline__ unsigned attn_general_scalar(const KParams& p, SmemHeade
   const bool owns_new = (j1 == n_pos);
   const int rows = min(j1, p.pos) - j0;                // rows that come from the cache
   const int n = j1 - j0;                               // + the new row, held in shared memory
-  const int rpt = p.stage_bytes / (HD * 2);            // cache rows per ring tile
+  constexpr int RB = HD * (FP8 ? 1 : 2);               // bytes of a cache row
+  const int rpt = p.stage_bytes / RB;                  // cache rows per ring tile
   const int n_t = (rows + rpt - 1) / rpt;              // ring tiles of K (and again of V)
   const AttnScratch<HD> AS(xs, n_rep);
   float* qs = AS.qs;                                   // [n_rep][HD]
@@ -1269,9 +1319,7 @@ __device__ __noinline__ unsigned attn_general_scalar(const KParams& p, SmemHeade
 #pragma unroll
       for (int e = 0; e < 8; e++) q[hh][e] = busy ? qs[h * HD + dl * 8 + e] : 0.f;
     }
-    auto score_row = [&](const uint4 kq, int t) {
-      const float kf[8] = {bf16_lo(kq.x), bf16_hi(kq.x), bf16_lo(kq.y), bf16_hi(kq.y),
-                           bf16_lo(kq.z), bf16_hi(kq.z), bf16_lo(kq.w), bf16_hi(kq.w)};
+    auto score_row = [&](const float (&kf)[8], int t) {
 #pragma unroll
       for (int hh = 0; hh < 4; hh++) {
         float s = kf[0] * q[hh][0];
@@ -1290,16 +1338,20 @@ __device__ __noinline__ unsigned attn_general_scalar(const KParams& p, SmemHeade
         const int r_t = min(rpt, rows - k * rpt);
         for (int r0 = wi * RPW; r0 < r_t; r0 += wph * RPW) {            // (warp-uniform bounds: shuffles inside)
           const int r = r0 + sub;
-          const uint4 kq = *reinterpret_cast<const uint4*>(tile + (size_t)min(r, r_t - 1) * (HD * 2) + dl * 16);
-          score_row(kq, r < r_t ? k * rpt + r : -1);
+          float kf[8];
+          cache8<FP8>(tile + (size_t)min(r, r_t - 1) * RB + dl * (RB / NC), kf);
+          score_row(kf, r < r_t ? k * rpt + r : -1);
         }
       }
       __syncwarp();
       if (c.lane == 0 && !c.bad) mbar_arrive(&c.sh->empty[stage]);
       if (++stage == S_) { stage = 0; parity ^= 1u; }
     }
-    if (owns_new && busy && wi == 0 && !c.bad)                            // the new row, from shared memory
-      score_row(reinterpret_cast<const uint4*>(knew)[dl], sub == 0 ? n - 1 : -1);
+    if (owns_new && busy && wi == 0 && !c.bad) {                          // the new row, from shared memory
+      float kf[8];
+      cache8<false>(reinterpret_cast<const unsigned char*>(knew) + dl * 16, kf);
+      score_row(kf, sub == 0 ? n - 1 : -1);
+    }
   }
   c.bad = cons_sync_or(c.bad);
   if (c.tid == 0) stamp(p, cta, 5 * l + 1, AMK_TR_PASS_BEGIN);
@@ -1329,9 +1381,7 @@ __device__ __noinline__ unsigned attn_general_scalar(const KParams& p, SmemHeade
     for (int hh = 0; hh < 4; hh++)
 #pragma unroll
       for (int e = 0; e < 8; e++) acc[hh][e] = 0.f;
-    auto add_row = [&](const uint4 vq, int t) {
-      const float vf[8] = {bf16_lo(vq.x), bf16_hi(vq.x), bf16_lo(vq.y), bf16_hi(vq.y),
-                           bf16_lo(vq.z), bf16_hi(vq.z), bf16_lo(vq.w), bf16_hi(vq.w)};
+    auto add_row = [&](const float (&vf)[8], int t) {
 #pragma unroll
       for (int hh = 0; hh < 4; hh++) {
         const float pw = S[min(hb * 4 + hh, n_rep - 1) * Lc + t];
@@ -1345,14 +1395,21 @@ __device__ __noinline__ unsigned attn_general_scalar(const KParams& p, SmemHeade
       if (busy && !c.bad) {
         const unsigned char* tile = ring + (size_t)stage * p.stage_bytes;
         const int r_t = min(rpt, rows - k * rpt);
-        for (int r = wi * RPW + sub; r < r_t; r += wph * RPW)
-          add_row(*reinterpret_cast<const uint4*>(tile + (size_t)r * (HD * 2) + dl * 16), k * rpt + r);
+        for (int r = wi * RPW + sub; r < r_t; r += wph * RPW) {
+          float vf[8];
+          cache8<FP8>(tile + (size_t)r * RB + dl * (RB / NC), vf);
+          add_row(vf, k * rpt + r);
+        }
       }
       __syncwarp();
       if (c.lane == 0 && !c.bad) mbar_arrive(&c.sh->empty[stage]);
       if (++stage == S_) { stage = 0; parity ^= 1u; }
     }
-    if (owns_new && busy && wi == 0 && sub == 0 && !c.bad) add_row(reinterpret_cast<const uint4*>(vnew)[dl], n - 1);
+    if (owns_new && busy && wi == 0 && sub == 0 && !c.bad) {
+      float vf[8];
+      cache8<false>(reinterpret_cast<const unsigned char*>(vnew) + dl * 16, vf);
+      add_row(vf, n - 1);
+    }
     // sum the lane groups of the warp, then leave the warp's partial in shared memory
 #pragma unroll
     for (int o = NC; o < 32; o <<= 1)
@@ -1489,13 +1546,13 @@ __device__ __noinline__ void producer(const KParams& p, SmemHeader* sh, unsigned
           if (tt < p.nkv * C) {
             const int g = tt / C, ch = tt - g * C;
             const int j0 = ch * Lc, rows = min(p.pos, j0 + Lc) - j0;
-            const int rpt = p.stage_bytes / (p.hd * 2);
-            const size_t first = (((size_t)l * p.nkv + g) * p.S + j0) * p.hd;      // in elements
+            const int rb = p.hd * p.kv_esz;                                         // bytes of a cache row
+            const int rpt = p.stage_bytes / rb;
+            const size_t first = (((size_t)l * p.nkv + g) * p.S + j0) * rb;        // in bytes
             for (int which = 0; which < 2 && ok; which++) {
-              const unsigned short* cache = which ? p.vcache : p.kcache;
+              const unsigned char* cache = which ? p.vcache : p.kcache;
               for (int r0 = 0; r0 < rows && ok; r0 += rpt)
-                issue(reinterpret_cast<const unsigned char*>(cache + first + (size_t)r0 * p.hd),
-                      (unsigned)(min(rpt, rows - r0) * p.hd * 2));
+                issue(cache + first + (size_t)r0 * rb, (unsigned)(min(rpt, rows - r0) * rb));
             }
           }
         }

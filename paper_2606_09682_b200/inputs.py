@@ -122,14 +122,18 @@ def make_token(shape: ModelShape, seed: int) -> int:
     return int(torch.randint(0, shape.vocab, (1,), generator=g).item())
 
 
-def make_kv_prefill(shape: ModelShape, seed: int, pos: int, device="cpu", std: float = 1.0) -> torch.Tensor:
+def make_kv_prefill(shape: ModelShape, seed: int, pos: int, device="cpu", std: float = 1.0,
+                    kv_dtype: str = "bf16") -> torch.Tensor:
     """The whole cache buffer (K then V, each [L][n_kv][max_seq][hd] bf16) with positions [0, pos) drawn
-    i.i.d. N(0, std^2) and every other slot zero."""
+    i.i.d. N(0, std^2) and every other slot zero.  ``kv_dtype="fp8"``: the same draws as e4m3 codes (uint8; torch's
+    conversion -- any valid code is a valid input)."""
     dev = torch.device(device)
     L, g_, S, hd = shape.n_layers, shape.n_kv_heads, shape.max_seq, shape.head_dim
     kv = torch.zeros((2, L, g_, S, hd), dtype=torch.bfloat16, device=dev)
     if pos > 0:
         kv[:, :, :, :pos, :] = _normal_bf16((2, L, g_, pos, hd), std, seed, 9, dev)
+    if kv_dtype == "fp8":
+        return kv.to(torch.float32).to(torch.float8_e4m3fn).view(torch.uint8).view(-1)
     return kv.view(-1)
 
 
@@ -152,7 +156,7 @@ def weights_to_numpy(w: Dict) -> Dict:
 
 
 def streamed_bytes(shape: ModelShape, wdtype: str = "bf16", pos: int = 0, group: int = 128,
-                   quantize_lm_head: bool = False) -> Dict[str, float]:
+                   quantize_lm_head: bool = False, kv_dtype: str = "bf16") -> Dict[str, float]:
     """Algorithmic bytes one decode step must move: weights + scales + KV read/write + activations.
     ``quantize_lm_head``: the LM head is streamed at the layers' width (with its scales) instead of as bf16."""
     H, L, I, V = shape.hidden, shape.n_layers, shape.mlp, shape.vocab
@@ -178,6 +182,7 @@ def streamed_bytes(shape: ModelShape, wdtype: str = "bf16", pos: int = 0, group:
         head, head_sc = 1.0 * V * H, 4.0 * V * H / group
     weights = L * wl + head + 2.0 * (2 * L + 1) * H + 2.0 * H            # linears + LM head + norms + one embedding row
     scales = L * sc + head_sc
-    kv = 2.0 * L * nkv * hd * 2 * pos + 2.0 * L * nkv * hd * 2
+    kv_esz = 1.0 if kv_dtype == "fp8" else 2.0
+    kv = 2.0 * L * nkv * hd * kv_esz * pos + 2.0 * L * nkv * hd * kv_esz
     act = 4.0 * (L * (4 * H + (nq + 2 * nkv) * hd + nq * hd + 2 * I) + 2 * H) + 4.0 * V
     return {"weights": weights, "scales": scales, "kv": kv, "act": act, "total": weights + scales + kv + act}

@@ -30,13 +30,26 @@ def bf16_ulp_distance(a_bits, b_bits):
     return np.abs(key(a_bits) - key(b_bits))
 
 
-def oracle_model(shape, weights_gpu, wdtype, quantize_lm_head=False):
+def kv_words(kv_gpu):
+    """The cache as the oracle keeps it: one 16-bit word per element (a bf16 bit pattern, or an e4m3 code)."""
+    if kv_gpu.dtype == torch.uint8:
+        return kv_gpu.cpu().numpy().astype(np.uint16)
+    return kv_gpu.view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def e4m3_f32(codes):
+    c = torch.from_numpy(np.ascontiguousarray(codes).astype(np.uint8))
+    return c.view(torch.float8_e4m3fn).to(torch.float32).numpy()
+
+
+def oracle_model(shape, weights_gpu, wdtype, quantize_lm_head=False, kv_dtype="bf16"):
     """The oracle's model of the same seeded bf16 weights, quantised by the oracle's own quantiser."""
     wnp = inp.weights_to_numpy(weights_gpu)
     wq = orc.quantize_weights(wnp, WD[wdtype], 128)
     if quantize_lm_head:
         wq = orc.quantize_lm_head(wq, WD[wdtype], 128, tied=shape.tied)
-    return orc.Model(shape, wq, wdtype=WD[wdtype], group=128, quantize_lm_head=quantize_lm_head), wq
+    return orc.Model(shape, wq, wdtype=WD[wdtype], group=128, quantize_lm_head=quantize_lm_head,
+                     kv_dtype=orc.KV_E4M3 if kv_dtype == "fp8" else orc.KV_BF16), wq
 
 
 def check_argmax(logits_oracle, tok_gpu):
@@ -59,13 +72,18 @@ def max_err(a, b):
     return float(np.abs(a - b).max() / max(np.abs(b).max(), 1e-30))
 
 
-def check_kv_rows(rows_gpu, rows_own):
-    """The appended K / V rows of both sides, as bf16 bit patterns of the same shape [..., hd].  They are roundings
+def check_kv_rows(rows_gpu, rows_own, fp8=False):
+    """The appended K / V rows of both sides, as bf16 bit patterns (e4m3 codes) of the same shape [..., hd].  They are roundings
     of fp32 values that agree to ~1e-6, so they are equal or neighbours -- except where the value itself is
     rounding noise around zero (there a bf16 step is far smaller than that 1e-6): such entries must be tiny
     against their row.  Returns (largest distance in bf16 steps, fraction one step apart, number further apart)."""
-    d = bf16_ulp_distance(rows_gpu, rows_own)
-    g_f, o_f = bf16_f32(rows_gpu), bf16_f32(rows_own)
+    if fp8:
+        key = lambda x: np.where(x & 0x80, -(x & 0x7F).astype(np.int32), (x & 0x7F).astype(np.int32))
+        d = np.abs(key(np.asarray(rows_gpu)) - key(np.asarray(rows_own)))
+        g_f, o_f = e4m3_f32(rows_gpu), e4m3_f32(rows_own)
+    else:
+        d = bf16_ulp_distance(rows_gpu, rows_own)
+        g_f, o_f = bf16_f32(rows_gpu), bf16_f32(rows_own)
     row_scale = np.abs(o_f).max(axis=-1, keepdims=True)
     far = d > 1
     assert not (far & (np.abs(g_f - o_f) > KV_NEAR_ZERO * row_scale)).any(), (int(d.max()), int(far.sum()))
@@ -84,7 +102,7 @@ def compare_step(shape, dec, model, token, pos, kv_gpu, kv_cpu, check_hidden=Tru
     dec.amk_decode_step(token, pos, kv_gpu)
     st, msg = dec.amk_last_status()
     assert st == 0, msg
-    kvg = kv_gpu.view(torch.int16).cpu().numpy().view(np.uint16).reshape(2, L, G, S, hd)
+    kvg = kv_words(kv_gpu).reshape(2, L, G, S, hd)
     rows_gpu = np.ascontiguousarray(kvg[:, :, :, pos, :])
     logits_o, tok_o, hidden_o = model.decode_step(token, pos, kv_cpu, want_hidden=check_hidden, rows_pref=rows_gpu)
     logits_g = dec.logits.cpu().numpy()
@@ -110,7 +128,8 @@ def compare_step(shape, dec, model, token, pos, kv_gpu, kv_cpu, check_hidden=Tru
     mask[pos] = False
     assert np.array_equal(kvg[:, :, :, mask, :], kvb[:, :, :, mask, :]), "a slot other than pos changed"
     # ... and the new rows are the oracle's own roundings or their neighbours
-    out["kv_ulp_max"], out["kv_one_step_frac"], out["kv_far"] = check_kv_rows(rows_gpu, model.rows_own.reshape(rows_gpu.shape))
+    out["kv_ulp_max"], out["kv_one_step_frac"], out["kv_far"] = check_kv_rows(
+        rows_gpu, model.rows_own.reshape(rows_gpu.shape), fp8=kv_gpu.dtype == torch.uint8)
     # keep both caches identical from here on so later steps compare like with like
-    kv_cpu[:] = kv_gpu.view(torch.int16).cpu().numpy().view(np.uint16)
+    kv_cpu[:] = kv_words(kv_gpu)
     return out

@@ -113,6 +113,18 @@ def test_tinyllama_shape(amk, wdtype, pos):
     dec.close()
 
 
+@pytest.mark.parametrize("wdtype,pos", [("bf16", 1024), ("int8", 0), ("int4", 300)])
+def test_tinyllama_shape_fp8_cache(amk, wdtype, pos):
+    """The TinyLlama shape with an fp8 (e4m3) KV cache: the whole step against the oracle with the same cache type."""
+    shape, w, _, dec = _build(amk, "tinyllama_1b", wdtype, 0xA3C7, kv_dtype="fp8")
+    model, _ = gc.oracle_model(shape, w, wdtype, kv_dtype="fp8")
+    kv_g = inp.make_kv_prefill(shape, 0xA3C7, pos, device="cuda", kv_dtype="fp8")
+    kv_c = gc.kv_words(kv_g).copy()
+    r = gc.compare_step(shape, dec, model, inp.make_token(shape, 0xA3C7), pos, kv_g, kv_c)
+    print("tinyllama fp8 cache", wdtype, pos, r)
+    dec.close()
+
+
 @pytest.mark.parametrize("wdtype,pos", [("int8", 0), ("int4", 200), ("int8g", 0)])
 def test_tinyllama_shape_quantised_lm_head(amk, wdtype, pos):
     shape, w, _, dec = _build(amk, "tinyllama_1b", wdtype, 0xA3C2, quantize_lm_head=True)

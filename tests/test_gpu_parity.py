@@ -11,15 +11,16 @@ pytestmark = pytest.mark.gpu
 import gpu_common as gc  # noqa: E402
 
 
-def _setup(name, wdtype, seed, std=0.05, norm_jitter=0.1, quantize_lm_head=False, **kw):
+def _setup(name, wdtype, seed, std=0.05, norm_jitter=0.1, quantize_lm_head=False, kv_dtype="bf16", **kw):
     from paper_2606_09682_b200 import binding as amk
     shape = inp.SHAPES[name]
     w = inp.make_weights(shape, seed, device="cuda", std=std, norm_jitter=norm_jitter)
     wq = amk.quantize_weights(w, wdtype)
     if quantize_lm_head:
         wq = amk.quantize_lm_head(wq, wdtype, shape.tied)
-    dec = amk.Decoder(shape, wq, wdtype, flags=amk.AMK_FLAG_DEBUG_HIDDEN, quantize_lm_head=quantize_lm_head, **kw)
-    model, _ = gc.oracle_model(shape, w, wdtype, quantize_lm_head)
+    dec = amk.Decoder(shape, wq, wdtype, flags=amk.AMK_FLAG_DEBUG_HIDDEN, quantize_lm_head=quantize_lm_head,
+                      kv_dtype=kv_dtype, **kw)
+    model, _ = gc.oracle_model(shape, w, wdtype, quantize_lm_head, kv_dtype)
     return shape, dec, model
 
 
@@ -55,6 +56,27 @@ def test_quantised_lm_head(name, wdtype):
         tok = int(rng.integers(0, shape.vocab))
         r = gc.compare_step(shape, dec, model, tok, pos, kv_g, kv_c)
         print(name, wdtype, "quantised head", pos, r)
+    dec.close()
+
+
+@pytest.mark.parametrize("name,wdtype", [("mini", "bf16"), ("mini_ragged", "bf16"), ("mini_hd128", "int8"), ("mini_wide", "int4")])
+def test_fp8_cache_multi_step_and_prefilled(name, wdtype):
+    """kv_dtype = fp8 (e4m3): appended rows are the oracle's e4m3 roundings or their neighbours, attention reads the
+    8-bit entries -- from an empty cache over a few positions, then on a pre-filled cache with several chunks, a
+    ragged tail, a chunk boundary and the last slot."""
+    shape, dec, model = _setup(name, wdtype, seed=28, kv_dtype="fp8")
+    kv_g, kv_c = dec.new_cache(), model.new_cache()
+    rng = np.random.default_rng(5)
+    for pos in range(5):
+        tok = int(rng.integers(0, shape.vocab))
+        r = gc.compare_step(shape, dec, model, tok, pos, kv_g, kv_c)
+        print(name, wdtype, "fp8 cache", pos, r)
+    tok = inp.make_token(shape, 12)
+    for pos in (31, 32, 77, 200 if shape.max_seq > 200 else shape.max_seq - 2, shape.max_seq - 1):
+        kv_g = inp.make_kv_prefill(shape, 13, pos, device="cuda", kv_dtype="fp8")
+        kv_c = gc.kv_words(kv_g).copy()
+        r = gc.compare_step(shape, dec, model, tok, pos, kv_g, kv_c)
+        print(name, wdtype, "fp8 cache, pre-filled", pos, r)
     dec.close()
 
 
