@@ -105,7 +105,7 @@ typedef struct amk_config {
   /* tuning knobs, 0 = automatic */
   uint32_t stage_bytes;      /* bytes per shared-memory ring stage (multiple of 1024)                  */
   uint32_t n_stages;         /* ring depth                                                             */
-  uint32_t max_inflight;     /* bulk copies a block keeps in flight (<= n_stages; 0 = default 3)        */
+  uint32_t max_inflight;     /* bulk copies a block keeps in flight (<= n_stages; 0 = default 2)        */
   uint32_t sync_mode;        /* 0 = automatic = 1.  1: activations carry sequence numbers, nothing else orders
                                 the tasks (no counters, no fences): the mode every published figure uses.
                                 2: as 1, AND every task ends with a release-increment that the next task's

@@ -450,9 +450,10 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
       status = AMK_ERR_UNSUPPORTED;
       goto fail;
     }
-    // default: three copies in flight per block -- enough to saturate HBM from 148 blocks; more only deepens the
-    // memory system's queues, which every dependency-carrying load then waits behind (measured: 3 beats 5 by 2-4 %)
-    uint32_t max_inflight = cfg->max_inflight ? cfg->max_inflight : 3;
+    // default: two copies of 32 KB in flight per block -- enough to saturate HBM from 148 blocks; more only deepens
+    // the memory system's queues, which every dependency-carrying load then waits behind (measured: 3 beats 5 by
+    // 2-4 %, 2 beats 3 by 0.5-1.3 % on most shapes and ties on the rest)
+    uint32_t max_inflight = cfg->max_inflight ? cfg->max_inflight : 2;
     if (max_inflight > n_stages) max_inflight = n_stages;
     const size_t smem_bytes = hdr + act + (size_t)n_stages * stage_bytes;
     int per_sm = 0;

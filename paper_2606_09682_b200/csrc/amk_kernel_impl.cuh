@@ -1760,7 +1760,14 @@ static DecodeKernel pick_kernel(int wdtype, int hd) {
 
 cudaError_t AMK_ATTRS(int wdtype, int hd, size_t smem_bytes, int* max_blocks_per_sm) {
   DecodeKernel k = pick_kernel(wdtype, hd);
-  cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+  // the device's limit, not this handle's need: a handle created later with a smaller plan must not lower the
+  // attribute under a handle that is still in use
+  int dev = 0, optin = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  if (e != cudaSuccess) return e;
+  if ((size_t)optin < smem_bytes) return cudaErrorInvalidValue;
+  e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, optin);
   if (e != cudaSuccess) return e;
   return cudaOccupancyMaxActiveBlocksPerMultiprocessor(max_blocks_per_sm, k, kThreads, smem_bytes);
 }

@@ -284,3 +284,26 @@ def test_knob_search_on_a_small_grid(amk):
         if t.latency_us is not None:
             assert t.latency_us >= floor_us
     assert res["best_us"] >= floor_us
+
+
+def test_handles_with_different_shared_memory_plans_coexist(amk):
+    """A handle created later with a smaller shared-memory plan (smaller ring stages) must not break an earlier
+    handle's launches: both step, alternately, and each repeats its own result bit for bit."""
+    shape = inp.SHAPES["mini_wide"]
+    w = inp.make_weights(shape, 61, device="cuda")
+    wq = amk.quantize_weights(w, "int4")
+    big = amk.Decoder(shape, wq, "int4")
+    small = amk.Decoder(shape, wq, "int4", stage_bytes=8192, n_stages=2)
+    assert small.plan().smem_bytes < big.plan().smem_bytes
+    kv_b, kv_s = big.new_cache(), small.new_cache()
+    outs = []
+    for _ in range(2):
+        for dec, kv in ((big, kv_b), (small, kv_s)):
+            dec.amk_decode_step(7, 0, kv)
+            st, msg = dec.amk_last_status()
+            assert st == 0, msg
+            outs.append(dec.logits.clone())
+    assert torch.equal(outs[0], outs[2]) and torch.equal(outs[1], outs[3])
+    assert torch.allclose(outs[0], outs[1], rtol=0, atol=1e-3 * float(outs[0].abs().max()))
+    big.close()
+    small.close()
