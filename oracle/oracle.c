@@ -16,12 +16,17 @@
  * Arithmetic: activations are stored as fp32; every dot product, sum of squares and softmax sum is
  * accumulated in fp64; the KV cache holds bf16 (round to nearest even at append) and attention reads
  * the rounded entries, including the one appended in the same step.
+ * Variants beyond the paper's text, each the same step with one storage type changed: grouped int8
+ * weights (wdtype 3: the int8 rule per row and group of columns; Section 7 mentions dequantising "per
+ * group") and an fp8 e4m3 KV cache (kv_dtype 1: entries rounded to nearest even, saturating at +-448).
  *
  * Parity pins (tests/test_oracle_*.py): RMSNorm closed forms; RoPE pair-norm preservation, the pos=0
  * identity and hand values; softmax rows summing to one; attention at pos 0 returning the cached V;
  * split-K combine equal to the unsplit result; exact-integer GEMVs; integer pack/unpack round trips and
- * hand-worked quantiser rows; a second, dense, cache-free recomputation of a 2-layer hidden-64 toy; a
- * library cross-check against a random-init transformers LlamaForCausalLM.
+ * hand-worked quantiser rows (per row and per group); the e4m3 conversions against torch's float8_e4m3fn
+ * (all codes, all midpoints, saturation); a second, dense, cache-free recomputation of a 2-layer
+ * hidden-64 toy (also with every quantised weight type and with the fp8 cache); a library cross-check
+ * against a random-init transformers LlamaForCausalLM.
  * Parity unpinned: whether an *untied* LM head stays bf16 in the quantised variants is not fixed by the
  * paper; both readings are implemented (quantize_lm_head 0 / 1) and each is pinned against the dense form,
  * but which of the two the paper's kernels used cannot be pinned from its text.

@@ -173,7 +173,7 @@ def main():
 
     ap = argparse.ArgumentParser()
     ap.add_argument("--shape", default="tinyllama_1b", choices=sorted(inp.SHAPES))
-    ap.add_argument("--wdtype", default="bf16", choices=["bf16", "int8", "int4"])
+    ap.add_argument("--wdtype", default="bf16", choices=["bf16", "int8", "int4", "int8g"])
     ap.add_argument("--pos", type=int, default=0)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--max-trials", type=int, default=24)

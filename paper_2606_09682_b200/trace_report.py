@@ -94,7 +94,7 @@ def report(tr, shape, pos, cycles):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--shape", default="tinyllama_1b", choices=sorted(inp.SHAPES))
-    ap.add_argument("--wdtype", default="bf16", choices=["bf16", "int8", "int4"])
+    ap.add_argument("--wdtype", default="bf16", choices=["bf16", "int8", "int4", "int8g"])
     ap.add_argument("--pos", type=int, default=0)
     ap.add_argument("--cycles", action="store_true")
     ap.add_argument("--sync-mode", type=int, default=1)
