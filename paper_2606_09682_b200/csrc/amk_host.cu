@@ -88,7 +88,11 @@ amk_status check_config(const amk_config* c) {
   return AMK_OK;
 }
 
-uint32_t stage_bytes_of(const amk_config* c) { return c->stage_bytes ? c->stage_bytes : 32768u; }
+// Ring stage size.  Default 32 KB; 48 KB for int4, whose consumers do the most work per byte: fewer, larger tiles
+// mean fewer waits and arrivals per unit (knob search: Llama-3-8B int4 1254 -> 1222 us; no gain for the others).
+uint32_t stage_bytes_of(const amk_config* c) {
+  return c->stage_bytes ? c->stage_bytes : (c->wdtype == AMK_W_INT4 ? 49152u : 32768u);
+}
 
 // `weights`: relative streaming rate of each slot (nullptr: equal shares).
 Plan make_plan(const amk_config* c, int n_blocks, const double* weights, bool with_tiles,
@@ -452,8 +456,8 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     }
     // default: two copies of 32 KB in flight per block -- enough to saturate HBM from 148 blocks; more only deepens
     // the memory system's queues, which every dependency-carrying load then waits behind (measured: 3 beats 5 by
-    // 2-4 %, 2 beats 3 by 0.5-1.3 % on most shapes and ties on the rest)
-    uint32_t max_inflight = cfg->max_inflight ? cfg->max_inflight : 2;
+    // 2-4 %, 2 beats 3 by 0.5-1.3 % on most shapes and ties on the rest); int4 (three 48 KB stages): all three
+    uint32_t max_inflight = cfg->max_inflight ? cfg->max_inflight : (cfg->wdtype == AMK_W_INT4 ? 3 : 2);
     if (max_inflight > n_stages) max_inflight = n_stages;
     const size_t smem_bytes = hdr + act + (size_t)n_stages * stage_bytes;
     int per_sm = 0;
@@ -580,7 +584,14 @@ amk_status amk_create(const amk_config* cfg, const amk_weights* wts, void* packe
     p.trace = (cfg->flags & AMK_FLAG_TRACE) ? (unsigned long long*)(h->ws + h->wl.trace) : nullptr;
     p.ktime = (unsigned long long*)(h->ws + h->wl.ktime);
     p.stage_bytes = (int)stage_bytes; p.n_stages = (int)n_stages; p.max_inflight = (int)max_inflight;
-    p.l2_ahead = cfg->l2_ahead == 0 ? 6 : (cfg->l2_ahead > 32 ? 0 : (int)cfg->l2_ahead);
+    // L2 look-ahead, automatic: two tiles beyond the ring; six where a layer streams so much per block (more than
+    // 2 MB: Llama-3-8B bf16) that the step runs at the HBM rate and the deeper look-ahead keeps HBM busier
+    // (measured: 2 beats 6 by 0.5-1.6 % on the dependency-bound shapes, 6 beats 2 by 0.7 % on that one)
+    {
+      const double per_block = (double)(h->pl.weight_stream_bytes) / (L > 0 ? L : 1) / (double)n_blocks;
+      const int automatic = (cfg->wdtype == AMK_W_BF16 && per_block > 2.0e6) ? 6 : 2;
+      p.l2_ahead = cfg->l2_ahead == 0 ? automatic : (cfg->l2_ahead > 32 ? 0 : (int)cfg->l2_ahead);
+    }
     p.act_bytes = (int)act;
     p.timeout_ns = 1000ull * (cfg->wait_timeout_us ? cfg->wait_timeout_us : 200000u);
     p.drop_phase = -1; p.drop_block = -1;
